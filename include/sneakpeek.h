@@ -1,0 +1,187 @@
+/*
+ * sneakpeek.h -- C ABI of the B200 scoring-and-selection library.
+ *
+ * The library runs, on one GPU, the step an inference-serving scheduler repeats every round in
+ * SneakPeek (arXiv 2505.06641): it evaluates a SneakPeek model on every pending request to get a
+ * per-class posterior (Section 4.1), turns it into data-aware accuracies of every candidate model
+ * variant (Eq. 9), and then runs group-level greedy scheduling rounds (Eq. 12-14, Algorithm 1)
+ * with (model variant, batch size) candidates scored by the summed utility of Eq. 2.
+ *
+ * Conventions
+ *   - Every function returns an sp_status; nothing throws or aborts across this boundary.
+ *     sp_last_error() gives a text for the last non-OK status of a context.
+ *   - "HOST" / "DEVICE" in a comment says where a pointer must point.  Device pointers must belong
+ *     to the context's device.  Work is enqueued on the context's CUDA stream and is asynchronous
+ *     unless stated; sp_check() waits for it and reports errors found on the device.
+ *   - Times are int64 nanoseconds on one common clock.  Model ids are GLOBAL ids
+ *     g = (number of models of applications 0..a-1) + j for variant j of application a.
+ *   - The context owns the device memory it allocates; caller buffers stay the caller's.
+ *   - There is no CPU fallback: without a usable CUDA device every call fails with SP_ECUDA.
+ */
+#ifndef SNEAKPEEK_H_
+#define SNEAKPEEK_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sp_ctx sp_ctx; /* opaque */
+
+typedef enum {
+    SP_OK = 0,
+    SP_EINVAL = 1, /* bad argument, shape or value (also: bad value found on the device) */
+    SP_ENOMEM = 2, /* device or host allocation failed */
+    SP_ECUDA = 3,  /* a CUDA call failed */
+    SP_ESTATE = 4, /* call made in the wrong order (no profiles, no scored requests, ...) */
+    SP_ELIMIT = 5  /* a device-side iteration limit was hit; results are incomplete */
+} sp_status;
+
+enum { SP_F32 = 0, SP_BF16 = 1 };                       /* feature / head-weight storage type */
+enum { SP_PEN_STEP = 0 };                               /* penalty of Eq. 2: step function of Section 5.1 */
+enum { SP_PENDING = 0, SP_SCHEDULED = 1, SP_EXPIRED = 2 };
+
+/*
+ * Profiles registered for the applications (Section 2.2 / 3.2: per-label accuracy, inference
+ * latency and model-load latency of every variant) plus the SneakPeek model itself
+ * (Definition 4.1.1), here a linear head per application followed by a softmax, and the
+ * Dirichlet prior of Eq. 10.  All pointers are HOST pointers; the arrays are copied to the
+ * device during sp_load_profiles() and may be freed afterwards.
+ * With n_instances = I > 1 the context holds I independent schedulers that share the shapes
+ * below but have their own heads, profiles, clock and queues; every per-instance array then
+ * has a leading [I] axis.
+ */
+typedef struct {
+    int32_t n_instances;           /* I >= 1 */
+    int32_t n_apps;                /* A >= 1 applications (= request groups of Section 4.2) */
+    int32_t n_classes;             /* C >= 1 labels; an application with fewer labels pads with bias -inf, recall 0 */
+    int32_t feat_dim;              /* D >= 1 */
+    int32_t feat_dtype;            /* SP_F32 or SP_BF16: type of the features AND of head_w */
+    const int32_t *models_per_app; /* [A], each >= 1 (shared by all instances) */
+    const void *head_w;            /* [I][A][D][C], C fastest */
+    const float *head_b;           /* [I][A][C] */
+    const float *prior_alpha;      /* [I][A][C] Dirichlet hyper-parameters (Eq. 10), or NULL: theta = softmax output */
+    float evidence_k;              /* kappa > 0: the head's output p counts as evidence y = kappa * p in Eq. 11 */
+    const float *recall;           /* [I][sumM][C] per-model per-label accuracy in [0,1] */
+    const int64_t *lat_alpha_ns;   /* [I][sumM]  batch latency l(m,b) = alpha_m + beta_m * b, both >= 0 */
+    const int64_t *lat_beta_ns;    /* [I][sumM] */
+    const int64_t *swap_ns;        /* [I][sumM]  time to load model m when another model is resident, >= 0 */
+    const int32_t *batch_sizes;    /* [n_batch_sizes] strictly ascending, >= 1 (shared) */
+    int32_t n_batch_sizes;         /* 1..16 */
+    const int32_t *penalty_kind;   /* [A] SP_PEN_STEP (shared), or NULL = all step */
+    double prio_time_scale_s;      /* tau > 0 in exp(-(d - T)/tau) of Eq. 12, seconds */
+} sp_profiles;
+
+/* One executed batch (one greedy pick of Algorithm 1's loop). */
+typedef struct {
+    int32_t instance, round, app, model, batch, n_members, n_expired, exact;
+    int64_t t_start_ns, t_end_ns;
+    double utility;        /* summed Eq. 2 utility of the members */
+    double group_priority; /* Eq. 14 of the chosen application at t_start */
+} sp_round_rec;            /* 64 bytes.  batch = chosen allowed batch size, n_members = min(batch, live);
+                              n_expired = requests retired since the previous record; exact = bit 0: the
+                              application, bit 1: the candidate was decided by the fp64 re-evaluation */
+
+/* Per-request result: the schedule entry s_ij of Section 3.1 (model = j as a global id, order = s_ij). */
+typedef struct {
+    int32_t status; /* SP_PENDING / SP_SCHEDULED / SP_EXPIRED */
+    int32_t round;  /* round that scheduled or retired it, -1 while pending */
+    int32_t model;  /* global model id, -1 unless scheduled */
+    int32_t pad_;
+    int64_t order;  /* 1-based execution order inside its instance, 0 unless scheduled */
+} sp_req_rec;       /* 24 bytes */
+
+typedef struct {
+    int32_t trace_mode;   /* 0: every scored request is pending at once; 1: a request joins when arrival <= clock */
+    double guard_utility; /* relative margin under which candidate utilities are re-evaluated in fp64 (default 1e-4) */
+    double guard_priority;/* same for group priorities (default 2e-5) */
+} sp_options;
+
+typedef struct {
+    int64_t kernel_launches;   /* kernels this context has launched so far */
+    int64_t rounds;            /* rounds executed since the last sp_reset (all instances) */
+    int64_t exact_utility;     /* rounds whose candidate was decided in fp64 */
+    int64_t exact_priority;    /* rounds whose application was decided in fp64 */
+    int64_t exact_rows;        /* request rows re-scored in fp64 */
+} sp_stats;
+
+/* Creates a context on CUDA device `device` that enqueues on `cuda_stream` (a cudaStream_t; NULL = the
+ * legacy default stream).  *out is NULL on failure. */
+sp_status sp_create(sp_ctx **out, int device, void *cuda_stream);
+void sp_destroy(sp_ctx *ctx);
+const char *sp_last_error(const sp_ctx *ctx);
+
+/* Validates and uploads the profiles (synchronous).  Drops any scored requests.  Clocks start at 0 with no
+ * model resident.  SP_EINVAL on a bad shape/value, naming it in sp_last_error(). */
+sp_status sp_load_profiles(sp_ctx *ctx, const sp_profiles *profiles);
+
+sp_status sp_set_options(sp_ctx *ctx, const sp_options *opt);
+
+/* Sets the clock T and the resident model L (global id, -1 = none) of one instance, or of all (instance = -1). */
+sp_status sp_set_clock(sp_ctx *ctx, int32_t instance, int64_t t_ns, int32_t loaded_model);
+/* Same with per-instance values; t_ns [I], loaded_model [I] are DEVICE pointers. */
+sp_status sp_set_clocks(sp_ctx *ctx, const int64_t *t_ns, const int32_t *loaded_model);
+
+/*
+ * Scores n requests (Section 4.1 and Eq. 9, Eq. 12's variance factor) and makes them the context's request
+ * table with ids 0..n-1 (a second call without sp_reset() in between fails with SP_ESTATE).
+ * All pointers are DEVICE pointers and are BORROWED until sp_reset(), sp_load_profiles() or sp_destroy():
+ * the scheduler reads deadlines and, for near-ties, the raw features again.
+ *   feats       [n][D] row-major, float or bf16 as in the profiles; 16-byte aligned
+ *   app         [n] application of each request, 0..A-1
+ *   arrival_ns  [n]; deadline_ns [n]
+ *   instance    [n] instance of each request, non-decreasing; NULL when I == 1.  In trace mode arrivals
+ *               must be non-decreasing inside an instance.
+ *   acc_out     [n][Mmax] float, optional (NULL): receives the data-aware accuracies, columns >= M_app are 0.
+ * Violations found on the device (bad app/instance, order) surface as SP_EINVAL from sp_check().
+ */
+sp_status sp_score(sp_ctx *ctx, int64_t n, const void *feats, const int32_t *app, const int64_t *arrival_ns,
+                   const int64_t *deadline_ns, const int32_t *instance, float *acc_out);
+
+/* Copies scores of requests first..first+n-1 to DEVICE buffers: acc [n][Mmax] float and/or v [n] float
+ * (v = 1 + population variance of the request's accuracies); either may be NULL. */
+sp_status sp_get_scores(sp_ctx *ctx, int64_t first, int64_t n, float *acc, float *v);
+
+/*
+ * Runs up to max_rounds greedy rounds per instance back to back on the device (Algorithm 1's loop, one
+ * batch per round): arrivals join, hopeless requests are retired, the application with the highest
+ * Eq. 14 priority is chosen, every (model, batch size) candidate of it is scored by summed Eq. 2 utility,
+ * the best is emitted (ties: lowest application, lowest model, smallest batch), its members leave the
+ * queue, the clock advances by the batch latency (+ swap) and the model becomes resident.  An instance
+ * stops early when nothing is pending and no arrival is left.
+ *   rounds_out  DEVICE [I][cap] or NULL: record k of this call of instance i goes to rounds_out[i*cap + k], k < cap
+ *   n_done      DEVICE [I] or NULL: rounds executed by this call
+ */
+sp_status sp_schedule_round(sp_ctx *ctx, int32_t max_rounds, sp_round_rec *rounds_out, int64_t cap,
+                            int32_t *n_done);
+
+/* Copies the records of requests first..first+n-1 to a DEVICE buffer. */
+sp_status sp_get_requests(sp_ctx *ctx, int64_t first, int64_t n, sp_req_rec *out);
+/* Copies every instance's clock and resident model to DEVICE buffers t_ns [I], loaded_model [I]. */
+sp_status sp_get_clocks(sp_ctx *ctx, int64_t *t_ns, int32_t *loaded_model);
+
+/* Forgets the scored requests and queues; profiles, options, clocks and resident models stay. */
+sp_status sp_reset(sp_ctx *ctx);
+
+/* Waits for the context's stream and returns the first error recorded on the device since the last
+ * sp_check(): SP_EINVAL (bad request data), SP_ELIMIT (iteration limit), else SP_OK. */
+sp_status sp_check(sp_ctx *ctx);
+sp_status sp_get_stats(sp_ctx *ctx, sp_stats *out /* HOST */);
+
+/*
+ * Whole path from HOST buffers: uploads the requests, scores them, runs every instance to completion
+ * (at most max_rounds rounds each), downloads the results, and waits.  Replaces the request table.
+ * feats/app/arrival_ns/deadline_ns/instance as in sp_score() but HOST pointers (pinned memory makes the
+ * copies faster); t0_ns [I] and loaded0 [I] (NULL = keep) are the starting clocks and resident models.
+ * Outputs, all HOST and optional: reqs_out [n], rounds_out [I][cap], n_done [I].
+ */
+sp_status sp_run_host(sp_ctx *ctx, int64_t n, const void *feats, const int32_t *app, const int64_t *arrival_ns,
+                      const int64_t *deadline_ns, const int32_t *instance, const int64_t *t0_ns,
+                      const int32_t *loaded0, int32_t max_rounds, sp_req_rec *reqs_out,
+                      sp_round_rec *rounds_out, int64_t cap, int32_t *n_done);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SNEAKPEEK_H_ */

@@ -1,0 +1,550 @@
+// C ABI of the scoring-and-selection library: context, validation, device buffers, kernel launches.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "sp_common.cuh"
+#include "sp_group.cuh"
+#include "sp_score_small.cuh"
+#include "sp_score_tiled.cuh"
+#include "sp_sched.cuh"
+
+using namespace sp;
+
+namespace {
+
+struct Buf {                     // a device allocation that only grows
+    void *p = nullptr;
+    size_t bytes = 0;
+};
+
+struct HostProfiles {            // host copies of the shared (small) profile arrays
+    std::vector<int32_t> models_per_app, batch_sizes;
+};
+
+}  // namespace
+
+struct sp_ctx {
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    std::string err;
+    bool have_profiles = false;
+    bool have_table = false;
+    HostProfiles hp;
+    DevProfiles P{};
+    DevTable tb{};
+    sp_options opt{0, 1e-4, 2e-5};
+    int64_t launches = 0;
+    int sched_threads = 1024;
+    int small_ct = 0;            // labels per lane of the small-head kernel, 0 = use the tiled kernel
+    size_t small_smem = 0;
+    // profile buffers
+    Buf W, bias, recall, prior, prior_dot, prior_sum, lat_alpha, lat_beta, swap;
+    // per-instance state and scratch
+    Buf state, zbuf, flags, stats, cnt, gstart, cursor, small_start, tiled_start;
+    // per-request buffers
+    Buf acc32, v32, acc64, v64, exact, recs, perm, q_id0, q_id1, q_dl0, q_dl1, q_pw0, q_pw1, sort_scratch;
+    // staging of sp_run_host
+    Buf h_feats, h_app, h_arrival, h_deadline, h_instance, h_t0, h_loaded, h_rounds, h_ndone;
+};
+
+namespace {
+
+sp_status fail(sp_ctx *c, sp_status s, const std::string &msg) {
+    if (c) c->err = msg;
+    return s;
+}
+
+#define SP_CUDA(ctx, call)                                                                           \
+    do {                                                                                             \
+        cudaError_t e_ = (call);                                                                     \
+        if (e_ != cudaSuccess)                                                                       \
+            return fail(ctx, e_ == cudaErrorMemoryAllocation ? SP_ENOMEM : SP_ECUDA,                 \
+                        std::string(#call) + ": " + cudaGetErrorString(e_));                         \
+    } while (0)
+
+sp_status ensure(sp_ctx *c, Buf &b, size_t bytes) {
+    if (bytes <= b.bytes && b.p) return SP_OK;
+    if (bytes == 0) bytes = 16;
+    if (b.p) {
+        SP_CUDA(c, cudaStreamSynchronize(c->stream));
+        SP_CUDA(c, cudaFree(b.p));
+        b.p = nullptr; b.bytes = 0;
+    }
+    SP_CUDA(c, cudaMalloc(&b.p, bytes));
+    b.bytes = bytes;
+    return SP_OK;
+}
+
+void release(Buf &b) {
+    if (b.p) cudaFree(b.p);
+    b.p = nullptr; b.bytes = 0;
+}
+
+#define SP_TRY(expr)                       \
+    do {                                   \
+        sp_status s_ = (expr);             \
+        if (s_ != SP_OK) return s_;        \
+    } while (0)
+
+sp_status upload(sp_ctx *c, Buf &b, const void *host, size_t bytes) {
+    SP_TRY(ensure(c, b, bytes));
+    SP_CUDA(c, cudaMemcpyAsync(b.p, host, bytes, cudaMemcpyHostToDevice, c->stream));
+    return SP_OK;
+}
+
+sp_status launched(sp_ctx *c, const char *what) {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(c, SP_ECUDA, std::string(what) + ": " + cudaGetErrorString(e));
+    ++c->launches;
+    return SP_OK;
+}
+
+// mode 0: full reset (clock 0, nothing resident); mode 1: forget queues, keep clock and resident model
+__global__ void k_state_reset(InstState *st, int n_inst, int mode) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_inst) return;
+    InstState s = st[i];
+    if (mode == 0) { s.T = 0; s.L = -1; }
+    s.next_order = 1; s.Tref = 0; s.inserted = 0; s.round = 0; s.exp_since = 0; s.started = 0;
+    for (int a = 0; a < kMaxApps; ++a) { s.head[a] = 0; s.tail[a] = 0; s.cur[a] = 0; }
+    st[i] = s;
+}
+
+__global__ void k_set_clock(InstState *st, int n_inst, int only, int64_t t, int32_t loaded) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_inst || (only >= 0 && i != only)) return;
+    st[i].T = t; st[i].L = loaded;
+}
+
+// per-instance values; a null vector keeps what is there
+__global__ void k_set_clocks(InstState *st, int n_inst, const int64_t *tv, const int32_t *lv) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_inst) return;
+    if (tv) st[i].T = tv[i];
+    if (lv) st[i].L = lv[i];
+}
+
+__global__ void k_get_clock(const InstState *st, int n_inst, int64_t *t, int32_t *l) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_inst) return;
+    if (t) t[i] = st[i].T;
+    if (l) l[i] = st[i].L;
+}
+
+__global__ void k_init_requests(sp_req_rec *recs, unsigned char *exact, int64_t n) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    sp_req_rec r; r.status = SP_PENDING; r.round = -1; r.model = -1; r.pad_ = 0; r.order = 0;
+    recs[i] = r;
+    exact[i] = 0;
+}
+
+int small_ct_for(int C) { return C <= 10 ? 5 : C <= 20 ? 10 : C <= 32 ? 16 : C <= 64 ? 32 : 0; }
+
+template <int CT>
+sp_status launch_small(sp_ctx *c, int grid, float *acc_out) {
+    auto kern = k_score_small<CT>;
+    SP_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->small_smem));
+    kern<<<grid, kSmallThreads, c->small_smem, c->stream>>>(c->P, c->tb, (const int32_t *)c->small_start.p, acc_out,
+                                                            (const int *)c->flags.p);
+    return launched(c, "k_score_small");
+}
+
+}  // namespace
+
+// =================================================================================================
+extern "C" {
+
+sp_status sp_create(sp_ctx **out, int device, void *cuda_stream) {
+    if (!out) return SP_EINVAL;
+    *out = nullptr;
+    int n_dev = 0;
+    if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device < 0 || device >= n_dev) return SP_ECUDA;
+    if (cudaSetDevice(device) != cudaSuccess) return SP_ECUDA;
+    sp_ctx *c = new (std::nothrow) sp_ctx();
+    if (!c) return SP_ENOMEM;
+    c->device = device;
+    c->stream = (cudaStream_t)cuda_stream;
+    if (ensure(c, c->flags, 2 * sizeof(int)) != SP_OK || ensure(c, c->stats, 4 * sizeof(unsigned long long)) != SP_OK ||
+        cudaMemsetAsync(c->flags.p, 0, 2 * sizeof(int), c->stream) != cudaSuccess ||
+        cudaMemsetAsync(c->stats.p, 0, 4 * sizeof(unsigned long long), c->stream) != cudaSuccess) {
+        delete c;
+        return SP_ECUDA;
+    }
+    *out = c;
+    return SP_OK;
+}
+
+void sp_destroy(sp_ctx *c) {
+    if (!c) return;
+    cudaSetDevice(c->device);
+    cudaStreamSynchronize(c->stream);
+    Buf *all[] = {&c->W, &c->bias, &c->recall, &c->prior, &c->prior_dot, &c->prior_sum, &c->lat_alpha, &c->lat_beta,
+                  &c->swap, &c->state, &c->zbuf, &c->flags, &c->stats, &c->cnt, &c->gstart, &c->cursor,
+                  &c->small_start, &c->tiled_start, &c->acc32, &c->v32, &c->acc64, &c->v64, &c->exact, &c->recs,
+                  &c->perm, &c->q_id0, &c->q_id1, &c->q_dl0, &c->q_dl1, &c->q_pw0, &c->q_pw1, &c->sort_scratch,
+                  &c->h_feats, &c->h_app, &c->h_arrival, &c->h_deadline, &c->h_instance, &c->h_t0, &c->h_loaded,
+                  &c->h_rounds, &c->h_ndone};
+    for (Buf *b : all) release(*b);
+    delete c;
+}
+
+const char *sp_last_error(const sp_ctx *c) { return c ? c->err.c_str() : "null context"; }
+
+sp_status sp_load_profiles(sp_ctx *c, const sp_profiles *p) {
+    if (!c) return SP_EINVAL;
+    if (!p) return fail(c, SP_EINVAL, "profiles is NULL");
+    SP_CUDA(c, cudaSetDevice(c->device));
+    const int I = p->n_instances, A = p->n_apps, C = p->n_classes, D = p->feat_dim, nB = p->n_batch_sizes;
+    if (I < 1) return fail(c, SP_EINVAL, "n_instances must be >= 1");
+    if (A < 1 || A > kMaxApps) return fail(c, SP_EINVAL, "n_apps must be 1..16");
+    if (C < 1 || C > kMaxClasses) return fail(c, SP_EINVAL, "n_classes must be 1..4096");
+    if (D < 1) return fail(c, SP_EINVAL, "feat_dim must be >= 1");
+    if (p->feat_dtype != SP_F32 && p->feat_dtype != SP_BF16) return fail(c, SP_EINVAL, "feat_dtype must be SP_F32 or SP_BF16");
+    if (nB < 1 || nB > kMaxBatchSizes) return fail(c, SP_EINVAL, "n_batch_sizes must be 1..16");
+    if (!p->models_per_app || !p->head_w || !p->head_b || !p->recall || !p->lat_alpha_ns || !p->lat_beta_ns ||
+        !p->swap_ns || !p->batch_sizes)
+        return fail(c, SP_EINVAL, "a required profile array is NULL");
+    if (!(p->prio_time_scale_s > 0.0) || !std::isfinite(p->prio_time_scale_s))
+        return fail(c, SP_EINVAL, "prio_time_scale_s must be positive and finite");
+    int sumM = 0, Mmax = 0;
+    for (int a = 0; a < A; ++a) {
+        const int m = p->models_per_app[a];
+        if (m < 1 || m > kMaxModelsPerApp) return fail(c, SP_EINVAL, "models_per_app entries must be 1..16");
+        sumM += m; Mmax = m > Mmax ? m : Mmax;
+    }
+    for (int b = 0; b < nB; ++b) {
+        if (p->batch_sizes[b] < 1 || p->batch_sizes[b] > kMaxBatch || (b && p->batch_sizes[b] <= p->batch_sizes[b - 1]))
+            return fail(c, SP_EINVAL, "batch_sizes must be strictly ascending in 1..1024");
+    }
+    if (p->penalty_kind)
+        for (int a = 0; a < A; ++a)
+            if (p->penalty_kind[a] != SP_PEN_STEP) return fail(c, SP_EINVAL, "only the step penalty is implemented");
+    const int64_t n_models = (int64_t)I * sumM;
+    const int64_t lat_limit = (int64_t)1 << 50;
+    for (int64_t k = 0; k < n_models; ++k) {
+        const int64_t al = p->lat_alpha_ns[k], be = p->lat_beta_ns[k], sw = p->swap_ns[k];
+        if (al < 0 || be < 0 || sw < 0 || al > lat_limit || be > lat_limit / kMaxBatch || sw > lat_limit)
+            return fail(c, SP_EINVAL, "latency and swap profiles must be in [0, 2^50] ns");
+    }
+    for (int64_t k = 0; k < n_models * C; ++k)
+        if (!(p->recall[k] >= 0.f && p->recall[k] <= 1.f)) return fail(c, SP_EINVAL, "recall must be in [0,1]");
+    if (p->prior_alpha) {
+        if (!(p->evidence_k > 0.f)) return fail(c, SP_EINVAL, "evidence_k must be > 0 when a prior is given");
+        for (int64_t k = 0; k < (int64_t)I * A * C; ++k)
+            if (!(p->prior_alpha[k] >= 0.f) || !std::isfinite(p->prior_alpha[k]))
+                return fail(c, SP_EINVAL, "prior_alpha must be finite and >= 0");
+    }
+    // shared memory the scheduler kernel needs for its candidate tables (sort buffer is sized at launch)
+    const int bmax = p->batch_sizes[nB - 1];
+    const SchedSmem ss(0, Mmax, bmax, kMaxModelsPerApp * kMaxBatchSizes);
+    if (ss.end > 96 * 1024) return fail(c, SP_EINVAL, "models_per_app x largest batch size is too large for one block");
+
+    c->have_profiles = false;
+    c->have_table = false;
+    c->hp.models_per_app.assign(p->models_per_app, p->models_per_app + A);
+    c->hp.batch_sizes.assign(p->batch_sizes, p->batch_sizes + nB);
+    const size_t esz = p->feat_dtype == SP_BF16 ? 2 : 4;
+    SP_TRY(upload(c, c->W, p->head_w, (size_t)I * A * D * C * esz));
+    SP_TRY(upload(c, c->bias, p->head_b, (size_t)I * A * C * 4));
+    SP_TRY(upload(c, c->recall, p->recall, (size_t)n_models * C * 4));
+    SP_TRY(upload(c, c->lat_alpha, p->lat_alpha_ns, (size_t)n_models * 8));
+    SP_TRY(upload(c, c->lat_beta, p->lat_beta_ns, (size_t)n_models * 8));
+    SP_TRY(upload(c, c->swap, p->swap_ns, (size_t)n_models * 8));
+    std::vector<float> pdot, psum;
+    if (p->prior_alpha) {
+        // sum_c alpha_c recall[m][c] and sum_c alpha_c: the prior's share of Eq. 9 under the posterior mean
+        pdot.resize((size_t)n_models); psum.resize((size_t)I * A);
+        for (int i = 0; i < I; ++i) {
+            int g = 0;
+            for (int a = 0; a < A; ++a) {
+                const float *al = p->prior_alpha + ((size_t)i * A + a) * C;
+                double s = 0.0;
+                for (int k = 0; k < C; ++k) s += (double)al[k];
+                psum[(size_t)i * A + a] = (float)s;
+                for (int j = 0; j < p->models_per_app[a]; ++j, ++g) {
+                    const float *r = p->recall + ((size_t)i * sumM + g) * C;
+                    double t = 0.0;
+                    for (int k = 0; k < C; ++k) t += (double)al[k] * (double)r[k];
+                    pdot[(size_t)i * sumM + g] = (float)t;
+                }
+            }
+        }
+        SP_TRY(upload(c, c->prior, p->prior_alpha, (size_t)I * A * C * 4));
+        SP_TRY(upload(c, c->prior_dot, pdot.data(), pdot.size() * 4));
+        SP_TRY(upload(c, c->prior_sum, psum.data(), psum.size() * 4));
+    }
+    DevProfiles &P = c->P;
+    P = DevProfiles{};
+    P.I = I; P.A = A; P.C = C; P.D = D; P.dtype = p->feat_dtype; P.sumM = sumM; P.Mmax = Mmax; P.nB = nB;
+    P.W = c->W.p; P.bias = (const float *)c->bias.p; P.recall = (const float *)c->recall.p;
+    P.prior = p->prior_alpha ? (const float *)c->prior.p : nullptr;
+    P.prior_dot = p->prior_alpha ? (const float *)c->prior_dot.p : nullptr;
+    P.prior_sum = p->prior_alpha ? (const float *)c->prior_sum.p : nullptr;
+    P.kappa = p->evidence_k;
+    P.lat_alpha = (const int64_t *)c->lat_alpha.p; P.lat_beta = (const int64_t *)c->lat_beta.p;
+    P.swap = (const int64_t *)c->swap.p;
+    P.tau = p->prio_time_scale_s;
+    for (int a = 0, g = 0; a <= A; ++a) { P.mfirst[a] = g; if (a < A) g += p->models_per_app[a]; }
+    for (int b = 0; b < nB; ++b) P.batch[b] = p->batch_sizes[b];
+
+    // kernel choices that depend on the shapes only
+    c->sched_threads = I > 1 ? 128 : 1024;
+    c->small_ct = 0;
+    if (p->feat_dtype == SP_F32 && D % 4 == 0 && C <= 64) {
+        const int ct = small_ct_for(C);
+        const SmallSmem L(A, D, sumM, (ct + 3) & ~3);
+        const size_t bytes = (size_t)L.end * sizeof(float);
+        if (bytes <= 200 * 1024) { c->small_ct = ct; c->small_smem = bytes; }
+    }
+    const size_t nkeys = (size_t)I * A;
+    SP_TRY(ensure(c, c->state, (size_t)I * sizeof(InstState)));
+    SP_TRY(ensure(c, c->zbuf, (size_t)I * (c->sched_threads / 32) * C * sizeof(double)));
+    SP_TRY(ensure(c, c->cnt, nkeys * 4));
+    SP_TRY(ensure(c, c->cursor, nkeys * 4));
+    SP_TRY(ensure(c, c->gstart, (nkeys + 1) * 8));
+    SP_TRY(ensure(c, c->tiled_start, (nkeys + 1) * 4));
+    SP_TRY(ensure(c, c->small_start, ((size_t)I + 1) * 4));
+    SP_CUDA(c, cudaMemsetAsync(c->state.p, 0, (size_t)I * sizeof(InstState), c->stream));
+    k_state_reset<<<(I + 255) / 256, 256, 0, c->stream>>>((InstState *)c->state.p, I, 0);
+    SP_TRY(launched(c, "k_state_reset"));
+    SP_CUDA(c, cudaMemsetAsync(c->flags.p, 0, 2 * sizeof(int), c->stream));
+    SP_CUDA(c, cudaStreamSynchronize(c->stream));   // the host arrays may be freed on return
+    c->have_profiles = true;
+    return SP_OK;
+}
+
+sp_status sp_set_options(sp_ctx *c, const sp_options *o) {
+    if (!c) return SP_EINVAL;
+    if (!o || !(o->guard_utility >= 0.0) || !(o->guard_priority >= 0.0) || o->guard_utility > 1.0 || o->guard_priority > 1.0)
+        return fail(c, SP_EINVAL, "guards must be in [0,1]");
+    if (c->have_table && (o->trace_mode != 0) != (c->opt.trace_mode != 0))
+        return fail(c, SP_ESTATE, "trace_mode cannot change while requests are scored; call sp_reset first");
+    c->opt = *o;
+    return SP_OK;
+}
+
+sp_status sp_set_clock(sp_ctx *c, int32_t instance, int64_t t_ns, int32_t loaded) {
+    if (!c) return SP_EINVAL;
+    if (!c->have_profiles) return fail(c, SP_ESTATE, "no profiles loaded");
+    if (instance < -1 || instance >= c->P.I || loaded < -1 || loaded >= c->P.sumM)
+        return fail(c, SP_EINVAL, "instance or model id out of range");
+    SP_CUDA(c, cudaSetDevice(c->device));
+    k_set_clock<<<(c->P.I + 255) / 256, 256, 0, c->stream>>>((InstState *)c->state.p, c->P.I, instance, t_ns, loaded);
+    return launched(c, "k_set_clock");
+}
+
+sp_status sp_set_clocks(sp_ctx *c, const int64_t *t_ns, const int32_t *loaded) {
+    if (!c) return SP_EINVAL;
+    if (!c->have_profiles) return fail(c, SP_ESTATE, "no profiles loaded");
+    SP_CUDA(c, cudaSetDevice(c->device));
+    k_set_clocks<<<(c->P.I + 255) / 256, 256, 0, c->stream>>>((InstState *)c->state.p, c->P.I, t_ns, loaded);
+    return launched(c, "k_set_clocks");
+}
+
+sp_status sp_get_clocks(sp_ctx *c, int64_t *t_ns, int32_t *loaded) {
+    if (!c) return SP_EINVAL;
+    if (!c->have_profiles) return fail(c, SP_ESTATE, "no profiles loaded");
+    SP_CUDA(c, cudaSetDevice(c->device));
+    k_get_clock<<<(c->P.I + 255) / 256, 256, 0, c->stream>>>((const InstState *)c->state.p, c->P.I, t_ns, loaded);
+    return launched(c, "k_get_clock");
+}
+
+sp_status sp_reset(sp_ctx *c) {
+    if (!c) return SP_EINVAL;
+    if (!c->have_profiles) return fail(c, SP_ESTATE, "no profiles loaded");
+    SP_CUDA(c, cudaSetDevice(c->device));
+    k_state_reset<<<(c->P.I + 255) / 256, 256, 0, c->stream>>>((InstState *)c->state.p, c->P.I, 1);
+    SP_TRY(launched(c, "k_state_reset"));
+    SP_CUDA(c, cudaMemsetAsync((int *)c->flags.p + 1, 0, sizeof(int), c->stream));
+    SP_CUDA(c, cudaMemsetAsync(c->stats.p, 0, 4 * sizeof(unsigned long long), c->stream));
+    c->have_table = false;
+    c->tb.n = 0;
+    return SP_OK;
+}
+
+sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, const int64_t *arrival_ns,
+                   const int64_t *deadline_ns, const int32_t *instance, float *acc_out) {
+    if (!c) return SP_EINVAL;
+    if (!c->have_profiles) return fail(c, SP_ESTATE, "no profiles loaded");
+    if (c->have_table) return fail(c, SP_ESTATE, "requests already scored; call sp_reset first");
+    if (n < 0 || n > ((int64_t)1 << 40)) return fail(c, SP_EINVAL, "n out of range");
+    if (n > 0 && (!feats || !app || !arrival_ns || !deadline_ns)) return fail(c, SP_EINVAL, "a request array is NULL");
+    if (c->P.I > 1 && n > 0 && !instance) return fail(c, SP_EINVAL, "instance is required when n_instances > 1");
+    if (((uintptr_t)feats & 15) != 0) return fail(c, SP_EINVAL, "feats must be 16-byte aligned");
+    SP_CUDA(c, cudaSetDevice(c->device));
+    const DevProfiles &P = c->P;
+    const size_t nn = (size_t)(n > 0 ? n : 1), nkeys = (size_t)P.I * P.A;
+    SP_TRY(ensure(c, c->acc32, nn * P.Mmax * 4));
+    SP_TRY(ensure(c, c->v32, nn * 4));
+    SP_TRY(ensure(c, c->acc64, nn * P.Mmax * 8));
+    SP_TRY(ensure(c, c->v64, nn * 8));
+    SP_TRY(ensure(c, c->exact, nn));
+    SP_TRY(ensure(c, c->recs, nn * sizeof(sp_req_rec)));
+    SP_TRY(ensure(c, c->perm, nn * 8));
+    SP_TRY(ensure(c, c->q_id0, nn * 8));
+    SP_TRY(ensure(c, c->q_id1, nn * 8));
+    SP_TRY(ensure(c, c->q_dl0, nn * 8));
+    SP_TRY(ensure(c, c->q_dl1, nn * 8));
+    SP_TRY(ensure(c, c->q_pw0, nn * 8));
+    SP_TRY(ensure(c, c->q_pw1, nn * 8));
+    SP_TRY(ensure(c, c->sort_scratch, nn * sizeof(SortKey)));
+    DevTable &tb = c->tb;
+    tb.n = n; tb.feats = feats; tb.app = app; tb.arrival = arrival_ns; tb.deadline = deadline_ns;
+    tb.instance = P.I > 1 ? instance : nullptr;
+    tb.acc32 = (float *)c->acc32.p; tb.v32 = (float *)c->v32.p; tb.acc64 = (double *)c->acc64.p;
+    tb.v64 = (double *)c->v64.p; tb.exact = (unsigned char *)c->exact.p; tb.recs = (sp_req_rec *)c->recs.p;
+    tb.cnt = (int32_t *)c->cnt.p; tb.gstart = (int64_t *)c->gstart.p; tb.perm = (int64_t *)c->perm.p;
+    tb.cursor = (int32_t *)c->cursor.p;
+
+    SP_CUDA(c, cudaMemsetAsync(tb.cnt, 0, nkeys * 4, c->stream));
+    SP_CUDA(c, cudaMemsetAsync(tb.cursor, 0, nkeys * 4, c->stream));
+    const unsigned gb = (unsigned)((n + 255) / 256);
+    if (n > 0) {
+        k_init_requests<<<gb, 256, 0, c->stream>>>(tb.recs, tb.exact, n);
+        SP_TRY(launched(c, "k_init_requests"));
+        k_group_count<<<gb, 256, 0, c->stream>>>(P, tb, c->opt.trace_mode, (int *)c->flags.p);
+        SP_TRY(launched(c, "k_group_count"));
+    }
+    k_group_scan<<<1, 1024, 0, c->stream>>>((int)nkeys, P.A, tb.cnt, tb.gstart, (int32_t *)c->tiled_start.p,
+                                            (int32_t *)c->small_start.p);
+    SP_TRY(launched(c, "k_group_scan"));
+    if (n > 0) {
+        if (c->small_ct) {
+            const int grid = (int)(n / kSmallRows + P.I);
+            switch (c->small_ct) {
+                case 5: SP_TRY(launch_small<5>(c, grid, acc_out)); break;
+                case 10: SP_TRY(launch_small<10>(c, grid, acc_out)); break;
+                case 16: SP_TRY(launch_small<16>(c, grid, acc_out)); break;
+                default: SP_TRY(launch_small<32>(c, grid, acc_out)); break;
+            }
+        } else {
+            k_group_scatter<<<gb, 256, 0, c->stream>>>(P, tb, (const int *)c->flags.p);
+            SP_TRY(launched(c, "k_group_scatter"));
+            const int grid = (int)(n / kTiledRows + (int64_t)nkeys);
+            if (P.dtype == SP_BF16)
+                k_score_tiled<true><<<grid, kTiledThreads, 0, c->stream>>>(P, tb, (const int32_t *)c->tiled_start.p, acc_out,
+                                                                        (const int *)c->flags.p);
+            else
+                k_score_tiled<false><<<grid, kTiledThreads, 0, c->stream>>>(P, tb, (const int32_t *)c->tiled_start.p, acc_out,
+                                                                         (const int *)c->flags.p);
+            SP_TRY(launched(c, "k_score_tiled"));
+        }
+    }
+    c->have_table = true;
+    return SP_OK;
+}
+
+sp_status sp_get_scores(sp_ctx *c, int64_t first, int64_t n, float *acc, float *v) {
+    if (!c) return SP_EINVAL;
+    if (!c->have_table) return fail(c, SP_ESTATE, "no scored requests");
+    if (first < 0 || n < 0 || first + n > c->tb.n) return fail(c, SP_EINVAL, "request range out of bounds");
+    SP_CUDA(c, cudaSetDevice(c->device));
+    if (acc && n)
+        SP_CUDA(c, cudaMemcpyAsync(acc, c->tb.acc32 + first * c->P.Mmax, (size_t)n * c->P.Mmax * 4, cudaMemcpyDeviceToDevice, c->stream));
+    if (v && n) SP_CUDA(c, cudaMemcpyAsync(v, c->tb.v32 + first, (size_t)n * 4, cudaMemcpyDeviceToDevice, c->stream));
+    return SP_OK;
+}
+
+sp_status sp_get_requests(sp_ctx *c, int64_t first, int64_t n, sp_req_rec *out) {
+    if (!c) return SP_EINVAL;
+    if (!c->have_table) return fail(c, SP_ESTATE, "no scored requests");
+    if (first < 0 || n < 0 || first + n > c->tb.n || (n && !out)) return fail(c, SP_EINVAL, "request range out of bounds");
+    SP_CUDA(c, cudaSetDevice(c->device));
+    if (n) SP_CUDA(c, cudaMemcpyAsync(out, c->tb.recs + first, (size_t)n * sizeof(sp_req_rec), cudaMemcpyDeviceToDevice, c->stream));
+    return SP_OK;
+}
+
+sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_out, int64_t cap, int32_t *n_done) {
+    if (!c) return SP_EINVAL;
+    if (!c->have_table) return fail(c, SP_ESTATE, "no scored requests");
+    if (max_rounds < 0 || cap < 0) return fail(c, SP_EINVAL, "max_rounds and cap must be >= 0");
+    SP_CUDA(c, cudaSetDevice(c->device));
+    const DevProfiles &P = c->P;
+    SchedParams sp{};
+    sp.P = P; sp.tb = c->tb; sp.state = (InstState *)c->state.p;
+    sp.q_id[0] = (int64_t *)c->q_id0.p; sp.q_id[1] = (int64_t *)c->q_id1.p;
+    sp.q_dl[0] = (int64_t *)c->q_dl0.p; sp.q_dl[1] = (int64_t *)c->q_dl1.p;
+    sp.q_pw[0] = (double *)c->q_pw0.p; sp.q_pw[1] = (double *)c->q_pw1.p;
+    sp.sort_scratch = (SortKey *)c->sort_scratch.p; sp.zbuf = (double *)c->zbuf.p;
+    sp.flags = (int *)c->flags.p; sp.stats = (unsigned long long *)c->stats.p;
+    sp.trace_mode = c->opt.trace_mode; sp.guard_u = c->opt.guard_utility; sp.guard_p = c->opt.guard_priority;
+    sp.max_rounds = max_rounds; sp.rounds_out = rounds_out; sp.cap = rounds_out ? cap : 0; sp.n_done = n_done;
+    sp.bmax = P.batch[P.nB - 1];
+    // shared-memory sort buffer: whole instance when it fits, else the global scratch takes over
+    const int64_t per_inst = P.I > 1 ? (c->tb.n + P.I - 1) / P.I * 2 : c->tb.n;
+    int sort_cap = P.I > 1 ? 1024 : 8192;
+    while (sort_cap > 64 && sort_cap / 2 >= per_inst) sort_cap /= 2;
+    sp.sort_cap = sort_cap;
+    const SchedSmem L(sort_cap, P.Mmax, sp.bmax, kMaxModelsPerApp * kMaxBatchSizes);
+    SP_CUDA(c, cudaFuncSetAttribute(k_sched, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.end));
+    k_sched<<<P.I, c->sched_threads, L.end, c->stream>>>(sp);
+    return launched(c, "k_sched");
+}
+
+sp_status sp_check(sp_ctx *c) {
+    if (!c) return SP_EINVAL;
+    SP_CUDA(c, cudaSetDevice(c->device));
+    int flags[2] = {0, 0};
+    SP_CUDA(c, cudaMemcpyAsync(flags, c->flags.p, sizeof flags, cudaMemcpyDeviceToHost, c->stream));
+    SP_CUDA(c, cudaStreamSynchronize(c->stream));
+    if (flags[0] != kDevOk) SP_CUDA(c, cudaMemsetAsync(c->flags.p, 0, sizeof(int), c->stream));
+    if (flags[0] == kDevLimit) return fail(c, SP_ELIMIT, "a device-side iteration limit was hit");
+    if (flags[0] == kDevBadRequest)
+        return fail(c, SP_EINVAL, "request arrays rejected on the device (app/instance out of range or not ordered)");
+    return SP_OK;
+}
+
+sp_status sp_get_stats(sp_ctx *c, sp_stats *out) {
+    if (!c || !out) return SP_EINVAL;
+    SP_CUDA(c, cudaSetDevice(c->device));
+    unsigned long long s[4];
+    SP_CUDA(c, cudaMemcpyAsync(s, c->stats.p, sizeof s, cudaMemcpyDeviceToHost, c->stream));
+    SP_CUDA(c, cudaStreamSynchronize(c->stream));
+    out->kernel_launches = c->launches;
+    out->rounds = (int64_t)s[0]; out->exact_utility = (int64_t)s[1]; out->exact_priority = (int64_t)s[2];
+    out->exact_rows = (int64_t)s[3];
+    return SP_OK;
+}
+
+sp_status sp_run_host(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, const int64_t *arrival_ns,
+                      const int64_t *deadline_ns, const int32_t *instance, const int64_t *t0_ns,
+                      const int32_t *loaded0, int32_t max_rounds, sp_req_rec *reqs_out, sp_round_rec *rounds_out,
+                      int64_t cap, int32_t *n_done) {
+    if (!c) return SP_EINVAL;
+    if (!c->have_profiles) return fail(c, SP_ESTATE, "no profiles loaded");
+    if (n < 0 || (n > 0 && (!feats || !app || !arrival_ns || !deadline_ns))) return fail(c, SP_EINVAL, "a request array is NULL");
+    if (c->P.I > 1 && n > 0 && !instance) return fail(c, SP_EINVAL, "instance is required when n_instances > 1");
+    if (cap < 0 || max_rounds < 0) return fail(c, SP_EINVAL, "max_rounds and cap must be >= 0");
+    SP_CUDA(c, cudaSetDevice(c->device));
+    const DevProfiles &P = c->P;
+    const size_t esz = P.dtype == SP_BF16 ? 2 : 4;
+    SP_TRY(sp_reset(c));
+    SP_TRY(upload(c, c->h_feats, feats, (size_t)n * P.D * esz));
+    SP_TRY(upload(c, c->h_app, app, (size_t)n * 4));
+    SP_TRY(upload(c, c->h_arrival, arrival_ns, (size_t)n * 8));
+    SP_TRY(upload(c, c->h_deadline, deadline_ns, (size_t)n * 8));
+    if (P.I > 1) SP_TRY(upload(c, c->h_instance, instance, (size_t)n * 4));
+    if (t0_ns) SP_TRY(upload(c, c->h_t0, t0_ns, (size_t)P.I * 8));
+    if (loaded0) SP_TRY(upload(c, c->h_loaded, loaded0, (size_t)P.I * 4));
+    if (t0_ns || loaded0)
+        SP_TRY(sp_set_clocks(c, t0_ns ? (const int64_t *)c->h_t0.p : nullptr, loaded0 ? (const int32_t *)c->h_loaded.p : nullptr));
+    SP_TRY(sp_score(c, n, c->h_feats.p, (const int32_t *)c->h_app.p, (const int64_t *)c->h_arrival.p,
+                    (const int64_t *)c->h_deadline.p, P.I > 1 ? (const int32_t *)c->h_instance.p : nullptr, nullptr));
+    const bool want_rounds = rounds_out && cap > 0;
+    if (want_rounds) SP_TRY(ensure(c, c->h_rounds, (size_t)P.I * cap * sizeof(sp_round_rec)));
+    SP_TRY(ensure(c, c->h_ndone, (size_t)P.I * 4));
+    SP_TRY(sp_schedule_round(c, max_rounds, want_rounds ? (sp_round_rec *)c->h_rounds.p : nullptr, cap, (int32_t *)c->h_ndone.p));
+    if (reqs_out && n)
+        SP_CUDA(c, cudaMemcpyAsync(reqs_out, c->tb.recs, (size_t)n * sizeof(sp_req_rec), cudaMemcpyDeviceToHost, c->stream));
+    if (want_rounds)
+        SP_CUDA(c, cudaMemcpyAsync(rounds_out, c->h_rounds.p, (size_t)P.I * cap * sizeof(sp_round_rec), cudaMemcpyDeviceToHost, c->stream));
+    if (n_done) SP_CUDA(c, cudaMemcpyAsync(n_done, c->h_ndone.p, (size_t)P.I * 4, cudaMemcpyDeviceToHost, c->stream));
+    return sp_check(c);
+}
+
+}  // extern "C"

@@ -1,0 +1,104 @@
+// Grouping pass of sp_score(): validates the request arrays and counts / orders requests by
+// (instance, application).  The counts size every application's queue region; the permutation
+// feeds the tiled scoring kernel, which needs tiles of requests that share one head.
+#pragma once
+
+#include "sp_common.cuh"
+
+namespace sp {
+
+constexpr int kTiledRows = 64;    // requests per tile of the tiled scoring kernel
+constexpr int kSmallRows = 128;   // requests per tile of the small-head scoring kernel
+
+// flags[0]: device status (DevErr), flags[1]: 1 when the request table failed validation.
+__global__ void k_group_count(DevProfiles P, DevTable tb, int trace_mode, int *flags) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= tb.n) return;
+    const int a = tb.app[i];
+    const int inst = tb.instance ? tb.instance[i] : 0;
+    bool bad = a < 0 || a >= P.A || inst < 0 || inst >= P.I;
+    if (!bad && i > 0) {
+        const int prev = tb.instance ? tb.instance[i - 1] : 0;
+        if (prev > inst) bad = true;
+        if (trace_mode && prev == inst && tb.arrival[i - 1] > tb.arrival[i]) bad = true;
+    }
+    if (bad) {
+        dev_error(&flags[0], kDevBadRequest);
+        flags[1] = 1;
+        return;
+    }
+    const int key = inst * P.A + a;
+    // one atomic per distinct key in the warp
+    const unsigned peers = __match_any_sync(__activemask(), key);
+    if ((int)(__ffs(peers) - 1) == (int)(threadIdx.x & 31)) atomicAdd(&tb.cnt[key], __popc(peers));
+}
+
+// Single block.  gstart = exclusive prefix of cnt (int64); tiled_start = exclusive prefix of
+// ceil(cnt / kTiledRows) per (instance, app); small_start = exclusive prefix over instances of
+// ceil(requests of the instance / kSmallRows).
+__global__ void __launch_bounds__(1024) k_group_scan(int n_keys, int A, const int32_t *cnt, int64_t *gstart,
+                                                     int32_t *tiled_start, int32_t *small_start) {
+    __shared__ long long warp_sum[32];
+    __shared__ long long carry[3];
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    if (tid < 3) carry[tid] = 0;
+    __syncthreads();
+    // pass 0: gstart, pass 1: tiled tiles, pass 2: small tiles (over instances)
+    for (int pass = 0; pass < 3; ++pass) {
+        const int len = pass == 2 ? n_keys / A : n_keys;
+        for (int base = 0; base < len; base += 1024) {
+            const int k = base + tid;
+            long long val = 0;
+            if (k < len) {
+                if (pass == 0) val = cnt[k];
+                else if (pass == 1) val = (cnt[k] + kTiledRows - 1) / kTiledRows;
+                else {
+                    long long s = 0;
+                    for (int a = 0; a < A; ++a) s += cnt[k * A + a];
+                    val = (s + kSmallRows - 1) / kSmallRows;
+                }
+            }
+            long long incl = val;
+            for (int o = 1; o < 32; o <<= 1) {
+                const long long t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            if (lane == 31) warp_sum[wid] = incl;
+            __syncthreads();
+            if (wid == 0) {
+                long long w = warp_sum[lane];
+                for (int o = 1; o < 32; o <<= 1) {
+                    const long long t = __shfl_up_sync(0xffffffffu, w, o);
+                    if (lane >= o) w += t;
+                }
+                warp_sum[lane] = w;
+            }
+            __syncthreads();
+            const long long excl = carry[pass] + (wid ? warp_sum[wid - 1] : 0) + incl - val;
+            if (k < len) {
+                if (pass == 0) gstart[k] = excl;
+                else if (pass == 1) tiled_start[k] = (int32_t)excl;
+                else small_start[k] = (int32_t)excl;
+            }
+            __syncthreads();
+            if (tid == 0) carry[pass] += warp_sum[31];
+            __syncthreads();
+        }
+        if (tid == 0) {
+            if (pass == 0) gstart[len] = carry[0];
+            else if (pass == 1) tiled_start[len] = (int32_t)carry[1];
+            else small_start[len] = (int32_t)carry[2];
+        }
+        __syncthreads();
+    }
+}
+
+__global__ void k_group_scatter(DevProfiles P, DevTable tb, const int *flags) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= tb.n || flags[1]) return;
+    const int key = (tb.instance ? tb.instance[i] : 0) * P.A + tb.app[i];
+    const int pos = atomicAdd(&tb.cursor[key], 1);
+    tb.perm[tb.gstart[key] + pos] = i;
+}
+
+}  // namespace sp

@@ -1,0 +1,575 @@
+// Persistent greedy scheduling kernel: one thread block runs all rounds of one instance on the device.
+//
+// Per round (Section 4.2 and Algorithm 1 of the paper, one batch per iteration of its loop):
+//   1. requests whose arrival time has passed join their application's queue, kept sorted by (deadline, id);
+//   2. requests that no candidate of their application could complete in time are retired (utility 0 under
+//      the step penalty of Section 5.1);
+//   3. group priority (Eq. 14 over Eq. 12) of every non-empty application; the highest goes next;
+//   4. every (model variant, batch size) candidate of that application: completion time from the latency
+//      profile (+ swap time when the model is not resident), summed member utility (Eq. 2) from fp64 prefix
+//      sums over the deadline-sorted head of the queue and a binary search for the members that are late;
+//   5. block-wide argmax (ties: lowest model, then smallest batch), emit s_ij, advance clock and queue head.
+// Accuracies come from the fp32 scoring kernels.  Whenever the two best group priorities or candidate
+// utilities are closer than a guard band (far wider than the fp32 error), the rows involved are re-scored
+// in fp64 from the raw features and the decision is taken on those values.
+#pragma once
+
+#include "sp_common.cuh"
+
+namespace sp {
+
+struct InstState {
+    int64_t T, next_order, Tref, inserted;   // inserted: requests of the instance that have joined a queue
+    int32_t L, round, exp_since, started;
+    int32_t head[kMaxApps], tail[kMaxApps], cur[kMaxApps];   // queue positions relative to the region start
+};
+
+struct SortKey { int64_t dl; int32_t id_rel; int32_t app; };  // id_rel: request id - first id of the instance
+
+struct SchedParams {
+    DevProfiles P;
+    DevTable tb;
+    InstState *state;           // [I]
+    int64_t *q_id[2];           // [n] request ids, queue regions at gstart[key]
+    int64_t *q_dl[2];           // [n] deadlines in queue order
+    double *q_pw[2];            // [n] v * exp(-(deadline - Tref)/tau) in queue order
+    SortKey *sort_scratch;      // [n]
+    double *zbuf;               // [I][warps][C] logits scratch of the fp64 re-evaluation
+    int *flags;
+    unsigned long long *stats;  // rounds, exact_utility, exact_priority, exact_rows
+    int trace_mode;
+    double guard_u, guard_p;
+    int max_rounds;
+    sp_round_rec *rounds_out;
+    int64_t cap;
+    int32_t *n_done;
+    int sort_cap;               // SortKey entries available in shared memory
+    int bmax;                   // largest allowed batch size
+};
+
+__device__ __forceinline__ bool key_less(const SortKey &a, const SortKey &b) {
+    if (a.app != b.app) return a.app < b.app;
+    if (a.dl != b.dl) return a.dl < b.dl;
+    return a.id_rel < b.id_rel;
+}
+
+// Sorting network with ascending comparators only (first step of every merge mirrors the partner), so
+// a length that is not a power of two needs no padding: a partner index >= n stands for +infinity.
+__device__ void block_sort(SortKey *keys, int n) {
+    int p2 = 1;
+    while (p2 < n) p2 <<= 1;
+    for (int k = 2; k <= p2; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int t = threadIdx.x; t < (p2 >> 1); t += blockDim.x) {
+                // t-th pair of this step: low index i has bit j clear
+                const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+                const int partner = (j == (k >> 1)) ? (i ^ (k - 1)) : (i ^ j);
+                if (partner < n && i < n) {
+                    const SortKey a = keys[i], b = keys[partner];
+                    if (key_less(b, a)) { keys[i] = b; keys[partner] = a; }
+                }
+            }
+            __syncthreads();
+        }
+    }
+}
+
+__device__ __forceinline__ double block_sum(double v, double *red) {
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();
+    if (lane == 0) red[wid] = v;
+    __syncthreads();
+    if (wid == 0) {
+        double w = lane < (int)(blockDim.x >> 5) ? red[lane] : 0.0;
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) w += __shfl_xor_sync(0xffffffffu, w, o);
+        if (lane == 0) red[32] = w;
+    }
+    __syncthreads();
+    return red[32];
+}
+
+// fp64 re-scoring of one request by one warp, written to acc64 / v64.  Plain definition of Section 4.1 /
+// Eq. 9 / Eq. 12 with separate multiplies and adds (no fused multiply-add).
+__device__ void exact_row(const SchedParams &sp, int inst, int64_t id, double *zrow) {
+    const DevProfiles &P = sp.P;
+    const int lane = threadIdx.x & 31;
+    const int a = sp.tb.app[id];
+    const int64_t head = (int64_t)inst * P.A + a;
+    const int C = P.C, D = P.D;
+    for (int c0 = 0; c0 < C; c0 += 32) {
+        const int c = c0 + lane;
+        double z = c < C ? (double)P.bias[head * C + c] : 0.0;
+        if (c < C)
+            for (int d = 0; d < D; ++d) {
+                const double x = (double)load_feat(sp.tb.feats, P.dtype, id * D + d);
+                const double w = (double)load_feat(P.W, P.dtype, (head * D + d) * C + c);
+                z = __dadd_rn(z, __dmul_rn(x, w));
+            }
+        if (c < C) zrow[c] = z;
+    }
+    __syncwarp();
+    double m = -INFINITY;
+    for (int c = lane; c < C; c += 32) m = fmax(m, zrow[c]);
+    for (int o = 16; o >= 1; o >>= 1) m = fmax(m, __shfl_xor_sync(0xffffffffu, m, o));
+    double s = 0.0;
+    for (int c = lane; c < C; c += 32) { const double e = exp(zrow[c] - m); zrow[c] = e; s += e; }
+    for (int o = 16; o >= 1; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    __syncwarp();
+    double asum = 0.0;
+    if (P.prior) asum = (double)P.prior_sum[head];   // refined below in fp64
+    if (P.prior) {
+        double t = 0.0;
+        for (int c = lane; c < C; c += 32) t += (double)P.prior[head * C + c];
+        for (int o = 16; o >= 1; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+        asum = t;
+    }
+    for (int c = lane; c < C; c += 32) {
+        double th = zrow[c] / s;
+        if (P.prior) th = ((double)P.prior[head * C + c] + (double)P.kappa * th) / (asum + (double)P.kappa);
+        zrow[c] = th;
+    }
+    __syncwarp();
+    const int m0 = P.mfirst[a], M = P.mfirst[a + 1] - m0;
+    double mean = 0.0, accv[kMaxModelsPerApp];
+    for (int j = 0; j < kMaxModelsPerApp; ++j) {
+        accv[j] = 0.0;
+        if (j < M) {
+            const float *r = P.recall + ((int64_t)inst * P.sumM + m0 + j) * C;
+            double t = 0.0;
+            for (int c = lane; c < C; c += 32) t = __dadd_rn(t, __dmul_rn(zrow[c], (double)r[c]));
+            for (int o = 16; o >= 1; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+            accv[j] = t;
+            mean += t;
+        }
+    }
+    mean /= (double)M;
+    double var = 0.0;
+    for (int j = 0; j < kMaxModelsPerApp; ++j)
+        if (j < M) var += (accv[j] - mean) * (accv[j] - mean);
+    if (lane == 0) {
+        for (int j = 0; j < P.Mmax; ++j) sp.tb.acc64[id * P.Mmax + j] = j < M ? accv[j] : 0.0;
+        sp.tb.v64[id] = 1.0 + var / (double)M;
+        __threadfence_block();
+        sp.tb.exact[id] = 1;
+    }
+    __syncwarp();
+}
+
+// Re-scores (if not done before) the requests at queue positions [k0, k1) of one queue buffer.
+__device__ void exact_rows(const SchedParams &sp, int inst, const int64_t *qid, int64_t k0, int64_t k1) {
+    const int warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    double *zrow = sp.zbuf + ((int64_t)inst * nwarps + warp) * sp.P.C;
+    unsigned long long done = 0;
+    for (int64_t k = k0 + warp; k < k1; k += nwarps) {
+        const int64_t id = qid[k];
+        if (!sp.tb.exact[id]) { exact_row(sp, inst, id, zrow); ++done; }
+    }
+    if ((threadIdx.x & 31) == 0 && done) atomicAdd(&sp.stats[3], done);
+    __syncthreads();
+}
+
+}  // namespace sp
+
+namespace sp {
+
+// Shared-memory carve-up of k_sched (bytes, 16-byte aligned pieces).
+struct SchedSmem {
+    size_t keys, pref, accs, mem_id, mem_dl, cand_u, cand_e, cand_bp, end;
+    __host__ __device__ SchedSmem(int sort_cap, int Mmax, int bmax, int ncand) {
+        size_t o = 0;
+        keys = o;    o += (size_t)sort_cap * sizeof(SortKey);
+        pref = o;    o += (size_t)Mmax * (bmax + 1) * sizeof(double);
+        mem_id = o;  o += (size_t)bmax * sizeof(int64_t);
+        mem_dl = o;  o += (size_t)bmax * sizeof(int64_t);
+        cand_u = o;  o += (size_t)ncand * sizeof(double);
+        cand_e = o;  o += (size_t)ncand * sizeof(int64_t);
+        accs = o;    o += (size_t)bmax * Mmax * sizeof(float);
+        cand_bp = o; o += (size_t)ncand * sizeof(int);
+        end = (o + 15) & ~(size_t)15;
+    }
+};
+
+__device__ __forceinline__ double prio_weight(double v, int64_t dl, int64_t tref, double tau) {
+    return v * exp(-((double)(dl - tref) * 1e-9 / tau));
+}
+
+// Warp 0: argmax of cand_u over [0, ncand) with ties to the lowest index; also counts the entries within
+// the relative guard of the maximum and the largest batch among them.  Results are valid in every lane.
+__device__ __forceinline__ void warp_argmax(const double *cand_u, const int *cand_bp, int ncand, double guard,
+                                            int &best, double &best_u, int &n_close, int &max_bp) {
+    const int lane = threadIdx.x & 31;
+    double bu = -INFINITY;
+    int bi = 0x7fffffff;
+    for (int ci = lane; ci < ncand; ci += 32) {
+        const double u = cand_u[ci];
+        if (u > bu) { bu = u; bi = ci; }
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+        const double ou = __shfl_xor_sync(0xffffffffu, bu, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ou > bu || (ou == bu && oi < bi)) { bu = ou; bi = oi; }
+    }
+    const double thr = bu - fabs(bu) * guard;
+    int cnt = 0, mb = 0;
+    for (int ci = lane; ci < ncand; ci += 32) {
+        const double u = cand_u[ci];
+        if (u >= thr && u != -INFINITY) { ++cnt; mb = max(mb, cand_bp[ci]); }
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+        cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+        mb = max(mb, __shfl_xor_sync(0xffffffffu, mb, o));
+    }
+    best = bi; best_u = bu; n_close = cnt; max_bp = mb;
+}
+
+__global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
+    extern __shared__ __align__(16) unsigned char dyn[];
+    __shared__ InstState st;
+    __shared__ double red[33];
+    __shared__ double s_P[kMaxApps];
+    __shared__ int s_seg[kMaxApps + 2];
+    __shared__ int s_newhead[kMaxApps];
+    __shared__ int64_t s_nnew;
+    __shared__ int s_best_app, s_exactP, s_best_ci, s_nclose, s_maxbp;
+    __shared__ double s_best_u, s_best_p;
+    __shared__ unsigned char s_contend[kMaxApps];
+
+    const DevProfiles &P = sp.P;
+    const DevTable &tb = sp.tb;
+    const int tid = threadIdx.x, NT = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarps = NT >> 5;
+    const int inst = blockIdx.x, A = P.A, nB = P.nB, Mmax = P.Mmax, bmax = sp.bmax;
+    const int ncand_max = kMaxModelsPerApp * kMaxBatchSizes;
+    const SchedSmem L(sp.sort_cap, Mmax, bmax, ncand_max);
+    SortKey *smem_keys = reinterpret_cast<SortKey *>(dyn + L.keys);
+    double *pref = reinterpret_cast<double *>(dyn + L.pref);
+    float *accs = reinterpret_cast<float *>(dyn + L.accs);
+    int64_t *mem_id = reinterpret_cast<int64_t *>(dyn + L.mem_id);
+    int64_t *mem_dl = reinterpret_cast<int64_t *>(dyn + L.mem_dl);
+    double *cand_u = reinterpret_cast<double *>(dyn + L.cand_u);
+    int64_t *cand_e = reinterpret_cast<int64_t *>(dyn + L.cand_e);
+    int *cand_bp = reinterpret_cast<int *>(dyn + L.cand_bp);
+
+    if (sp.flags[1]) {                       // request table failed validation: do nothing
+        if (tid == 0 && sp.n_done) sp.n_done[inst] = 0;
+        return;
+    }
+    const int64_t r0 = tb.gstart[(int64_t)inst * A], r1 = tb.gstart[(int64_t)(inst + 1) * A];
+    const int64_t n_inst = r1 - r0;
+    if (tid == 0) st = sp.state[inst];
+    __syncthreads();
+
+    const double tau = P.tau;
+    const int64_t *al = P.lat_alpha + (int64_t)inst * P.sumM;
+    const int64_t *be = P.lat_beta + (int64_t)inst * P.sumM;
+    const int64_t *sw = P.swap + (int64_t)inst * P.sumM;
+    int rounds_done = 0;
+    unsigned long long n_exact_u = 0, n_exact_p = 0;
+    const int64_t max_iter = (int64_t)sp.max_rounds + 2 * n_inst + 8;
+    bool finished = false;
+
+    for (int64_t iter = 0; iter < max_iter; ++iter) {
+        if (rounds_done >= sp.max_rounds) { finished = true; break; }
+        // ---------------------------------------------------------------- 1. arrivals join their queues
+        if (tid == 0) {
+            if (!st.started) { st.started = 1; st.Tref = st.T; }
+            int64_t lo = st.inserted, hi = n_inst;
+            if (sp.trace_mode) {              // first request (in arrival order) that has not arrived yet
+                while (lo < hi) {
+                    const int64_t mid = (lo + hi) >> 1;
+                    if (tb.arrival[r0 + mid] <= st.T) lo = mid + 1; else hi = mid;
+                }
+            } else lo = n_inst;
+            s_nnew = lo - st.inserted;
+        }
+        __syncthreads();
+        const int64_t nnew = s_nnew;
+        if (nnew > 0) {
+            const int64_t ap = st.inserted;
+            SortKey *keys = nnew <= sp.sort_cap ? smem_keys : sp.sort_scratch + r0 + ap;
+            for (int64_t t = tid; t < nnew; t += NT) {
+                const int64_t id = r0 + ap + t;
+                SortKey k; k.dl = tb.deadline[id]; k.id_rel = (int32_t)(ap + t); k.app = tb.app[id];
+                keys[t] = k;
+            }
+            __syncthreads();
+            block_sort(keys, (int)nnew);
+            if (tid <= A) {                   // first sorted position whose application is >= tid
+                int lo = 0, hi = (int)nnew;
+                while (lo < hi) { const int mid = (lo + hi) >> 1; if (keys[mid].app < tid) lo = mid + 1; else hi = mid; }
+                s_seg[tid] = lo;
+            }
+            __syncthreads();
+            for (int a = 0; a < A; ++a) {
+                const int nn = s_seg[a + 1] - s_seg[a];
+                if (nn == 0) continue;
+                const int64_t base = tb.gstart[(int64_t)inst * A + a];
+                const int head = st.head[a], tail = st.tail[a], nl = tail - head, c = st.cur[a];
+                const SortKey *nk = keys + s_seg[a];
+                if (nl == 0) {
+                    for (int t = tid; t < nn; t += NT) {
+                        const int64_t id = r0 + nk[t].id_rel, pos = base + tail + t;
+                        sp.q_id[c][pos] = id; sp.q_dl[c][pos] = nk[t].dl;
+                        sp.q_pw[c][pos] = prio_weight((double)tb.v32[id], nk[t].dl, st.Tref, tau);
+                    }
+                } else {
+                    const int d = 1 - c;
+                    const int64_t *lid = sp.q_id[c] + base + head, *ldl = sp.q_dl[c] + base + head;
+                    for (int k = tid; k < nl; k += NT) {        // live element: count new elements before it
+                        const int64_t dl = ldl[k], idr = lid[k] - r0;
+                        int lo = 0, hi = nn;
+                        while (lo < hi) {
+                            const int mid = (lo + hi) >> 1;
+                            const bool less = nk[mid].dl < dl || (nk[mid].dl == dl && nk[mid].id_rel < idr);
+                            if (less) lo = mid + 1; else hi = mid;
+                        }
+                        const int64_t pos = base + head + k + lo;
+                        sp.q_id[d][pos] = lid[k]; sp.q_dl[d][pos] = dl; sp.q_pw[d][pos] = sp.q_pw[c][base + head + k];
+                    }
+                    for (int t = tid; t < nn; t += NT) {        // new element: count live elements before it
+                        const int64_t dl = nk[t].dl, idr = nk[t].id_rel;
+                        int lo = 0, hi = nl;
+                        while (lo < hi) {
+                            const int mid = (lo + hi) >> 1;
+                            const bool less = ldl[mid] < dl || (ldl[mid] == dl && (lid[mid] - r0) < idr);
+                            if (less) lo = mid + 1; else hi = mid;
+                        }
+                        const int64_t id = r0 + idr, pos = base + head + t + lo;
+                        sp.q_id[d][pos] = id; sp.q_dl[d][pos] = dl;
+                        sp.q_pw[d][pos] = prio_weight((double)tb.v32[id], dl, st.Tref, tau);
+                    }
+                }
+            }
+            __syncthreads();
+            if (tid == 0) {
+                for (int a = 0; a < A; ++a) {
+                    const int nn = s_seg[a + 1] - s_seg[a];
+                    if (nn == 0) continue;
+                    if (st.tail[a] - st.head[a] > 0) st.cur[a] = 1 - st.cur[a];
+                    st.tail[a] += nn;
+                }
+                st.inserted += nnew;
+            }
+            __syncthreads();
+        }
+        int64_t live = 0;
+        for (int a = 0; a < A; ++a) live += st.tail[a] - st.head[a];
+        if (live == 0) {
+            if (st.inserted < n_inst) {       // idle: wake at the next arrival
+                __syncthreads();
+                if (tid == 0) st.T = tb.arrival[r0 + st.inserted];
+                __syncthreads();
+                continue;
+            }
+            finished = true;
+            break;
+        }
+        // keep exp((T - Tref)/tau) in range: re-reference the stored priority weights now and then
+        if ((double)(st.T - st.Tref) * 1e-9 / tau > 32.0) {
+            for (int a = 0; a < A; ++a) {
+                const int64_t base = tb.gstart[(int64_t)inst * A + a];
+                const int c = st.cur[a];
+                for (int k = st.head[a] + tid; k < st.tail[a]; k += NT)
+                    sp.q_pw[c][base + k] = prio_weight((double)tb.v32[sp.q_id[c][base + k]], sp.q_dl[c][base + k], st.T, tau);
+            }
+            __syncthreads();
+            if (tid == 0) st.Tref = st.T;
+            __syncthreads();
+        }
+        // ---------------------------------------------------------------- 2. retire hopeless requests
+        if (tid < A) {
+            const int a = tid, head = st.head[a], tail = st.tail[a];
+            int nh = head;
+            if (tail > head) {
+                int64_t emin = INT64_MAX;
+                for (int g = P.mfirst[a]; g < P.mfirst[a + 1]; ++g) {
+                    const int64_t e = st.T + (g != st.L ? sw[g] : 0) + al[g] + be[g] * (int64_t)P.batch[0];
+                    emin = e < emin ? e : emin;
+                }
+                const int64_t *dl = sp.q_dl[st.cur[a]] + tb.gstart[(int64_t)inst * A + a];
+                int lo = head, hi = tail;
+                while (lo < hi) { const int mid = (lo + hi) >> 1; if (dl[mid] < emin) lo = mid + 1; else hi = mid; }
+                nh = lo;
+            }
+            s_newhead[a] = nh;
+        }
+        __syncthreads();
+        for (int a = 0; a < A; ++a) {
+            const int64_t *qid = sp.q_id[st.cur[a]] + tb.gstart[(int64_t)inst * A + a];
+            for (int k = st.head[a] + tid; k < s_newhead[a]; k += NT) {
+                sp_req_rec r; r.status = SP_EXPIRED; r.round = st.round; r.model = -1; r.pad_ = 0; r.order = 0;
+                tb.recs[qid[k]] = r;
+            }
+        }
+        __syncthreads();
+        if (tid == 0)
+            for (int a = 0; a < A; ++a) { st.exp_since += s_newhead[a] - st.head[a]; st.head[a] = s_newhead[a]; }
+        __syncthreads();
+        live = 0;
+        for (int a = 0; a < A; ++a) live += st.tail[a] - st.head[a];
+        if (live == 0) continue;
+        // ---------------------------------------------------------------- 3. group priorities (Eq. 14)
+        for (int a = 0; a < A; ++a) {
+            const int na = st.tail[a] - st.head[a];
+            if (na == 0) { if (tid == 0) s_P[a] = -INFINITY; continue; }
+            const double *pw = sp.q_pw[st.cur[a]] + tb.gstart[(int64_t)inst * A + a];
+            double part = 0.0;
+            for (int k = st.head[a] + tid; k < st.tail[a]; k += NT) part += pw[k];
+            const double S = block_sum(part, red);
+            if (tid == 0) s_P[a] = S / (double)na;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            int ba = -1;
+            for (int a = 0; a < A; ++a)
+                if (s_P[a] != -INFINITY && (ba < 0 || s_P[a] > s_P[ba])) ba = a;
+            int close = 0;
+            for (int a = 0; a < A; ++a) {
+                const bool c = s_P[a] != -INFINITY && s_P[a] >= s_P[ba] * (1.0 - sp.guard_p);
+                s_contend[a] = c; close += c;
+            }
+            s_best_app = ba;
+            s_exactP = close > 1;
+            s_best_p = s_P[ba] * exp((double)(st.T - st.Tref) * 1e-9 / tau);
+        }
+        __syncthreads();
+        int round_exact = 0;
+        if (s_exactP) {                        // near-tie between groups: decide on fp64 scores
+            for (int a = 0; a < A; ++a) {
+                if (!s_contend[a]) continue;
+                const int64_t base = tb.gstart[(int64_t)inst * A + a];
+                const int c = st.cur[a];
+                exact_rows(sp, inst, sp.q_id[c] + base, st.head[a], st.tail[a]);
+                double part = 0.0;
+                for (int k = st.head[a] + tid; k < st.tail[a]; k += NT) {
+                    const double dt = (double)(sp.q_dl[c][base + k] - st.T) * 1e-9 / tau;
+                    part += tb.v64[sp.q_id[c][base + k]] * exp(-dt);
+                }
+                const double S = block_sum(part, red);
+                if (tid == 0) s_P[a] = S / (double)(st.tail[a] - st.head[a]);
+            }
+            __syncthreads();
+            if (tid == 0) {
+                int ba = -1;
+                for (int a = 0; a < A; ++a)
+                    if (s_contend[a] && (ba < 0 || s_P[a] > s_P[ba])) ba = a;
+                s_best_app = ba; s_best_p = s_P[ba];
+            }
+            __syncthreads();
+            round_exact |= 1; ++n_exact_p;
+        }
+        // ---------------------------------------------------------------- 4. candidates of the chosen group
+        const int a = s_best_app;
+        const int64_t base = tb.gstart[(int64_t)inst * A + a];
+        const int c = st.cur[a], head = st.head[a], na = st.tail[a] - head;
+        const int nb = na < bmax ? na : bmax;
+        const int m0 = P.mfirst[a], M = P.mfirst[a + 1] - m0, ncand = M * nB;
+        for (int k = tid; k < nb; k += NT) {
+            mem_id[k] = sp.q_id[c][base + head + k];
+            mem_dl[k] = sp.q_dl[c][base + head + k];
+        }
+        __syncthreads();
+        for (int k = tid; k < nb * Mmax; k += NT) {
+            const int r = k / Mmax, j = k - r * Mmax;
+            accs[k] = tb.acc32[mem_id[r] * Mmax + j];
+        }
+        __syncthreads();
+        for (int j = warp; j < M; j += nwarps) {      // fp64 prefix sums of the members' accuracies, per model
+            double *pj = pref + (size_t)j * (bmax + 1);
+            double carry = 0.0;
+            if (lane == 0) pj[0] = 0.0;
+            for (int k0 = 0; k0 < nb; k0 += 32) {
+                const int k = k0 + lane;
+                double v = k < nb ? (double)accs[k * Mmax + j] : 0.0;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const double t = __shfl_up_sync(0xffffffffu, v, o);
+                    if (lane >= o) v += t;
+                }
+                v += carry;
+                if (k < nb) pj[k + 1] = v;
+                carry = __shfl_sync(0xffffffffu, v, 31);
+            }
+        }
+        __syncthreads();
+        for (int ci = tid; ci < ncand; ci += NT) {
+            const int j = ci / nB, bi = ci - j * nB, g = m0 + j;
+            const int b = P.batch[bi];
+            const bool valid = bi == 0 || P.batch[bi - 1] < na;   // a larger size with the same members never wins
+            const int bp = b < na ? b : na;
+            const int64_t e = st.T + (g != st.L ? sw[g] : 0) + al[g] + be[g] * (int64_t)bp;
+            int lo = 0, hi = bp;                                   // members with deadline < e are late
+            while (lo < hi) { const int mid = (lo + hi) >> 1; if (mem_dl[mid] < e) lo = mid + 1; else hi = mid; }
+            const double *pj = pref + (size_t)j * (bmax + 1);
+            cand_u[ci] = valid ? pj[bp] - pj[lo] : -INFINITY;
+            cand_e[ci] = e; cand_bp[ci] = bp;
+        }
+        __syncthreads();
+        if (warp == 0) {
+            int best, ncl, mbp; double bu;
+            warp_argmax(cand_u, cand_bp, ncand, sp.guard_u, best, bu, ncl, mbp);
+            if (lane == 0) { s_best_ci = best; s_best_u = bu; s_nclose = ncl; s_maxbp = mbp; }
+        }
+        __syncthreads();
+        if (s_nclose > 1) {                    // near-tie between candidates: decide on fp64 scores
+            const double thr = s_best_u - fabs(s_best_u) * sp.guard_u;
+            exact_rows(sp, inst, sp.q_id[c] + base, head, head + s_maxbp);
+            for (int ci = tid; ci < ncand; ci += NT) {
+                const double u32 = cand_u[ci];
+                double u = -INFINITY;
+                if (u32 >= thr && u32 != -INFINITY) {
+                    const int j = ci / nB, bp = cand_bp[ci];
+                    const int64_t e = cand_e[ci];
+                    u = 0.0;
+                    for (int k = 0; k < bp; ++k)
+                        if (!(mem_dl[k] < e)) u = __dadd_rn(u, tb.acc64[mem_id[k] * Mmax + j]);
+                }
+                cand_u[ci] = u;
+            }
+            __syncthreads();
+            if (warp == 0) {
+                int best, ncl, mbp; double bu;
+                warp_argmax(cand_u, cand_bp, ncand, 0.0, best, bu, ncl, mbp);
+                if (lane == 0) { s_best_ci = best; s_best_u = bu; }
+            }
+            __syncthreads();
+            round_exact |= 2; ++n_exact_u;
+        }
+        // ---------------------------------------------------------------- 5. emit, remove, advance the clock
+        const int ci = s_best_ci, bj = ci / nB, bbi = ci - bj * nB, g = m0 + bj;
+        const int bp = cand_bp[ci];
+        const int64_t e = cand_e[ci];
+        for (int k = tid; k < bp; k += NT) {
+            sp_req_rec r; r.status = SP_SCHEDULED; r.round = st.round; r.model = g; r.pad_ = 0;
+            r.order = st.next_order + k;
+            tb.recs[mem_id[k]] = r;
+        }
+        __syncthreads();
+        if (tid == 0) {
+            if (sp.rounds_out && rounds_done < sp.cap) {
+                sp_round_rec rr;
+                rr.instance = inst; rr.round = st.round; rr.app = a; rr.model = g; rr.batch = P.batch[bbi];
+                rr.n_members = bp; rr.n_expired = st.exp_since; rr.exact = round_exact;
+                rr.t_start_ns = st.T; rr.t_end_ns = e; rr.utility = s_best_u; rr.group_priority = s_best_p;
+                sp.rounds_out[(int64_t)inst * sp.cap + rounds_done] = rr;
+            }
+            st.head[a] += bp; st.T = e; st.L = g; st.round += 1; st.next_order += bp; st.exp_since = 0;
+        }
+        ++rounds_done;
+        __syncthreads();
+    }
+    if (tid == 0) {
+        if (!finished && rounds_done < sp.max_rounds) dev_error(&sp.flags[0], kDevLimit);
+        sp.state[inst] = st;
+        if (sp.n_done) sp.n_done[inst] = rounds_done;
+        if (rounds_done) atomicAdd(&sp.stats[0], (unsigned long long)rounds_done);
+        if (n_exact_u) atomicAdd(&sp.stats[1], n_exact_u);
+        if (n_exact_p) atomicAdd(&sp.stats[2], n_exact_p);
+    }
+}
+
+}  // namespace sp

@@ -1,0 +1,166 @@
+"""Parity of the CUDA library with the CPU oracle, element by element (needs a B200; run with -m gpu)."""
+import numpy as np
+import pytest
+
+from paper_2505_06641_b200 import synth
+from helpers import manual_workload
+from parity import ACC_RTOL, check_schedule, check_scores
+
+pytestmark = pytest.mark.gpu
+
+
+def _both(w, guards=None, **kw):
+    from oracle import oracle
+    from paper_2505_06641_b200 import api, runner
+    s = oracle.score(w)
+    od = oracle.drain(w, s.acc, s.v, **{k: v for k, v in kw.items() if k in ("max_rounds", "cap")})
+    ses = runner.Session(w)
+    if guards is not None:
+        api.sp_set_options(ses.ctx, trace_mode=bool(w.trace_mode), guard_utility=guards[0], guard_priority=guards[1])
+    res = ses.run(**kw)
+    ses.close()
+    return s, od, res
+
+
+CASES = [("C1", {}), ("C2", {}), ("C3", dict(n_requests=3000)), ("C4", dict(n_instances=40)),
+         ("C5", dict(n_requests=20000)),
+         ("C1", dict(n_requests=1)), ("C1", dict(n_requests=129)), ("C2", dict(n_requests=65)),
+         ("C4", dict(n_instances=3, n_requests=131)), ("C3", dict(n_requests=70, models=5))]
+
+
+@pytest.mark.parametrize("name,kw", CASES)
+def test_scores_and_schedule_match_oracle(name, kw):
+    w = synth.make_workload(name, **kw)
+    s, od, res = _both(w)
+    worst = check_scores(res, s)
+    skipped = check_schedule(w, res, od)
+    assert skipped == 0, "unexpected near-tie in a seeded case"
+    assert worst < ACC_RTOL
+
+
+@pytest.mark.parametrize("name,kw", [("C1", {}), ("C2", {}), ("C4", dict(n_instances=12)),
+                                     ("C5", dict(n_requests=4000)), ("C3", dict(n_requests=400))])
+def test_fp64_reevaluation_path_gives_the_same_schedule(name, kw):
+    """Guards of 1.0 send every round through the fp64 re-scoring; the schedule must not change."""
+    w = synth.make_workload(name, **kw)
+    s, od, res = _both(w, guards=(1.0, 1.0))
+    check_schedule(w, res, od)
+    nr = int(res.n_rounds.sum())
+    assert res.stats["exact_utility"] > 0 and res.stats["exact_rows"] > 0
+    multi = res.rounds["exact"][res.rounds["n_members"] > 0]
+    assert np.all(multi & 2 | (multi == 0) | (multi & 1)) and nr == res.stats["rounds"]
+    # utilities decided in fp64 agree with the oracle to rounding
+    for k in range(int(w.n_instances)):
+        n = int(od.n_rounds[k])
+        ex = (res.rounds[k, :n]["exact"] & 2) != 0
+        np.testing.assert_allclose(res.rounds[k, :n]["utility"][ex], od.rounds[k, :n]["utility"][ex], rtol=1e-12)
+
+
+def test_dirichlet_prior_and_ragged_model_sets():
+    rng = np.random.default_rng(11)
+    n, c = 200, 7
+    w = manual_workload(rng.dirichlet(np.ones(c), size=n), rng.uniform(0.2, 0.99, size=(6, c)),
+                        app=rng.integers(0, 3, size=n), deadline_ms=rng.uniform(50, 900, size=n),
+                        alpha_ms=rng.uniform(2, 20, size=6), beta_ms=rng.uniform(0.5, 5, size=6),
+                        swap_ms=rng.uniform(5, 50, size=6), batch_sizes=[1, 2, 4, 8], models_per_app=[1, 2, 3],
+                        prior_alpha=np.full((3, c), 0.5), evidence_k=5.0)
+    s, od, res = _both(w)
+    check_scores(res, s)
+    check_schedule(w, res, od)
+    assert np.all(res.acc[w.app == 0, 1:] == 0) and np.all(res.v[w.app == 0] == 1.0)
+
+
+def test_padded_classes_with_minus_inf_bias():
+    w = synth.make_workload("C1", n_requests=100)
+    w.head_b[0, 1, 6:] = -np.inf          # application 1 has only 6 labels
+    w.recall[0, 4:8, 6:] = 0.0
+    s, od, res = _both(w)
+    check_scores(res, s)
+    check_schedule(w, res, od)
+
+
+def test_empty_request_set():
+    from paper_2505_06641_b200 import runner
+    w = synth.make_workload("C1", n_requests=1)
+    for f in ("feats", "app", "arrival_ns", "deadline_ns", "instance"):
+        setattr(w, f, getattr(w, f)[:0])
+    ses = runner.Session(w)
+    res = ses.run(max_rounds=4, cap=4)
+    assert res.n_rounds[0] == 0 and len(res.reqs) == 0
+    ses.close()
+
+
+def test_rounds_can_be_run_in_several_calls():
+    from oracle import oracle
+    from paper_2505_06641_b200 import api, runner
+    import torch
+    w = synth.make_workload("C2")
+    s = oracle.score(w)
+    od = oracle.drain(w, s.acc, s.v)
+    ses = runner.Session(w)
+    ses.upload(); ses.alloc_outputs(64); ses.score()
+    got = []
+    for _ in range(40):
+        ses.schedule(3)
+        api.sp_check(ses.ctx)
+        k = int(ses.n_done.cpu()[0])
+        got.append(ses.rounds.cpu().numpy().reshape(1, -1).view(api.ROUND_DTYPE)[0, :k].copy())
+        if k < 3:
+            break
+    got = np.concatenate(got)
+    assert len(got) == od.n_rounds[0]
+    for f in ("round", "app", "model", "batch", "n_members", "n_expired", "t_start_ns", "t_end_ns"):
+        assert np.array_equal(got[f], od.rounds[0, :len(got)][f]), f
+    ses.close()
+
+
+def test_trace_mode_idle_clock_jump():
+    w = manual_workload([[0.5, 0.5]] * 3, [[0.8, 0.8]], app=[0] * 3, deadline_ms=[100, 130, 1100],
+                        arrival_ms=[0, 5, 1000], alpha_ms=[10], beta_ms=[10], swap_ms=[0], batch_sizes=[1, 2],
+                        models_per_app=[1], trace_mode=True)
+    s, od, res = _both(w)
+    check_schedule(w, res, od)
+    assert [int(x) // synth.MS for x in res.rounds[0, :3]["t_start_ns"]] == [0, 20, 1000]
+
+
+def test_host_buffer_entry_point_matches_device_path():
+    from paper_2505_06641_b200 import api, runner
+    w = synth.make_workload("C4", n_instances=9)
+    ses = runner.Session(w)
+    ref = ses.run()
+    n, ni, cap = w.n_requests, w.n_instances, ref.rounds.shape[1]
+    reqs = np.zeros(n, dtype=api.REQ_DTYPE)
+    rounds = np.zeros((ni, cap), dtype=api.ROUND_DTYPE)
+    nd = np.zeros(ni, dtype=np.int32)
+    api.sp_run_host(ses.ctx, n, w.feats, w.app, w.arrival_ns, w.deadline_ns, w.instance, w.t0_ns,
+                    np.full(ni, -1, dtype=np.int32), 10_000, reqs, rounds, cap, nd)
+    assert np.array_equal(reqs, ref.reqs) and np.array_equal(nd, ref.n_rounds)
+    for k in range(ni):
+        assert np.array_equal(rounds[k, :nd[k]], ref.rounds[k, :nd[k]])
+    ses.close()
+
+
+def test_errors_are_reported_not_crashes():
+    import torch
+    from paper_2505_06641_b200 import api, runner
+    w = synth.make_workload("C1")
+    ses = runner.Session(w)
+    ses.upload(); ses.alloc_outputs(8); ses.score()
+    with pytest.raises(api.SpError) as e:           # second score without reset
+        dv = ses.dev
+        api.sp_score(ses.ctx, ses.n, dv["feats"], dv["app"], dv["arrival"], dv["deadline"], None, None)
+    assert e.value.status == api.SP_ESTATE
+    ses.dev["app"][5] = 77                          # out-of-range application id
+    ses.score(); ses.schedule(8)
+    with pytest.raises(api.SpError) as e:
+        api.sp_check(ses.ctx)
+    assert e.value.status == api.SP_EINVAL
+    assert int(ses.n_done.cpu()[0]) == 0            # nothing was scheduled from a rejected table
+    ses.dev["app"][5] = 0
+    ses.score(); ses.schedule(8); api.sp_check(ses.ctx)
+    assert int(ses.n_done.cpu()[0]) > 0
+    w.batch_sizes = np.asarray([4, 2], dtype=np.int32)
+    with pytest.raises(api.SpError) as e:
+        api.sp_load_profiles(ses.ctx, w)
+    assert e.value.status == api.SP_EINVAL
+    ses.close()
