@@ -94,6 +94,7 @@ typedef struct {
 
 typedef struct {
     int32_t trace_mode;   /* 0: every scored request is pending at once; 1: a request joins when arrival <= clock */
+    int32_t timing;       /* 1: bracket the scoring and the scheduling kernel with CUDA events (see sp_stats) */
     double guard_utility; /* relative margin under which candidate utilities are re-evaluated in fp64 (default 1e-4) */
     double guard_priority;/* same for group priorities (default 2e-5) */
 } sp_options;
@@ -104,6 +105,10 @@ typedef struct {
     int64_t exact_utility;     /* rounds whose candidate was decided in fp64 */
     int64_t exact_priority;    /* rounds whose application was decided in fp64 */
     int64_t exact_rows;        /* request rows re-scored in fp64 */
+    /* With sp_options.timing: device time of the scoring kernel / the scheduling kernel alone, summed over the
+     * calls since the previous sp_get_stats() (at most 512 calls are kept), and the number of calls summed. */
+    int64_t score_calls, sched_calls;
+    double score_kernel_ms, sched_kernel_ms;
 } sp_stats;
 
 /* Creates a context on CUDA device `device` that enqueues on `cuda_stream` (a cudaStream_t; NULL = the

@@ -50,12 +50,14 @@ class _Profiles(C.Structure):
 
 
 class _Options(C.Structure):
-    _fields_ = [("trace_mode", C.c_int32), ("guard_utility", C.c_double), ("guard_priority", C.c_double)]
+    _fields_ = [("trace_mode", C.c_int32), ("timing", C.c_int32), ("guard_utility", C.c_double),
+                ("guard_priority", C.c_double)]
 
 
 class _Stats(C.Structure):
     _fields_ = [("kernel_launches", C.c_int64), ("rounds", C.c_int64), ("exact_utility", C.c_int64),
-                ("exact_priority", C.c_int64), ("exact_rows", C.c_int64)]
+                ("exact_priority", C.c_int64), ("exact_rows", C.c_int64), ("score_calls", C.c_int64),
+                ("sched_calls", C.c_int64), ("score_kernel_ms", C.c_double), ("sched_kernel_ms", C.c_double)]
 
 
 _lib = None
@@ -153,8 +155,8 @@ def sp_load_profiles(ctx: int, w) -> None:
 
 
 def sp_set_options(ctx: int, trace_mode: bool = False, guard_utility: float = 1e-4,
-                   guard_priority: float = 2e-5) -> None:
-    o = _Options(int(bool(trace_mode)), float(guard_utility), float(guard_priority))
+                   guard_priority: float = 2e-5, timing: bool = False) -> None:
+    o = _Options(int(bool(trace_mode)), int(bool(timing)), float(guard_utility), float(guard_priority))
     _ok(ctx, load_library().sp_set_options(ctx, C.byref(o)))
 
 
@@ -198,7 +200,7 @@ def sp_check(ctx: int) -> None:
 def sp_get_stats(ctx: int) -> dict:
     s = _Stats()
     _ok(ctx, load_library().sp_get_stats(ctx, C.byref(s)))
-    return {k: int(getattr(s, k)) for k, _ in _Stats._fields_}
+    return {k: getattr(s, k) for k, _ in _Stats._fields_}
 
 
 def sp_run_host(ctx: int, n: int, feats: np.ndarray, app: np.ndarray, arrival_ns: np.ndarray,

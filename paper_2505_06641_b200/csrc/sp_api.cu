@@ -36,7 +36,8 @@ struct sp_ctx {
     HostProfiles hp;
     DevProfiles P{};
     DevTable tb{};
-    sp_options opt{0, 1e-4, 2e-5};
+    sp_options opt{0, 0, 1e-4, 2e-5};
+    std::vector<cudaEvent_t> ev_score, ev_sched;   // start/stop pairs recorded since the last sp_get_stats
     int64_t launches = 0;
     int sched_threads = 1024;
     int small_ct = 0;            // labels per lane of the small-head kernel, 0 = use the tiled kernel
@@ -143,6 +144,30 @@ __global__ void k_init_requests(sp_req_rec *recs, unsigned char *exact, int64_t 
     exact[i] = 0;
 }
 
+constexpr size_t kMaxTimedCalls = 512;
+
+// Records an event on the context's stream and keeps it in `list` (timing option only).
+sp_status mark(sp_ctx *c, std::vector<cudaEvent_t> &list) {
+    if (!c->opt.timing || list.size() >= 2 * kMaxTimedCalls) return SP_OK;
+    cudaEvent_t e;
+    SP_CUDA(c, cudaEventCreate(&e));
+    list.push_back(e);
+    SP_CUDA(c, cudaEventRecord(e, c->stream));
+    return SP_OK;
+}
+
+double drain_events(std::vector<cudaEvent_t> &list, int64_t *calls) {
+    double ms = 0.0;
+    *calls = 0;
+    for (size_t k = 0; k + 1 < list.size(); k += 2) {
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, list[k], list[k + 1]) == cudaSuccess) { ms += t; ++*calls; }
+    }
+    for (cudaEvent_t e : list) cudaEventDestroy(e);
+    list.clear();
+    return ms;
+}
+
 int small_ct_for(int C) { return C <= 10 ? 5 : C <= 20 ? 10 : C <= 32 ? 16 : C <= 64 ? 32 : 0; }
 
 template <int CT>
@@ -183,6 +208,9 @@ void sp_destroy(sp_ctx *c) {
     if (!c) return;
     cudaSetDevice(c->device);
     cudaStreamSynchronize(c->stream);
+    int64_t dummy;
+    drain_events(c->ev_score, &dummy);
+    drain_events(c->ev_sched, &dummy);
     Buf *all[] = {&c->W, &c->bias, &c->recall, &c->prior, &c->prior_dot, &c->prior_sum, &c->lat_alpha, &c->lat_beta,
                   &c->swap, &c->state, &c->zbuf, &c->flags, &c->stats, &c->cnt, &c->gstart, &c->cursor,
                   &c->small_start, &c->tiled_start, &c->acc32, &c->v32, &c->acc64, &c->v64, &c->exact, &c->recs,
@@ -414,6 +442,7 @@ sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, 
                                             (int32_t *)c->small_start.p);
     SP_TRY(launched(c, "k_group_scan"));
     if (n > 0) {
+        SP_TRY(mark(c, c->ev_score));
         if (c->small_ct) {
             const int grid = (int)(n / kSmallRows + P.I);
             switch (c->small_ct) {
@@ -434,6 +463,7 @@ sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, 
                                                                          (const int *)c->flags.p);
             SP_TRY(launched(c, "k_score_tiled"));
         }
+        SP_TRY(mark(c, c->ev_score));
     }
     c->have_table = true;
     return SP_OK;
@@ -482,8 +512,10 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
     sp.sort_cap = sort_cap;
     const SchedSmem L(sort_cap, P.Mmax, sp.bmax, kMaxModelsPerApp * kMaxBatchSizes);
     SP_CUDA(c, cudaFuncSetAttribute(k_sched, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.end));
+    SP_TRY(mark(c, c->ev_sched));
     k_sched<<<P.I, c->sched_threads, L.end, c->stream>>>(sp);
-    return launched(c, "k_sched");
+    SP_TRY(launched(c, "k_sched"));
+    return mark(c, c->ev_sched);
 }
 
 sp_status sp_check(sp_ctx *c) {
@@ -508,6 +540,8 @@ sp_status sp_get_stats(sp_ctx *c, sp_stats *out) {
     out->kernel_launches = c->launches;
     out->rounds = (int64_t)s[0]; out->exact_utility = (int64_t)s[1]; out->exact_priority = (int64_t)s[2];
     out->exact_rows = (int64_t)s[3];
+    out->score_kernel_ms = drain_events(c->ev_score, &out->score_calls);
+    out->sched_kernel_ms = drain_events(c->ev_sched, &out->sched_calls);
     return SP_OK;
 }
 
