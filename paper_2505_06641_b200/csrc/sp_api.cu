@@ -45,7 +45,7 @@ struct sp_ctx {
     // profile buffers
     Buf W, bias, recall, prior, prior_dot, prior_sum, lat_alpha, lat_beta, swap;
     // per-instance state and scratch
-    Buf state, zbuf, flags, stats, cnt, gstart, cursor, small_start, tiled_start;
+    Buf state, zbuf, flags, stats, cnt, gstart, cursor, small_start, tiled_start, small_tiles;
     // per-request buffers
     Buf acc32, v32, acc64, v64, exact, recs, perm, q_id0, q_id1, q_dl0, q_dl1, q_pw0, q_pw1, sort_scratch;
     // staging of sp_run_host
@@ -174,8 +174,7 @@ template <int CT>
 sp_status launch_small(sp_ctx *c, int grid, float *acc_out) {
     auto kern = k_score_small<CT>;
     SP_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->small_smem));
-    kern<<<grid, kSmallThreads, c->small_smem, c->stream>>>(c->P, c->tb, (const int32_t *)c->small_start.p, acc_out,
-                                                            (const int *)c->flags.p);
+    kern<<<grid, kSmallThreads, c->small_smem, c->stream>>>(c->P, c->tb, (const int4 *)c->small_tiles.p, acc_out);
     return launched(c, "k_score_small");
 }
 
@@ -213,7 +212,7 @@ void sp_destroy(sp_ctx *c) {
     drain_events(c->ev_sched, &dummy);
     Buf *all[] = {&c->W, &c->bias, &c->recall, &c->prior, &c->prior_dot, &c->prior_sum, &c->lat_alpha, &c->lat_beta,
                   &c->swap, &c->state, &c->zbuf, &c->flags, &c->stats, &c->cnt, &c->gstart, &c->cursor,
-                  &c->small_start, &c->tiled_start, &c->acc32, &c->v32, &c->acc64, &c->v64, &c->exact, &c->recs,
+                  &c->small_start, &c->tiled_start, &c->small_tiles, &c->acc32, &c->v32, &c->acc64, &c->v64, &c->exact, &c->recs,
                   &c->perm, &c->q_id0, &c->q_id1, &c->q_dl0, &c->q_dl1, &c->q_pw0, &c->q_pw1, &c->sort_scratch,
                   &c->h_feats, &c->h_app, &c->h_arrival, &c->h_deadline, &c->h_instance, &c->h_t0, &c->h_loaded,
                   &c->h_rounds, &c->h_ndone};
@@ -442,9 +441,16 @@ sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, 
                                             (int32_t *)c->small_start.p);
     SP_TRY(launched(c, "k_group_scan"));
     if (n > 0) {
+        int grid = 0;
+        if (c->small_ct) {
+            grid = (int)(n / kSmallRows + P.I);
+            SP_TRY(ensure(c, c->small_tiles, (size_t)grid * sizeof(int4)));
+            k_small_tiles<<<(grid + 255) / 256, 256, 0, c->stream>>>(P, tb, (const int32_t *)c->small_start.p, grid,
+                                                                     (int4 *)c->small_tiles.p, (const int *)c->flags.p);
+            SP_TRY(launched(c, "k_small_tiles"));
+        }
         SP_TRY(mark(c, c->ev_score));
         if (c->small_ct) {
-            const int grid = (int)(n / kSmallRows + P.I);
             switch (c->small_ct) {
                 case 5: SP_TRY(launch_small<5>(c, grid, acc_out)); break;
                 case 10: SP_TRY(launch_small<10>(c, grid, acc_out)); break;
@@ -454,7 +460,7 @@ sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, 
         } else {
             k_group_scatter<<<gb, 256, 0, c->stream>>>(P, tb, (const int *)c->flags.p);
             SP_TRY(launched(c, "k_group_scatter"));
-            const int grid = (int)(n / kTiledRows + (int64_t)nkeys);
+            grid = (int)(n / kTiledRows + (int64_t)nkeys);
             if (P.dtype == SP_BF16)
                 k_score_tiled<true><<<grid, kTiledThreads, 0, c->stream>>>(P, tb, (const int32_t *)c->tiled_start.p, acc_out,
                                                                         (const int *)c->flags.p);

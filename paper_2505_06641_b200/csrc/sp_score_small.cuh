@@ -51,14 +51,89 @@ __device__ __forceinline__ void load_half_row(float (&w)[CT], const float *p) {
     if (CT % 2) w[CT - 1] = p[CT - 1];
 }
 
+// Tile descriptors: tile t -> (instance, first request relative to the instance, rows), instance = -1 past the end.
+__global__ void k_small_tiles(DevProfiles P, DevTable tb, const int32_t *__restrict__ small_start, int n_tiles,
+                              int4 *__restrict__ desc, const int *__restrict__ flags) {
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= n_tiles) return;
+    int4 d = make_int4(-1, 0, 0, 0);
+    if (!flags[1] && t < small_start[P.I]) {
+        int lo = 0, hi = P.I;                 // instance with small_start[inst] <= t < small_start[inst + 1]
+        while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (small_start[mid] <= t) lo = mid; else hi = mid; }
+        const int64_t i0 = tb.gstart[(int64_t)lo * P.A], i1 = tb.gstart[(int64_t)(lo + 1) * P.A];
+        const int64_t r0 = (int64_t)(t - small_start[lo]) * kSmallRows;
+        d = make_int4(lo, (int)r0, (int)((i1 - i0 - r0) < kSmallRows ? (i1 - i0 - r0) : kSmallRows), 0);
+    }
+    desc[t] = d;
+}
+
+// Copies `nrows` rows of C floats from global memory into the two-halves layout [row][2][CTP] used by the
+// kernel below (lane half h owns labels h*CT .. h*CT+CT-1); positions without a label get `fill`.
+// Loads are issued in batches so that one global-memory latency covers many elements.
+template <int CT>
+__device__ __forceinline__ void stage_halves(float *__restrict__ dst, const float *__restrict__ src, int nrows, int C,
+                                             float fill) {
+    constexpr int CTP = (CT + 3) & ~3;
+    constexpr int U = 8;
+    const int tid = threadIdx.x;
+    if ((C & 3) == 0 && (((uintptr_t)src) & 15) == 0) {
+        // labels come in aligned groups of four: vector loads, scalar scatter; padding written separately
+        const int c4 = C >> 2, total = nrows * c4;
+        for (int q0 = tid; q0 < total; q0 += kSmallThreads * U) {
+            float4 v[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int q = q0 + u * kSmallThreads;
+                v[u] = q < total ? reinterpret_cast<const float4 *>(src)[q] : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int q = q0 + u * kSmallThreads;
+                if (q < total) {
+                    const int row = q / c4, c = (q - row * c4) * 4;
+                    const float e[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int cc = c + k, h = cc >= CT ? 1 : 0;
+                        dst[(row * 2 + h) * CTP + cc - h * CT] = e[k];
+                    }
+                }
+            }
+        }
+        const int lab1 = C - CT > 0 ? C - CT : 0;         // labels in the second half
+        const int lab0 = C < CT ? C : CT;
+        const int pad0 = CTP - lab0, pad1 = CTP - lab1, pads = pad0 + pad1;
+        for (int k = tid; k < nrows * pads; k += kSmallThreads) {
+            const int row = k / pads, r = k - row * pads;
+            if (r < pad0) dst[(row * 2) * CTP + lab0 + r] = fill;
+            else dst[(row * 2 + 1) * CTP + lab1 + (r - pad0)] = fill;
+        }
+    } else {
+        const int total = nrows * 2 * CTP;
+        for (int k0 = tid; k0 < total; k0 += kSmallThreads * U) {
+            float v[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int k = k0 + u * kSmallThreads;
+                const int c2 = k % (2 * CTP), row = k / (2 * CTP);
+                const int h = c2 / CTP, cc = c2 - h * CTP, c = h * CT + cc;
+                v[u] = (k < total && cc < CT && c < C) ? src[(int64_t)row * C + c] : fill;
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int k = k0 + u * kSmallThreads;
+                if (k < total) dst[k] = v[u];
+            }
+        }
+    }
+}
+
 // CT = labels per lane (two lanes share a request, so C <= 2*CT).
 template <int CT>
 __global__ void __launch_bounds__(kSmallThreads, 2)
-k_score_small(DevProfiles P, DevTable tb, const int32_t *__restrict__ small_start, float *__restrict__ acc_out,
-              const int *__restrict__ flags) {
+k_score_small(DevProfiles P, DevTable tb, const int4 *__restrict__ tiles, float *__restrict__ acc_out) {
     constexpr int CTP = (CT + 3) & ~3;
     extern __shared__ __align__(16) float smem[];
-    __shared__ int s_tile_inst, s_row0, s_rows;
     __shared__ int s_cnt[kMaxApps], s_first[kMaxApps + 1], s_unit0[kMaxApps + 1];
     __shared__ short s_phys[kSmallRows];          // request of the tile -> row in shared memory
     __shared__ short s_local[kSmallRows];         // row in shared memory -> request of the tile
@@ -67,26 +142,13 @@ k_score_small(DevProfiles P, DevTable tb, const int32_t *__restrict__ small_star
     const int A = P.A, C = P.C, D = P.D;
     const SmallSmem L(A, D, P.sumM, CTP);
 
-    if (tid == 0) {
-        // tile -> (instance, first row): binary search in the per-instance tile prefix
-        const int t = blockIdx.x;
-        int lo = 0, hi = P.I;                      // find inst with small_start[inst] <= t < small_start[inst+1]
-        if (flags[1] || t >= small_start[P.I]) { s_tile_inst = -1; }
-        else {
-            while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (small_start[mid] <= t) lo = mid; else hi = mid; }
-            s_tile_inst = lo;
-            const int64_t i0 = tb.gstart[(int64_t)lo * A], i1 = tb.gstart[(int64_t)(lo + 1) * A];
-            const int64_t r0 = i0 + (int64_t)(t - small_start[lo]) * kSmallRows;
-            s_row0 = (int)(r0 - i0);
-            s_rows = (int)((i1 - r0) < kSmallRows ? (i1 - r0) : kSmallRows);
-        }
-    }
+    const int4 desc = tiles[blockIdx.x];
+    const int inst = desc.x;
+    if (inst < 0) return;
+    const int64_t row0 = tb.gstart[(int64_t)inst * A] + desc.y;
+    const int rows = desc.z;
     if (tid < kMaxApps) s_cnt[tid] = 0;
     __syncthreads();
-    const int inst = s_tile_inst;
-    if (inst < 0) return;
-    const int64_t row0 = tb.gstart[(int64_t)inst * A] + s_row0;
-    const int rows = s_rows;
 
     // ---- applications of the tile's requests -> rows in application order
     int my_app = 0, my_rank = 0;
@@ -120,27 +182,9 @@ k_score_small(DevProfiles P, DevTable tb, const int32_t *__restrict__ small_star
             const int r = k / chunks, q = k - r * chunks;
             cp_async16(xs + s_phys[r] * (D + 4) + q * 4, feats + (row0 + r) * D + q * 4);
         }
-        const float *Wg = (const float *)P.W + (int64_t)inst * A * D * C;
-        float *ws = smem + L.w;
-        for (int k = tid; k < A * D * 2 * CTP; k += kSmallThreads) {
-            const int c2 = k % (2 * CTP), ad = k / (2 * CTP);
-            const int h = c2 / CTP, cc = c2 - h * CTP, c = h * CT + cc;
-            ws[k] = (cc < CT && c < C) ? Wg[(int64_t)ad * C + c] : 0.f;
-        }
-        const float *bg = P.bias + (int64_t)inst * A * C;
-        float *bs = smem + L.bias;
-        for (int k = tid; k < A * 2 * CTP; k += kSmallThreads) {
-            const int c2 = k % (2 * CTP), a = k / (2 * CTP);
-            const int h = c2 / CTP, cc = c2 - h * CTP, c = h * CT + cc;
-            bs[k] = (cc < CT && c < C) ? bg[a * C + c] : -INFINITY;
-        }
-        const float *rg = P.recall + (int64_t)inst * P.sumM * C;
-        float *rs = smem + L.recall;
-        for (int k = tid; k < P.sumM * 2 * CTP; k += kSmallThreads) {
-            const int c2 = k % (2 * CTP), g = k / (2 * CTP);
-            const int h = c2 / CTP, cc = c2 - h * CTP, c = h * CT + cc;
-            rs[k] = (cc < CT && c < C) ? rg[g * C + c] : 0.f;
-        }
+        stage_halves<CT>(smem + L.w, (const float *)P.W + (int64_t)inst * A * D * C, A * D, C, 0.f);
+        stage_halves<CT>(smem + L.bias, P.bias + (int64_t)inst * A * C, A, C, -INFINITY);
+        stage_halves<CT>(smem + L.recall, P.recall + (int64_t)inst * P.sumM * C, P.sumM, C, 0.f);
         cp_async_commit_wait_all();
     }
     __syncthreads();
