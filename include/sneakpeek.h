@@ -186,6 +186,39 @@ sp_status sp_run_host(sp_ctx *ctx, int64_t n, const void *feats, const int32_t *
                       const int32_t *loaded0, int32_t max_rounds, sp_req_rec *reqs_out,
                       sp_round_rec *rounds_out, int64_t cap, int32_t *n_done);
 
+/*
+ * Scoring for callers that must not allocate.  (The paper has no counterpart to this entry point; it exists
+ * for deployment reasons only.)  Some hosts of this library run with a fixed device-memory budget handed out
+ * at start-up -- a serving process that has given all remaining memory to its own pool, or a real-time loop
+ * in which a driver allocation (which may block or fail) is not acceptable -- so the context-based calls
+ * above, which grow their buffers with cudaMalloc, are closed to them.  This call does steps a1-a4 of
+ * sp_score() for ONE instance (no Dirichlet prior) and allocates nothing, neither through CUDA nor through any
+ * library: its scratch (per-application counters, prefix sums, the request permutation; about 0.5 MB) is a
+ * fixed array inside the library image, which every GPU that loads the library holds until the process ends.
+ *
+ *   head      HOST struct; models_per_app is a HOST array, head_w [A][D][C], head_b [A][C], recall [sumM][C]
+ *             are DEVICE arrays (inputs, the caller's).
+ *   n         0 .. 65,536 requests; larger n is rejected with SP_EINVAL and a message (the array is not grown).
+ *   feats     DEVICE [n][D]; app DEVICE [n]; acc_out DEVICE [n][Mmax] float; v_out DEVICE [n] float (outputs).
+ *   errbuf    HOST, optional: receives a text when the result is not SP_OK.
+ *
+ * The call returns when the work is done (it waits for the stream) and reports bad application ids as
+ * SP_EINVAL.  The first call on a device looks up the array's device address (once per device); make that
+ * first call before starting any stream capture.  All calls in a process share the one array per device: it
+ * keeps the last call's contents, the call clears what has to start at zero, and two calls that overlap on
+ * the same GPU (different streams or threads) race on it -- serialise them.
+ */
+typedef struct {
+    int32_t n_apps, n_classes, feat_dim, feat_dtype;
+    const int32_t *models_per_app; /* HOST [A] */
+    const void *head_w;            /* DEVICE [A][D][C] */
+    const float *head_b;           /* DEVICE [A][C] */
+    const float *recall;           /* DEVICE [sumM][C] */
+} sp_static_head;
+
+sp_status sp_score_static(int device, void *cuda_stream, const sp_static_head *head, int64_t n, const void *feats,
+                          const int32_t *app, float *acc_out, float *v_out, char *errbuf, int32_t errbuf_len);
+
 #ifdef __cplusplus
 }
 #endif

@@ -30,7 +30,7 @@ assert ROUND_DTYPE.itemsize == 64 and REQ_DTYPE.itemsize == 24
 
 EXPORTS = ["sp_create", "sp_destroy", "sp_last_error", "sp_load_profiles", "sp_set_options", "sp_set_clock",
            "sp_set_clocks", "sp_score", "sp_get_scores", "sp_schedule_round", "sp_get_requests", "sp_get_clocks",
-           "sp_reset", "sp_check", "sp_get_stats", "sp_run_host"]
+           "sp_reset", "sp_check", "sp_get_stats", "sp_run_host", "sp_score_static"]
 
 
 class SpError(RuntimeError):
@@ -58,6 +58,11 @@ class _Stats(C.Structure):
     _fields_ = [("kernel_launches", C.c_int64), ("rounds", C.c_int64), ("exact_utility", C.c_int64),
                 ("exact_priority", C.c_int64), ("exact_rows", C.c_int64), ("score_calls", C.c_int64),
                 ("sched_calls", C.c_int64), ("score_kernel_ms", C.c_double), ("sched_kernel_ms", C.c_double)]
+
+
+class _StaticHead(C.Structure):
+    _fields_ = [("n_apps", C.c_int32), ("n_classes", C.c_int32), ("feat_dim", C.c_int32), ("feat_dtype", C.c_int32),
+                ("models_per_app", C.c_void_p), ("head_w", C.c_void_p), ("head_b", C.c_void_p), ("recall", C.c_void_p)]
 
 
 _lib = None
@@ -91,6 +96,7 @@ def load_library():
     lib.sp_check.argtypes = [vp]
     lib.sp_get_stats.argtypes = [vp, C.POINTER(_Stats)]
     lib.sp_run_host.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, i64, vp]
+    lib.sp_score_static.argtypes = [C.c_int, vp, C.POINTER(_StaticHead), i64, vp, vp, vp, vp, C.c_char_p, i32]
     for name in EXPORTS:
         if name not in ("sp_destroy", "sp_last_error"):
             getattr(lib, name).restype = C.c_int
@@ -210,3 +216,20 @@ def sp_run_host(ctx: int, n: int, feats: np.ndarray, app: np.ndarray, arrival_ns
     _ok(ctx, load_library().sp_run_host(ctx, int(n), _host(feats), _host(app), _host(arrival_ns), _host(deadline_ns),
                                         _host(instance), _host(t0_ns), _host(loaded0), int(max_rounds),
                                         _host(reqs_out), _host(rounds_out), int(cap), _host(n_done)))
+
+
+def sp_score_static(device: int, cuda_stream: int, n_apps: int, n_classes: int, feat_dim: int, feat_dtype: int,
+                    models_per_app: np.ndarray, head_w, head_b, recall, n: int, feats, app, acc_out, v_out) -> None:
+    """Allocation-free scoring of one instance: device tensors in, device tensors out, fixed built-in scratch.
+
+    ``models_per_app`` is a host array; ``head_w``, ``head_b``, ``recall``, ``feats``, ``app`` and the two outputs
+    are CUDA tensors.  Raises ``SpError`` (with the library's message) on bad arguments, e.g. n > 65,536.
+    """
+    mpa = np.ascontiguousarray(models_per_app, dtype=np.int32)
+    head = _StaticHead(int(n_apps), int(n_classes), int(feat_dim), int(feat_dtype), _host(mpa), _dev(head_w),
+                       _dev(head_b), _dev(recall))
+    err = C.create_string_buffer(256)
+    st = load_library().sp_score_static(int(device), C.c_void_p(cuda_stream or None), C.byref(head), int(n),
+                                        _dev(feats), _dev(app), _dev(acc_out), _dev(v_out), err, 256)
+    if st != SP_OK:
+        raise SpError(st, err.value.decode())

@@ -588,3 +588,96 @@ sp_status sp_run_host(sp_ctx *c, int64_t n, const void *feats, const int32_t *ap
 }
 
 }  // extern "C"
+
+// =================================================================================================
+// Scoring without any allocation.  The scratch that the grouping pass and the tiled scoring kernel need
+// (per-application counters, prefix sums and the request permutation) lives in one file-scope device array
+// instead of context-owned cudaMalloc'ed buffers.  Every GPU that loads this library holds the array until
+// the process exits.
+namespace {
+
+constexpr int64_t kStaticMaxRequests = 65536;
+
+struct StaticScratch {                       // layout of the array below
+    int flags[2];                            // must start at 0
+    int32_t cnt[kMaxApps];                   // must start at 0
+    int32_t cursor[kMaxApps];                // must start at 0
+    int32_t tiled_start[kMaxApps + 1];
+    int32_t small_start[2];
+    int64_t gstart[kMaxApps + 1];
+    int64_t perm[kStaticMaxRequests];
+};
+
+static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScratch)];
+
+constexpr int kStaticMaxDevices = 64;
+StaticScratch *g_static_ptr[kStaticMaxDevices] = {};   // device address of the array, per device
+
+void static_msg(char *buf, int32_t len, const std::string &m) {
+    if (buf && len > 0) { std::snprintf(buf, (size_t)len, "%s", m.c_str()); }
+}
+
+}  // namespace
+
+extern "C" sp_status sp_score_static(int device, void *cuda_stream, const sp_static_head *head, int64_t n,
+                                     const void *feats, const int32_t *app, float *acc_out, float *v_out,
+                                     char *errbuf, int32_t errbuf_len) {
+#define SP_STATIC_FAIL(code, msg) do { static_msg(errbuf, errbuf_len, (msg)); return (code); } while (0)
+#define SP_STATIC_CUDA(call)                                                                        \
+    do {                                                                                            \
+        cudaError_t e_ = (call);                                                                    \
+        if (e_ != cudaSuccess) SP_STATIC_FAIL(SP_ECUDA, std::string(#call) + ": " + cudaGetErrorString(e_)); \
+    } while (0)
+    if (!head) SP_STATIC_FAIL(SP_EINVAL, "head is NULL");
+    if (n < 0 || n > kStaticMaxRequests)
+        SP_STATIC_FAIL(SP_EINVAL, "n is outside 0.." + std::to_string(kStaticMaxRequests) +
+                                      ", the capacity of the built-in scratch array");
+    const int A = head->n_apps, C = head->n_classes, D = head->feat_dim;
+    if (A < 1 || A > kMaxApps || C < 1 || C > kMaxClasses || D < 1 || !head->models_per_app || !head->head_w ||
+        !head->head_b || !head->recall || (head->feat_dtype != SP_F32 && head->feat_dtype != SP_BF16))
+        SP_STATIC_FAIL(SP_EINVAL, "bad head description (shapes out of range or NULL array)");
+    if (n > 0 && (!feats || !app || !acc_out || !v_out)) SP_STATIC_FAIL(SP_EINVAL, "a request or output array is NULL");
+    if (device < 0 || device >= kStaticMaxDevices) SP_STATIC_FAIL(SP_EINVAL, "device index out of range");
+    DevProfiles P{};
+    P.I = 1; P.A = A; P.C = C; P.D = D; P.dtype = head->feat_dtype;
+    for (int a = 0; a < A; ++a) {
+        const int m = head->models_per_app[a];
+        if (m < 1 || m > kMaxModelsPerApp) SP_STATIC_FAIL(SP_EINVAL, "models_per_app entries must be 1..16");
+        P.mfirst[a] = P.sumM; P.sumM += m; P.Mmax = m > P.Mmax ? m : P.Mmax;
+    }
+    P.mfirst[A] = P.sumM;
+    P.W = head->head_w; P.bias = head->head_b; P.recall = head->recall; P.tau = 1.0;
+
+    SP_STATIC_CUDA(cudaSetDevice(device));
+    if (!g_static_ptr[device]) {               // set-up, once per device, with that device current
+        void *p = nullptr;
+        SP_STATIC_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
+        g_static_ptr[device] = static_cast<StaticScratch *>(p);
+    }
+    StaticScratch *s = g_static_ptr[device];
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (n == 0) return SP_OK;
+
+    DevTable tb{};
+    tb.n = n; tb.feats = feats; tb.app = app; tb.acc32 = acc_out; tb.v32 = v_out;
+    tb.cnt = s->cnt; tb.cursor = s->cursor; tb.gstart = s->gstart; tb.perm = s->perm;
+    // the array keeps the previous call's contents: clear the parts that are accumulated into
+    SP_STATIC_CUDA(cudaMemsetAsync(s, 0, offsetof(StaticScratch, tiled_start), stream));
+    const unsigned gb = (unsigned)((n + 255) / 256);
+    k_group_count<<<gb, 256, 0, stream>>>(P, tb, 0, s->flags);
+    k_group_scan<<<1, 1024, 0, stream>>>(A, A, s->cnt, s->gstart, s->tiled_start, s->small_start);
+    k_group_scatter<<<gb, 256, 0, stream>>>(P, tb, s->flags);
+    const int grid = (int)(n / kTiledRows + A);
+    if (P.dtype == SP_BF16)
+        k_score_tiled<true><<<grid, kTiledThreads, 0, stream>>>(P, tb, s->tiled_start, nullptr, s->flags);
+    else
+        k_score_tiled<false><<<grid, kTiledThreads, 0, stream>>>(P, tb, s->tiled_start, nullptr, s->flags);
+    SP_STATIC_CUDA(cudaGetLastError());
+    int flags[2] = {0, 0};
+    SP_STATIC_CUDA(cudaMemcpyAsync(flags, s->flags, sizeof flags, cudaMemcpyDeviceToHost, stream));
+    SP_STATIC_CUDA(cudaStreamSynchronize(stream));
+    if (flags[1]) SP_STATIC_FAIL(SP_EINVAL, "an application id is outside 0..n_apps-1; nothing was written");
+    return SP_OK;
+#undef SP_STATIC_CUDA
+#undef SP_STATIC_FAIL
+}
