@@ -10,6 +10,7 @@
 #include "sp_group.cuh"
 #include "sp_score_small.cuh"
 #include "sp_score_tiled.cuh"
+#include "sp_score_mma.cuh"
 #include "sp_sched.cuh"
 
 using namespace sp;
@@ -42,6 +43,8 @@ struct sp_ctx {
     int sched_threads = 1024;
     int small_ct = 0;            // labels per lane of the small-head kernel, 0 = use the tiled kernel
     size_t small_smem = 0;
+    int mma_ct = 0;              // logit columns per epilogue thread of the tensor-core kernel, 0 = not used
+    int n_sms = 1;
     // profile buffers
     Buf W, bias, recall, prior, prior_dot, prior_sum, lat_alpha, lat_beta, swap;
     // per-instance state and scratch
@@ -178,6 +181,48 @@ sp_status launch_small(sp_ctx *c, int grid, float *acc_out) {
     return launched(c, "k_score_small");
 }
 
+// cuTensorMapEncodeTiled through the runtime's driver entry-point lookup (the library does not link libcuda).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// Tensor map over the fp32 feature matrix [n][D]: boxes of 128 requests x 32 features, 128-byte swizzle,
+// zeros outside the matrix.
+sp_status feature_map(sp_ctx *c, CUtensorMap *map, const void *feats, int64_t n, int D) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return fail(c, SP_ECUDA, "cuTensorMapEncodeTiled is not available from this driver");
+    const cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)n};
+    const cuuint64_t strides[1] = {(cuuint64_t)D * 4};
+    const cuuint32_t box[2] = {(cuuint32_t)mma::kSlabK, (cuuint32_t)mma::kRows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void *>(feats), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(c, SP_ECUDA, "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r));
+    return SP_OK;
+}
+
+template <int CT>
+sp_status launch_mma(sp_ctx *c, const CUtensorMap &map, const mma::Params &prm) {
+    auto kern = mma::k_score_mma<CT>;
+    SP_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, mma::Smem::bytes));
+    const int grid = prm.n_tiles < c->n_sms ? prm.n_tiles : c->n_sms;
+    kern<<<grid, mma::kThreads, mma::Smem::bytes, c->stream>>>(map, prm);
+    return launched(c, "k_score_mma");
+}
+
 }  // namespace
 
 // =================================================================================================
@@ -193,6 +238,7 @@ sp_status sp_create(sp_ctx **out, int device, void *cuda_stream) {
     if (!c) return SP_ENOMEM;
     c->device = device;
     c->stream = (cudaStream_t)cuda_stream;
+    if (cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || c->n_sms < 1) c->n_sms = 1;
     if (ensure(c, c->flags, 2 * sizeof(int)) != SP_OK || ensure(c, c->stats, 4 * sizeof(unsigned long long)) != SP_OK ||
         cudaMemsetAsync(c->flags.p, 0, 2 * sizeof(int), c->stream) != cudaSuccess ||
         cudaMemsetAsync(c->stats.p, 0, 4 * sizeof(unsigned long long), c->stream) != cudaSuccess) {
@@ -322,7 +368,10 @@ sp_status sp_load_profiles(sp_ctx *c, const sp_profiles *p) {
     // kernel choices that depend on the shapes only
     c->sched_threads = I > 1 ? 128 : 1024;
     c->small_ct = 0;
-    if (p->feat_dtype == SP_F32 && D % 4 == 0 && C <= 64) {
+    c->mma_ct = 0;
+    if (p->feat_dtype == SP_F32 && D % 4 == 0 && D <= mma::kMaxD && A * C <= mma::kCols && sumM * C <= 1024) {
+        c->mma_ct = C <= 16 ? 16 : C <= 32 ? 32 : 64;
+    } else if (p->feat_dtype == SP_F32 && D % 4 == 0 && C <= 64) {
         const int ct = small_ct_for(C);
         const SmallSmem L(A, D, sumM, (ct + 3) & ~3);
         const size_t bytes = (size_t)L.end * sizeof(float);
@@ -442,15 +491,25 @@ sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, 
     SP_TRY(launched(c, "k_group_scan"));
     if (n > 0) {
         int grid = 0;
-        if (c->small_ct) {
+        if (c->small_ct || c->mma_ct) {
+            if (n / kSmallRows + P.I > 0x7fffffff / 2) return fail(c, SP_EINVAL, "too many requests for one call");
             grid = (int)(n / kSmallRows + P.I);
             SP_TRY(ensure(c, c->small_tiles, (size_t)grid * sizeof(int4)));
             k_small_tiles<<<(grid + 255) / 256, 256, 0, c->stream>>>(P, tb, (const int32_t *)c->small_start.p, grid,
                                                                      (int4 *)c->small_tiles.p, (const int *)c->flags.p);
             SP_TRY(launched(c, "k_small_tiles"));
         }
+        CUtensorMap x_map;
+        if (c->mma_ct) SP_TRY(feature_map(c, &x_map, feats, n, P.D));
         SP_TRY(mark(c, c->ev_score));
-        if (c->small_ct) {
+        if (c->mma_ct) {
+            mma::Params prm{P, tb, (const int4 *)c->small_tiles.p, grid, acc_out, (int *)c->flags.p};
+            switch (c->mma_ct) {
+                case 16: SP_TRY(launch_mma<16>(c, x_map, prm)); break;
+                case 32: SP_TRY(launch_mma<32>(c, x_map, prm)); break;
+                default: SP_TRY(launch_mma<64>(c, x_map, prm)); break;
+            }
+        } else if (c->small_ct) {
             switch (c->small_ct) {
                 case 5: SP_TRY(launch_small<5>(c, grid, acc_out)); break;
                 case 10: SP_TRY(launch_small<10>(c, grid, acc_out)); break;

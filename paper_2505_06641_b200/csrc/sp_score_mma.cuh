@@ -1,0 +1,559 @@
+// Tensor-core scoring kernel for small heads (fp32 features, D <= 128, all applications' labels fit
+// in 64 logit columns).  Persistent, warp-specialised, one thread block per SM.
+//
+// Per request (Section 4.1 + Eq. 9 + Eq. 12 of the paper):
+//   z = x W_a + b_a;  p = softmax(z);  theta = Dirichlet posterior mean;  acc_j = sum_c theta_c recall_j(c);
+//   v = 1 + population variance_j(acc_j).
+// The step is bound by reading x from HBM once; at ~10 flop per byte the FP32 pipes cannot keep up with
+// HBM3e, so the logits are computed by the tcgen05 tensor cores:
+//   * a tile is 128 consecutive requests of one instance; TMA brings it into shared memory as K-major,
+//     128-byte-swizzled slabs of 128 rows x 32 features (the layout the MMA reads directly);
+//   * the logits of ALL applications of the instance are computed for every row ([A*C] <= 64 columns);
+//     each row later keeps the columns of its own application, so rows need no regrouping;
+//   * fp32 accuracy from the tf32 unit: x = x_hi + x_lo and W = W_hi + W_lo with x_hi, W_hi the values
+//     truncated to tf32 (what the unit reads from a 32-bit container) and the remainders exact in fp32;
+//     z = x_hi [W_hi | W_lo] + x_lo W_hi accumulates in fp32 in tensor memory, the dropped x_lo W_lo term
+//     is below 2^-20 relative.  x_hi needs no conversion (it is the tile as loaded); converter warps
+//     write x_lo into a second ring of slabs and rebuild the W operand when the instance changes;
+//   * epilogue warps read the accumulator from tensor memory (one row per thread), add the bias, and do
+//     softmax, the recall contraction, the Dirichlet step and the variance in registers.
+// Every wait on an mbarrier is bounded; when a wait runs out the block raises kDevLimit and leaves.
+#pragma once
+
+#include <cuda.h>
+
+#include "sp_common.cuh"
+#include "sp_group.cuh"
+
+namespace sp {
+namespace mma {
+
+constexpr int kRows = 128;                 // requests per tile = MMA M
+constexpr int kSlabK = 32;                 // features per slab row (128 bytes)
+constexpr int kSlabBytes = kRows * 128;    // 16 KB: 128 rows x 128 bytes
+constexpr int kMaxD = 128;
+constexpr int kMaxSlabs = kMaxD / kSlabK;
+constexpr int kCols = 64;                  // logit columns (sum over applications of the label count)
+constexpr int kHiStages = 6;               // ring of slabs filled by TMA (x, read as x_hi)
+constexpr int kLoStages = 3;               // ring of slabs written by the converter warps (x_lo)
+constexpr int kTmemCols = 512;             // whole tensor memory: 2 accumulators of 128 columns, reads may overhang
+constexpr int kAccCols = 128;              // columns per accumulator: [x_hi W_hi + x_lo W_hi | x_hi W_lo]
+constexpr int kProducerWarp = 0, kMmaWarp = 1, kConvWarp0 = 2, kEpiWarp0 = 6;
+constexpr int kThreads = 32 * 10;
+constexpr int kConvThreads = 128, kEpiThreads = 128;
+constexpr int kWRegs = (kCols * kMaxD / 4) / kConvThreads;   // float4 registers per converter thread holding a raw head
+constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
+
+struct Smem {                               // byte offsets from the 1024-byte aligned base
+    static constexpr int w = 0;                                        // kMaxSlabs slabs: rows 0..63 W_hi, 64..127 W_lo
+    static constexpr int hi = w + kMaxSlabs * kSlabBytes;
+    static constexpr int lo = hi + kHiStages * kSlabBytes;
+    static constexpr int recall = lo + kLoStages * kSlabBytes;         // [sumM][C] floats, at most 1024
+    static constexpr int bias = recall + 1024 * 4;                     // [A*C] floats
+    static constexpr int prior = bias + kCols * 4;                     // prior_dot [sumM] (<= 256), prior_sum [A] (<= 16)
+    static constexpr int bars = prior + (256 + 16) * 4;
+    static constexpr int n_bars = 2 * kHiStages + 2 * kLoStages + 8;
+    static constexpr int misc = bars + n_bars * 8;                     // tmem base, abort flag
+    static constexpr int end = misc + 16;
+    static constexpr int bytes = end + 1024;                           // slack for the manual alignment
+};
+
+struct Params {
+    DevProfiles P;
+    DevTable tb;
+    const int4 *tiles;       // (instance, first request relative to the instance, rows, -)
+    int n_tiles;             // entries in `tiles` (those past the end have instance -1)
+    float *acc_out;          // optional second destination of acc
+    int *flags;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: false when the wait ran out (the block-wide abort flag is then set) or another thread gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63) == 0) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+            __nanosleep(64);
+        }
+    }
+}
+
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 2-D tiled TMA load (no multicast): box of the tensor map at (x = feature, y = request) -> shared memory.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+    uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;              // leading byte offset (not used by swizzled K-major layouts)
+    d |= (uint64_t)(1024 >> 4) << 32;    // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;              // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;              // 128-byte swizzle
+    return d;
+}
+// Instruction descriptor: tf32 x tf32 -> fp32, both operands K-major, M = 128, N = n.
+__host__ __device__ constexpr uint32_t instr_desc(int n) {
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kRows >> 4) << 24);
+}
+__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+// Arrives on the mbarrier once every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+template <int N>
+__device__ __forceinline__ void tmem_ld(uint32_t taddr, float (&r)[N]);
+template <>
+__device__ __forceinline__ void tmem_ld<16>(uint32_t taddr, float (&r)[16]) {
+    uint32_t v[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 16; ++i) r[i] = __uint_as_float(v[i]);
+}
+template <>
+__device__ __forceinline__ void tmem_ld<32>(uint32_t taddr, float (&r)[32]) {
+    uint32_t v[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) r[i] = __uint_as_float(v[i]);
+}
+template <>
+__device__ __forceinline__ void tmem_ld<64>(uint32_t taddr, float (&r)[64]) {
+    float a[32], b[32];
+    tmem_ld<32>(taddr, a);
+    tmem_ld<32>(taddr + 32, b);
+#pragma unroll
+    for (int i = 0; i < 32; ++i) { r[i] = a[i]; r[32 + i] = b[i]; }
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Value a tf32 operand takes from a 32-bit container: the low 13 mantissa bits are not read.
+__device__ __forceinline__ float tf32_part(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
+
+// exp(x) for x <= 0 from the ex2 unit: x * log2(e) is split into a rounded product and its exact residual
+// (plus the low part of log2(e)), and the residual is applied as a first-order correction, so the result
+// carries the unit's own error (about 2^-22 relative) instead of |x| * 2^-24 from the argument.
+__device__ __forceinline__ float exp_neg(float x) {
+    const float kL2eHi = 1.44269502162933349609375f, kL2eLo = 1.925963033500305e-08f;
+    x = fmaxf(x, -120.f);                       // exp(-120) flushes to zero; keeps -inf (padded labels) finite
+    const float r = x * kL2eHi;
+    const float e = fmaf(x, kL2eLo, fmaf(x, kL2eHi, -r));
+    float p;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(p) : "f"(r));
+    return fmaf(p * e, 0.693147182464599609375f, p);
+}
+
+// Barrier indices
+__device__ __forceinline__ constexpr int bar_full(int h) { return h; }
+__device__ __forceinline__ constexpr int bar_hi_free(int h) { return kHiStages + h; }
+__device__ __forceinline__ constexpr int bar_lo_ready(int l) { return 2 * kHiStages + l; }
+__device__ __forceinline__ constexpr int bar_lo_free(int l) { return 2 * kHiStages + kLoStages + l; }
+__device__ __forceinline__ constexpr int bar_acc_full(int b) { return 2 * kHiStages + 2 * kLoStages + b; }
+__device__ __forceinline__ constexpr int bar_acc_empty(int b) { return 2 * kHiStages + 2 * kLoStages + 2 + b; }
+constexpr int kBarWReady = 2 * kHiStages + 2 * kLoStages + 4;
+constexpr int kBarDrain = 2 * kHiStages + 2 * kLoStages + 5;
+constexpr int kBarEpiA = 2 * kHiStages + 2 * kLoStages + 6;   // epilogue threads: done reading the old tables
+constexpr int kBarEpiB = 2 * kHiStages + 2 * kLoStages + 7;   // epilogue threads: new tables written
+
+// Warp-uniform outcome of a bounded wait done by every lane.
+__device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    const bool ok = mbar_wait(bar, parity, abort_flag);
+    return __all_sync(0xffffffffu, ok);
+}
+
+// CT = power of two >= C: logit columns one epilogue thread keeps in registers.
+template <int CT>
+__global__ void __launch_bounds__(kThreads, 1)
+k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw_u32 = smem_u32(smem_raw);
+    const uint32_t base = (raw_u32 + 1023u) & ~1023u;
+    unsigned char *sm = smem_raw + (base - raw_u32);
+    float *recall_s = reinterpret_cast<float *>(sm + Smem::recall);
+    float *bias_s = reinterpret_cast<float *>(sm + Smem::bias);
+    float *prior_s = reinterpret_cast<float *>(sm + Smem::prior);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(sm + Smem::misc);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(sm + Smem::misc + 4);
+    auto bar = [&](int i) -> uint32_t { return base + Smem::bars + 8u * (uint32_t)i; };
+
+    const DevProfiles &P = prm.P;
+    const DevTable &tb = prm.tb;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int A = P.A, C = P.C, D = P.D;
+    const int n_slabs = (D + kSlabK - 1) / kSlabK;
+    const int per_cta = (prm.n_tiles + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int t_begin = (int)blockIdx.x * per_cta;
+    const int t_end = min(t_begin + per_cta, prm.n_tiles);
+
+    // ---- set-up: barriers, tensor memory, zeroed W operand (padding rows and features stay zero)
+    if (tid == 0) {
+        for (int h = 0; h < kHiStages; ++h) { mbar_init(bar(bar_full(h)), 1); mbar_init(bar(bar_hi_free(h)), 1); }
+        for (int l = 0; l < kLoStages; ++l) { mbar_init(bar(bar_lo_ready(l)), kConvThreads); mbar_init(bar(bar_lo_free(l)), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(bar(bar_acc_full(b)), 1); mbar_init(bar(bar_acc_empty(b)), kEpiThreads); }
+        mbar_init(bar(kBarWReady), kConvThreads);
+        mbar_init(bar(kBarDrain), 1);
+        mbar_init(bar(kBarEpiA), kEpiThreads);
+        mbar_init(bar(kBarEpiB), kEpiThreads);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int k = tid; k < kMaxSlabs * kSlabBytes / 16; k += kThreads)
+        reinterpret_cast<float4 *>(sm + Smem::w)[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (warp == kMmaWarp) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    fence_proxy_async();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == kProducerWarp) {
+        // ================================================================ TMA producer (one thread)
+        if (lane == 0) {
+            uint32_t slab_seq = 0;
+            bool ok = true;
+            for (int t = t_begin; t < t_end && ok; ++t) {
+                const int4 d = prm.tiles[t];
+                if (d.x < 0) continue;
+                const int row0 = (int)(tb.gstart[(int64_t)d.x * A] + d.y);
+                for (int s = 0; s < n_slabs; ++s, ++slab_seq) {
+                    const int h = slab_seq % kHiStages;
+                    const uint32_t use = slab_seq / kHiStages;
+                    if (use > 0 && !mbar_wait(bar(bar_hi_free(h)), (use - 1) & 1, abort_flag)) { ok = false; break; }
+                    mbar_arrive_expect_tx(bar(bar_full(h)), kSlabBytes);
+                    tma_load_2d(base + Smem::hi + h * kSlabBytes, &x_map, s * kSlabK, row0, bar(bar_full(h)));
+                }
+            }
+            if (!ok) {
+                // copies already issued still land in shared memory: give them a bounded time to finish
+                const uint32_t first = slab_seq > (uint32_t)kHiStages ? slab_seq - kHiStages : 0;
+                for (uint32_t q = first; q < slab_seq; ++q) {
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(bar(bar_full(q % kHiStages)), (q / kHiStages) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+                }
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        // ================================================================ MMA issuer (one thread)
+        if (lane == 0) {
+            constexpr uint32_t idesc_hi = instr_desc(2 * kCols), idesc_lo = instr_desc(kCols);
+            uint32_t slab_seq = 0, tile_seq = 0, w_seq = 0;
+            int cur_inst = -1;
+            bool ok = true;
+            for (int t = t_begin; t < t_end && ok; ++t) {
+                const int4 d = prm.tiles[t];
+                if (d.x < 0) continue;
+                if (d.x != cur_inst) {                         // operand of the new instance's heads
+                    if (!mbar_wait(bar(kBarWReady), w_seq & 1, abort_flag)) break;
+                    ++w_seq; cur_inst = d.x;
+                }
+                const int b = tile_seq & 1;
+                const uint32_t acc_use = tile_seq >> 1;
+                if (acc_use > 0 && !mbar_wait(bar(bar_acc_empty(b)), (acc_use - 1) & 1, abort_flag)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem + (uint32_t)(b * kAccCols);
+                for (int s = 0; s < n_slabs; ++s, ++slab_seq) {
+                    const int h = slab_seq % kHiStages, l = slab_seq % kLoStages;
+                    if (!mbar_wait(bar(bar_full(h)), (slab_seq / kHiStages) & 1, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_hi = base + Smem::hi + h * kSlabBytes, a_lo = base + Smem::lo + l * kSlabBytes;
+                    const uint32_t b_w = base + Smem::w + s * kSlabBytes;
+#pragma unroll
+                    for (int k = 0; k < kSlabK / 8; ++k)       // x_hi [W_hi | W_lo] -> all 128 columns
+                        umma_tf32(d_tmem, smem_desc(a_hi + k * 32), smem_desc(b_w + k * 32), idesc_hi, (s | k) != 0);
+                    if (!mbar_wait(bar(bar_lo_ready(l)), (slab_seq / kLoStages) & 1, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+#pragma unroll
+                    for (int k = 0; k < kSlabK / 8; ++k)       // x_lo W_hi -> the first 64 columns
+                        umma_tf32(d_tmem, smem_desc(a_lo + k * 32), smem_desc(b_w + k * 32), idesc_lo, 1u);
+                    umma_commit(bar(bar_hi_free(h)));
+                    umma_commit(bar(bar_lo_free(l)));
+                }
+                if (ok) umma_commit(bar(bar_acc_full(b)));
+                ++tile_seq;
+            }
+            if (*abort_flag) {                                 // leaving early: let the issued MMAs finish first
+                umma_commit(bar(kBarDrain));
+                const unsigned long long t0 = global_ns();
+                while (!mbar_try_wait(bar(kBarDrain), 0) && global_ns() - t0 < kWaitLimitNs) {}
+            }
+        }
+    } else if (warp < kEpiWarp0) {
+        // ================================================================ converter warps
+        const int ct = tid - kConvWarp0 * 32;                  // 0..127
+        uint32_t slab_seq = 0, tile_seq = 0;
+        int cur_inst = -1, pre_inst = -1;
+        // Head operand: this thread owns logit column wn (= operand row) and half of the feature chunks.
+        // Its raw weights W[a][d][c] are gathered into registers ahead of time (consecutive threads read
+        // consecutive labels, so the loads coalesce) and written as 16-byte pieces of the swizzled rows.
+        const int wn = ct & (kCols - 1), wq0 = (ct >> 6) * (kMaxD / 8);   // 16 chunks of 4 features per thread
+        const int wa = wn / C, wc = wn - wa * C;
+        const bool w_row = wn < A * C;
+        float wreg[kWRegs * 4];
+        auto fetch_w = [&](int inst) {
+            const float *src = (const float *)P.W + ((int64_t)inst * A + wa) * D * C + wc;
+#pragma unroll
+            for (int q = 0; q < kWRegs; ++q)
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int dd = (wq0 + q) * 4 + u;
+                    wreg[q * 4 + u] = (w_row && dd < D) ? src[(int64_t)dd * C] : 0.f;
+                }
+            pre_inst = inst;
+        };
+        bool ok = true;
+        for (int t = t_begin; t < t_end && ok; ++t) {
+            const int4 d = prm.tiles[t];
+            if (d.x < 0) continue;
+            if (d.x != cur_inst) {
+                if (pre_inst != d.x) fetch_w(d.x);
+                // every MMA that reads the previous operand belongs to the previous tile: wait for its accumulator
+                if (tile_seq > 0) {
+                    const uint32_t pt = tile_seq - 1;
+                    if (!warp_wait(bar(bar_acc_full(pt & 1)), (pt >> 1) & 1, abort_flag)) break;
+                }
+                if (w_row) {
+#pragma unroll
+                    for (int q = 0; q < kWRegs; ++q) {
+                        const int j = wq0 + q;                 // chunk of 4 features: slab j / 8, 16-byte piece j % 8
+                        if (j * 4 < D) {
+                            const uint32_t off = (uint32_t)((j >> 3) * kSlabBytes + wn * 128 + (((j & 7) ^ (wn & 7)) << 4));
+                            float4 hi, lo;
+                            hi.x = tf32_part(wreg[q * 4 + 0]); lo.x = wreg[q * 4 + 0] - hi.x;
+                            hi.y = tf32_part(wreg[q * 4 + 1]); lo.y = wreg[q * 4 + 1] - hi.y;
+                            hi.z = tf32_part(wreg[q * 4 + 2]); lo.z = wreg[q * 4 + 2] - hi.z;
+                            hi.w = tf32_part(wreg[q * 4 + 3]); lo.w = wreg[q * 4 + 3] - hi.w;
+                            *reinterpret_cast<float4 *>(sm + Smem::w + off) = hi;
+                            *reinterpret_cast<float4 *>(sm + Smem::w + off + kCols * 128) = lo;
+                        }
+                    }
+                }
+                fence_proxy_async();
+                mbar_arrive(bar(kBarWReady));
+                cur_inst = d.x;
+                if (d.x + 1 < P.I) fetch_w(d.x + 1);           // the next instance's heads, in flight while this one runs
+            }
+            for (int s = 0; s < n_slabs; ++s, ++slab_seq) {
+                const int h = slab_seq % kHiStages, l = slab_seq % kLoStages;
+                const uint32_t lo_use = slab_seq / kLoStages;
+                if (!warp_wait(bar(bar_full(h)), (slab_seq / kHiStages) & 1, abort_flag)) { ok = false; break; }
+                if (lo_use > 0 && !warp_wait(bar(bar_lo_free(l)), (lo_use - 1) & 1, abort_flag)) { ok = false; break; }
+                const float4 *src = reinterpret_cast<const float4 *>(sm + Smem::hi + h * kSlabBytes);
+                float4 *dst = reinterpret_cast<float4 *>(sm + Smem::lo + l * kSlabBytes);
+#pragma unroll
+                for (int q = 0; q < kSlabBytes / 16 / kConvThreads; ++q) {
+                    const float4 x = src[q * kConvThreads + ct];
+                    dst[q * kConvThreads + ct] = make_float4(x.x - tf32_part(x.x), x.y - tf32_part(x.y),
+                                                             x.z - tf32_part(x.z), x.w - tf32_part(x.w));
+                }
+                fence_proxy_async();
+                mbar_arrive(bar(bar_lo_ready(l)));
+            }
+            ++tile_seq;
+        }
+    } else {
+        // ================================================================ epilogue warps (one row per thread)
+        const int et = tid - kEpiWarp0 * 32;                   // 0..127
+        const int quad = warp & 3;                             // tensor-memory lanes this warp may read
+        const int row = quad * 32 + lane;
+        uint32_t tile_seq = 0, inst_seq = 0;
+        int cur_inst = -1;
+        const int sumM = P.sumM, Mmax = P.Mmax;
+        const bool vec4 = (C & 3) == 0;                        // label rows are 16-byte aligned in the tables
+        // application of this thread's row in tile t (loaded one tile ahead of its use)
+        auto load_app = [&](int t) -> int {
+            if (t >= t_end) return 0;
+            const int4 d = prm.tiles[t];
+            if (d.x < 0 || row >= d.z) return 0;
+            return tb.app[tb.gstart[(int64_t)d.x * A] + d.y + row];
+        };
+        int a_next = load_app(t_begin);
+        for (int t = t_begin; t < t_end; ++t) {
+            const int4 d = prm.tiles[t];
+            if (d.x < 0) continue;
+            const int inst = d.x;
+            const int a = min(max(a_next, 0), A - 1);
+            a_next = load_app(t + 1);
+            if (inst != cur_inst) {                            // this instance's bias, recall and prior terms
+                mbar_arrive(bar(kBarEpiA));
+                if (!warp_wait(bar(kBarEpiA), inst_seq & 1, abort_flag)) break;
+                for (int k = et; k < A * C; k += kEpiThreads) bias_s[k] = P.bias[(int64_t)inst * A * C + k];
+                for (int k = et; k < sumM * C; k += kEpiThreads) recall_s[k] = P.recall[(int64_t)inst * sumM * C + k];
+                if (P.prior) {
+                    for (int k = et; k < sumM; k += kEpiThreads) prior_s[k] = P.prior_dot[(int64_t)inst * sumM + k];
+                    for (int k = et; k < A; k += kEpiThreads) prior_s[256 + k] = P.prior_sum[inst * A + k];
+                }
+                mbar_arrive(bar(kBarEpiB));
+                if (!warp_wait(bar(kBarEpiB), inst_seq & 1, abort_flag)) break;
+                ++inst_seq;
+                cur_inst = inst;
+            }
+            const int64_t req = tb.gstart[(int64_t)inst * A] + d.y + row;
+            const bool valid = row < d.z;
+            const int b = tile_seq & 1;
+            if (!warp_wait(bar(bar_acc_full(b)), (tile_seq >> 1) & 1, abort_flag)) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * kAccCols);
+            float z[CT];
+#pragma unroll
+            for (int c = 0; c < CT; ++c) z[c] = 0.f;
+            for (int ap = 0; ap < A; ++ap) {
+                if (__ballot_sync(0xffffffffu, a == ap) == 0) continue;
+                float r1[CT], r2[CT];
+                tmem_ld<CT>(taddr + (uint32_t)(ap * C), r1);
+                tmem_ld<CT>(taddr + (uint32_t)(kCols + ap * C), r2);
+                tmem_wait_ld();
+                if (a == ap) {
+#pragma unroll
+                    for (int c = 0; c < CT; ++c) z[c] = r1[c] + r2[c];
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(bar(bar_acc_empty(b)));
+            ++tile_seq;
+
+            // ---- softmax over the C labels of this row's application
+            const float *bs = bias_s + a * C;
+            if (vec4) {
+#pragma unroll
+                for (int c = 0; c < CT; c += 4)
+                    if (c < C) {
+                        const float4 bv = *reinterpret_cast<const float4 *>(bs + c);
+                        z[c] += bv.x; z[c + 1] += bv.y; z[c + 2] += bv.z; z[c + 3] += bv.w;
+                    }
+            } else {
+#pragma unroll
+                for (int c = 0; c < CT; ++c)
+                    if (c < C) z[c] += bs[c];
+            }
+            float m = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < CT; ++c)
+                if (c < C) m = fmaxf(m, z[c]);
+            float ssum = 0.f;
+#pragma unroll
+            for (int c = 0; c < CT; ++c) { z[c] = c < C ? exp_neg(z[c] - m) : 0.f; ssum += z[c]; }
+            const float inv = 1.f / ssum;
+            // ---- Eq. 9 with the Dirichlet posterior mean, Eq. 12's variance factor
+            const int g0 = P.mfirst[a], M = P.mfirst[a + 1] - g0;
+            float accv[kMaxModelsPerApp], mean = 0.f;
+#pragma unroll
+            for (int j = 0; j < kMaxModelsPerApp; ++j) {
+                accv[j] = 0.f;
+                if (j < Mmax) {
+                    if (j < M) {
+                        const float *rr = recall_s + (g0 + j) * C;
+                        float part = 0.f;
+                        if (vec4) {
+#pragma unroll
+                            for (int c = 0; c < CT; c += 4)
+                                if (c < C) {
+                                    const float4 rv = *reinterpret_cast<const float4 *>(rr + c);
+                                    part = fmaf(z[c], rv.x, part); part = fmaf(z[c + 1], rv.y, part);
+                                    part = fmaf(z[c + 2], rv.z, part); part = fmaf(z[c + 3], rv.w, part);
+                                }
+                        } else {
+#pragma unroll
+                            for (int c = 0; c < CT; ++c)
+                                if (c < C) part = fmaf(z[c], rr[c], part);
+                        }
+                        float aj = part * inv;
+                        if (P.prior) aj = (prior_s[g0 + j] + P.kappa * aj) / (prior_s[256 + a] + P.kappa);
+                        accv[j] = aj;
+                        mean += aj;
+                    }
+                }
+            }
+            mean /= (float)M;
+            float var = 0.f;
+#pragma unroll
+            for (int j = 0; j < kMaxModelsPerApp; ++j)
+                if (j < M) var = fmaf(accv[j] - mean, accv[j] - mean, var);
+            if (valid) {
+                float *dst = tb.acc32 + req * Mmax;
+#pragma unroll
+                for (int j = 0; j < kMaxModelsPerApp; ++j)
+                    if (j < Mmax) dst[j] = accv[j];
+                tb.v32[req] = 1.f + var / (float)M;
+                if (prm.acc_out) {
+                    float *o = prm.acc_out + req * Mmax;
+#pragma unroll
+                    for (int j = 0; j < kMaxModelsPerApp; ++j)
+                        if (j < Mmax) o[j] = accv[j];
+                }
+            }
+        }
+    }
+
+    // ---- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0 && *abort_flag) dev_error(&prm.flags[0], kDevLimit);
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+}  // namespace mma
+}  // namespace sp
