@@ -369,8 +369,8 @@ sp_status sp_load_profiles(sp_ctx *c, const sp_profiles *p) {
     c->sched_threads = I > 1 ? 128 : 1024;
     c->small_ct = 0;
     c->mma_ct = 0;
-    if (p->feat_dtype == SP_F32 && D % 4 == 0 && D <= mma::kMaxD && A * C <= mma::kCols && sumM * C <= 1024) {
-        c->mma_ct = C <= 16 ? 16 : C <= 32 ? 32 : 64;
+    if (p->feat_dtype == SP_F32 && D % 4 == 0 && D <= mma::kMaxD && A * C <= mma::kCols && sumM * ((C + 3) & ~3) <= 1024) {
+        c->mma_ct = C <= 8 ? 8 : C <= 16 ? 16 : C <= 24 ? 24 : C <= 32 ? 32 : C <= 48 ? 48 : 64;
     } else if (p->feat_dtype == SP_F32 && D % 4 == 0 && C <= 64) {
         const int ct = small_ct_for(C);
         const SmallSmem L(A, D, sumM, (ct + 3) & ~3);
@@ -505,8 +505,11 @@ sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, 
         if (c->mma_ct) {
             mma::Params prm{P, tb, (const int4 *)c->small_tiles.p, grid, acc_out, (int *)c->flags.p};
             switch (c->mma_ct) {
+                case 8: SP_TRY(launch_mma<8>(c, x_map, prm)); break;
                 case 16: SP_TRY(launch_mma<16>(c, x_map, prm)); break;
+                case 24: SP_TRY(launch_mma<24>(c, x_map, prm)); break;
                 case 32: SP_TRY(launch_mma<32>(c, x_map, prm)); break;
+                case 48: SP_TRY(launch_mma<48>(c, x_map, prm)); break;
                 default: SP_TRY(launch_mma<64>(c, x_map, prm)); break;
             }
         } else if (c->small_ct) {

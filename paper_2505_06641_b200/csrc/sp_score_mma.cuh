@@ -39,8 +39,10 @@ constexpr int kLoStages = 3;               // ring of slabs written by the conve
 constexpr int kTmemCols = 512;             // whole tensor memory: 2 accumulators of 128 columns, reads may overhang
 constexpr int kAccCols = 128;              // columns per accumulator: [x_hi W_hi + x_lo W_hi | x_hi W_lo]
 constexpr int kProducerWarp = 0, kMmaWarp = 1, kConvWarp0 = 2, kEpiWarp0 = 6;
-constexpr int kThreads = 32 * 10;
+constexpr int kEpiGroups = 2;              // epilogue warpgroups; group g takes every second tile and accumulator g
+constexpr int kThreads = 32 * (6 + 4 * kEpiGroups);
 constexpr int kConvThreads = 128, kEpiThreads = 128;
+constexpr float kLog2e = 1.44269502162933349609375f;   // folded into W and the bias: the softmax runs in base 2
 constexpr int kWRegs = (kCols * kMaxD / 4) / kConvThreads;   // float4 registers per converter thread holding a raw head
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
 
@@ -48,11 +50,13 @@ struct Smem {                               // byte offsets from the 1024-byte a
     static constexpr int w = 0;                                        // kMaxSlabs slabs: rows 0..63 W_hi, 64..127 W_lo
     static constexpr int hi = w + kMaxSlabs * kSlabBytes;
     static constexpr int lo = hi + kHiStages * kSlabBytes;
-    static constexpr int recall = lo + kLoStages * kSlabBytes;         // [sumM][C] floats, at most 1024
-    static constexpr int bias = recall + 1024 * 4;                     // [A*C] floats
-    static constexpr int prior = bias + kCols * 4;                     // prior_dot [sumM] (<= 256), prior_sum [A] (<= 16)
-    static constexpr int bars = prior + (256 + 16) * 4;
-    static constexpr int n_bars = 2 * kHiStages + 2 * kLoStages + 8;
+    // per-instance tables, one copy per epilogue group, label rows padded with zeros to a multiple of 4 floats (Cp):
+    // recall [sumM][Cp] (<= 1024 floats), bias * log2(e) [A][Cp] (<= 128), prior_dot [sumM] (<= 256), prior_sum [A] (<= 16)
+    static constexpr int tab_recall = 0, tab_bias = 1024, tab_pdot = tab_bias + 2 * kCols, tab_psum = tab_pdot + 256;
+    static constexpr int tab_floats = tab_psum + 16;
+    static constexpr int tabs = lo + kLoStages * kSlabBytes;
+    static constexpr int bars = tabs + kEpiGroups * tab_floats * 4;
+    static constexpr int n_bars = 2 * kHiStages + 2 * kLoStages + 6 + 2 * kEpiGroups;
     static constexpr int misc = bars + n_bars * 8;                     // tmem base, abort flag
     static constexpr int end = misc + 16;
     static constexpr int bytes = end + 1024;                           // slack for the manual alignment
@@ -62,7 +66,7 @@ struct Params {
     DevProfiles P;
     DevTable tb;
     const int4 *tiles;       // (instance, first request relative to the instance, rows, -)
-    int n_tiles;             // entries in `tiles` (those past the end have instance -1)
+    int n_tiles;             // entries in `tiles`; the valid ones come first, those past the end have instance -1
     float *acc_out;          // optional second destination of acc
     int *flags;
 };
@@ -95,8 +99,8 @@ __device__ __forceinline__ unsigned long long global_ns() {
     return t;
 }
 // Bounded wait: false when the wait ran out (the block-wide abort flag is then set) or another thread gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
+// The polling loop is kept out of line: it is entered only when the barrier is not ready yet.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
     const unsigned long long t0 = global_ns();
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
@@ -106,6 +110,10 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             __nanosleep(64);
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag);
 }
 
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -176,6 +184,36 @@ __device__ __forceinline__ void tmem_ld<32>(uint32_t taddr, float (&r)[32]) {
     for (int i = 0; i < 32; ++i) r[i] = __uint_as_float(v[i]);
 }
 template <>
+__device__ __forceinline__ void tmem_ld<8>(uint32_t taddr, float (&r)[8]) {
+    uint32_t v[8];
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                 : "r"(taddr)
+                 : "memory");
+#pragma unroll
+    for (int i = 0; i < 8; ++i) r[i] = __uint_as_float(v[i]);
+}
+template <>
+__device__ __forceinline__ void tmem_ld<24>(uint32_t taddr, float (&r)[24]) {
+    float a[16], b[8];
+    tmem_ld<16>(taddr, a);
+    tmem_ld<8>(taddr + 16, b);
+#pragma unroll
+    for (int i = 0; i < 16; ++i) r[i] = a[i];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) r[16 + i] = b[i];
+}
+template <>
+__device__ __forceinline__ void tmem_ld<48>(uint32_t taddr, float (&r)[48]) {
+    float a[32], b[16];
+    tmem_ld<32>(taddr, a);
+    tmem_ld<16>(taddr + 32, b);
+#pragma unroll
+    for (int i = 0; i < 32; ++i) r[i] = a[i];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) r[32 + i] = b[i];
+}
+template <>
 __device__ __forceinline__ void tmem_ld<64>(uint32_t taddr, float (&r)[64]) {
     float a[32], b[32];
     tmem_ld<32>(taddr, a);
@@ -188,17 +226,11 @@ __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.
 // Value a tf32 operand takes from a 32-bit container: the low 13 mantissa bits are not read.
 __device__ __forceinline__ float tf32_part(float x) { return __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
 
-// exp(x) for x <= 0 from the ex2 unit: x * log2(e) is split into a rounded product and its exact residual
-// (plus the low part of log2(e)), and the residual is applied as a first-order correction, so the result
-// carries the unit's own error (about 2^-22 relative) instead of |x| * 2^-24 from the argument.
-__device__ __forceinline__ float exp_neg(float x) {
-    const float kL2eHi = 1.44269502162933349609375f, kL2eLo = 1.925963033500305e-08f;
-    x = fmaxf(x, -120.f);                       // exp(-120) flushes to zero; keeps -inf (padded labels) finite
-    const float r = x * kL2eHi;
-    const float e = fmaf(x, kL2eLo, fmaf(x, kL2eHi, -r));
+// 2^x from the ex2 unit (about 2^-22 relative error; 2^-inf = 0).
+__device__ __forceinline__ float exp2_unit(float x) {
     float p;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(p) : "f"(r));
-    return fmaf(p * e, 0.693147182464599609375f, p);
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(p) : "f"(x));
+    return p;
 }
 
 // Barrier indices
@@ -210,8 +242,9 @@ __device__ __forceinline__ constexpr int bar_acc_full(int b) { return 2 * kHiSta
 __device__ __forceinline__ constexpr int bar_acc_empty(int b) { return 2 * kHiStages + 2 * kLoStages + 2 + b; }
 constexpr int kBarWReady = 2 * kHiStages + 2 * kLoStages + 4;
 constexpr int kBarDrain = 2 * kHiStages + 2 * kLoStages + 5;
-constexpr int kBarEpiA = 2 * kHiStages + 2 * kLoStages + 6;   // epilogue threads: done reading the old tables
-constexpr int kBarEpiB = 2 * kHiStages + 2 * kLoStages + 7;   // epilogue threads: new tables written
+// per epilogue group: A = every thread is done reading the old tables, B = the new tables are written
+__device__ __forceinline__ constexpr int bar_epi_a(int g) { return 2 * kHiStages + 2 * kLoStages + 6 + g; }
+__device__ __forceinline__ constexpr int bar_epi_b(int g) { return 2 * kHiStages + 2 * kLoStages + 6 + kEpiGroups + g; }
 
 // Warp-uniform outcome of a bounded wait done by every lane.
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
@@ -227,9 +260,6 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
     const uint32_t raw_u32 = smem_u32(smem_raw);
     const uint32_t base = (raw_u32 + 1023u) & ~1023u;
     unsigned char *sm = smem_raw + (base - raw_u32);
-    float *recall_s = reinterpret_cast<float *>(sm + Smem::recall);
-    float *bias_s = reinterpret_cast<float *>(sm + Smem::bias);
-    float *prior_s = reinterpret_cast<float *>(sm + Smem::prior);
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(sm + Smem::misc);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(sm + Smem::misc + 4);
     auto bar = [&](int i) -> uint32_t { return base + Smem::bars + 8u * (uint32_t)i; };
@@ -250,13 +280,14 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
         for (int b = 0; b < 2; ++b) { mbar_init(bar(bar_acc_full(b)), 1); mbar_init(bar(bar_acc_empty(b)), kEpiThreads); }
         mbar_init(bar(kBarWReady), kConvThreads);
         mbar_init(bar(kBarDrain), 1);
-        mbar_init(bar(kBarEpiA), kEpiThreads);
-        mbar_init(bar(kBarEpiB), kEpiThreads);
+        for (int g = 0; g < kEpiGroups; ++g) { mbar_init(bar(bar_epi_a(g)), kEpiThreads); mbar_init(bar(bar_epi_b(g)), kEpiThreads); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     for (int k = tid; k < kMaxSlabs * kSlabBytes / 16; k += kThreads)
         reinterpret_cast<float4 *>(sm + Smem::w)[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int k = tid; k < kEpiGroups * Smem::tab_floats; k += kThreads)      // the padding of the label rows stays zero
+        reinterpret_cast<float *>(sm + Smem::tabs)[k] = 0.f;
     if (warp == kMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -274,7 +305,7 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
             bool ok = true;
             for (int t = t_begin; t < t_end && ok; ++t) {
                 const int4 d = prm.tiles[t];
-                if (d.x < 0) continue;
+                if (d.x < 0) break;                            // valid tiles form a prefix of the block's range
                 const int row0 = (int)(tb.gstart[(int64_t)d.x * A] + d.y);
                 for (int s = 0; s < n_slabs; ++s, ++slab_seq) {
                     const int h = slab_seq % kHiStages;
@@ -302,7 +333,7 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
             bool ok = true;
             for (int t = t_begin; t < t_end && ok; ++t) {
                 const int4 d = prm.tiles[t];
-                if (d.x < 0) continue;
+                if (d.x < 0) break;                            // valid tiles form a prefix of the block's range
                 if (d.x != cur_inst) {                         // operand of the new instance's heads
                     if (!mbar_wait(bar(kBarWReady), w_seq & 1, abort_flag)) break;
                     ++w_seq; cur_inst = d.x;
@@ -364,7 +395,7 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
         bool ok = true;
         for (int t = t_begin; t < t_end && ok; ++t) {
             const int4 d = prm.tiles[t];
-            if (d.x < 0) continue;
+            if (d.x < 0) break;                            // valid tiles form a prefix of the block's range
             if (d.x != cur_inst) {
                 if (pre_inst != d.x) fetch_w(d.x);
                 // every MMA that reads the previous operand belongs to the previous tile: wait for its accumulator
@@ -378,11 +409,13 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
                         const int j = wq0 + q;                 // chunk of 4 features: slab j / 8, 16-byte piece j % 8
                         if (j * 4 < D) {
                             const uint32_t off = (uint32_t)((j >> 3) * kSlabBytes + wn * 128 + (((j & 7) ^ (wn & 7)) << 4));
+                            const float w0 = wreg[q * 4 + 0] * kLog2e, w1 = wreg[q * 4 + 1] * kLog2e;
+                            const float w2 = wreg[q * 4 + 2] * kLog2e, w3 = wreg[q * 4 + 3] * kLog2e;
                             float4 hi, lo;
-                            hi.x = tf32_part(wreg[q * 4 + 0]); lo.x = wreg[q * 4 + 0] - hi.x;
-                            hi.y = tf32_part(wreg[q * 4 + 1]); lo.y = wreg[q * 4 + 1] - hi.y;
-                            hi.z = tf32_part(wreg[q * 4 + 2]); lo.z = wreg[q * 4 + 2] - hi.z;
-                            hi.w = tf32_part(wreg[q * 4 + 3]); lo.w = wreg[q * 4 + 3] - hi.w;
+                            hi.x = tf32_part(w0); lo.x = w0 - hi.x;
+                            hi.y = tf32_part(w1); lo.y = w1 - hi.y;
+                            hi.z = tf32_part(w2); lo.z = w2 - hi.z;
+                            hi.w = tf32_part(w3); lo.w = w3 - hi.w;
                             *reinterpret_cast<float4 *>(sm + Smem::w + off) = hi;
                             *reinterpret_cast<float4 *>(sm + Smem::w + off + kCols * 128) = lo;
                         }
@@ -413,47 +446,81 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
         }
     } else {
         // ================================================================ epilogue warps (one row per thread)
-        const int et = tid - kEpiWarp0 * 32;                   // 0..127
+        const int eg = (warp - kEpiWarp0) >> 2;                // group: tiles eg, eg + 2, ... and accumulator eg
+        const int et = (tid - kEpiWarp0 * 32) & (kEpiThreads - 1);
         const int quad = warp & 3;                             // tensor-memory lanes this warp may read
         const int row = quad * 32 + lane;
-        uint32_t tile_seq = 0, inst_seq = 0;
-        int cur_inst = -1;
+        float *tab = reinterpret_cast<float *>(sm + Smem::tabs) + eg * Smem::tab_floats;
+        const float *recall_s = tab + Smem::tab_recall, *bias_s = tab + Smem::tab_bias;
+        const float *pdot_s = tab + Smem::tab_pdot, *psum_s = tab + Smem::tab_psum;
+        uint32_t inst_seq = 0;
+        int cur_inst = -1, pre_inst = -1;
         const int sumM = P.sumM, Mmax = P.Mmax;
-        const bool vec4 = (C & 3) == 0;                        // label rows are 16-byte aligned in the tables
-        // application of this thread's row in tile t (loaded one tile ahead of its use)
+        const int Cp = (C + 3) & ~3;                           // label stride of the tables in shared memory
+        // this instance's tables travel through registers so that the loads of the next instance are in flight
+        // while the current one is processed
+        float pre_rec[1024 / kEpiThreads], pre_bias = 0.f, pre_pdot[256 / kEpiThreads], pre_psum = 0.f;
+        auto fetch_tab = [&](int inst) {
+#pragma unroll
+            for (int q = 0; q < 1024 / kEpiThreads; ++q) {
+                const int k = q * kEpiThreads + et;
+                pre_rec[q] = k < sumM * C ? P.recall[(int64_t)inst * sumM * C + k] : 0.f;
+            }
+            pre_bias = et < A * C ? P.bias[(int64_t)inst * A * C + et] : 0.f;
+            if (P.prior) {
+#pragma unroll
+                for (int q = 0; q < 256 / kEpiThreads; ++q) {
+                    const int k = q * kEpiThreads + et;
+                    pre_pdot[q] = k < sumM ? P.prior_dot[(int64_t)inst * sumM + k] : 0.f;
+                }
+                pre_psum = et < A ? P.prior_sum[inst * A + et] : 0.f;
+            }
+            pre_inst = inst;
+        };
+        // application of this thread's row in tile t (loaded one of the group's tiles ahead of its use)
         auto load_app = [&](int t) -> int {
             if (t >= t_end) return 0;
             const int4 d = prm.tiles[t];
             if (d.x < 0 || row >= d.z) return 0;
             return tb.app[tb.gstart[(int64_t)d.x * A] + d.y + row];
         };
-        int a_next = load_app(t_begin);
-        for (int t = t_begin; t < t_end; ++t) {
+        int a_next = load_app(t_begin + eg);
+        for (int t = t_begin + eg; t < t_end; t += kEpiGroups) {
             const int4 d = prm.tiles[t];
-            if (d.x < 0) continue;
+            if (d.x < 0) break;                                // valid tiles form a prefix of the block's range
             const int inst = d.x;
             const int a = min(max(a_next, 0), A - 1);
-            a_next = load_app(t + 1);
-            if (inst != cur_inst) {                            // this instance's bias, recall and prior terms
-                mbar_arrive(bar(kBarEpiA));
-                if (!warp_wait(bar(kBarEpiA), inst_seq & 1, abort_flag)) break;
-                for (int k = et; k < A * C; k += kEpiThreads) bias_s[k] = P.bias[(int64_t)inst * A * C + k];
-                for (int k = et; k < sumM * C; k += kEpiThreads) recall_s[k] = P.recall[(int64_t)inst * sumM * C + k];
-                if (P.prior) {
-                    for (int k = et; k < sumM; k += kEpiThreads) prior_s[k] = P.prior_dot[(int64_t)inst * sumM + k];
-                    for (int k = et; k < A; k += kEpiThreads) prior_s[256 + k] = P.prior_sum[inst * A + k];
+            a_next = load_app(t + kEpiGroups);
+            if (inst != cur_inst) {
+                if (pre_inst != inst) fetch_tab(inst);
+                mbar_arrive(bar(bar_epi_a(eg)));
+                if (!warp_wait(bar(bar_epi_a(eg)), inst_seq & 1, abort_flag)) break;
+#pragma unroll
+                for (int q = 0; q < 1024 / kEpiThreads; ++q) {
+                    const int k = q * kEpiThreads + et;
+                    if (k < sumM * C) { const int g = k / C; tab[Smem::tab_recall + g * Cp + (k - g * C)] = pre_rec[q]; }
                 }
-                mbar_arrive(bar(kBarEpiB));
-                if (!warp_wait(bar(kBarEpiB), inst_seq & 1, abort_flag)) break;
+                if (et < A * C) { const int g = et / C; tab[Smem::tab_bias + g * Cp + (et - g * C)] = pre_bias * kLog2e; }
+                if (P.prior) {
+#pragma unroll
+                    for (int q = 0; q < 256 / kEpiThreads; ++q) {
+                        const int k = q * kEpiThreads + et;
+                        if (k < sumM) tab[Smem::tab_pdot + k] = pre_pdot[q];
+                    }
+                    if (et < A) tab[Smem::tab_psum + et] = pre_psum;
+                }
+                mbar_arrive(bar(bar_epi_b(eg)));
+                if (!warp_wait(bar(bar_epi_b(eg)), inst_seq & 1, abort_flag)) break;
                 ++inst_seq;
                 cur_inst = inst;
+                if (inst + 1 < P.I) fetch_tab(inst + 1);
             }
             const int64_t req = tb.gstart[(int64_t)inst * A] + d.y + row;
             const bool valid = row < d.z;
-            const int b = tile_seq & 1;
-            if (!warp_wait(bar(bar_acc_full(b)), (tile_seq >> 1) & 1, abort_flag)) break;
+            const uint32_t acc_use = (uint32_t)(t - t_begin) >> 1;      // earlier uses of accumulator eg
+            if (!warp_wait(bar(bar_acc_full(eg)), acc_use & 1, abort_flag)) break;
             tc_fence_after();
-            const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * kAccCols);
+            const uint32_t taddr = tmem + ((uint32_t)(quad * 32) << 16) + (uint32_t)(eg * kAccCols);
             float z[CT];
 #pragma unroll
             for (int c = 0; c < CT; ++c) z[c] = 0.f;
@@ -469,78 +536,56 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
                 }
             }
             tc_fence_before();
-            mbar_arrive(bar(bar_acc_empty(b)));
-            ++tile_seq;
+            mbar_arrive(bar(bar_acc_empty(eg)));
 
-            // ---- softmax over the C labels of this row's application
-            const float *bs = bias_s + a * C;
-            if (vec4) {
+            // ---- softmax over the C labels of this row's application (base 2: log2(e) is in W and the bias)
+            const float *bs = bias_s + a * Cp;
 #pragma unroll
-                for (int c = 0; c < CT; c += 4)
-                    if (c < C) {
-                        const float4 bv = *reinterpret_cast<const float4 *>(bs + c);
-                        z[c] += bv.x; z[c + 1] += bv.y; z[c + 2] += bv.z; z[c + 3] += bv.w;
-                    }
-            } else {
-#pragma unroll
-                for (int c = 0; c < CT; ++c)
-                    if (c < C) z[c] += bs[c];
-            }
+            for (int c = 0; c < CT; c += 4)
+                if (c < C) {
+                    const float4 bv = *reinterpret_cast<const float4 *>(bs + c);
+                    z[c] += bv.x; z[c + 1] += bv.y; z[c + 2] += bv.z; z[c + 3] += bv.w;
+                }
             float m = -INFINITY;
 #pragma unroll
             for (int c = 0; c < CT; ++c)
                 if (c < C) m = fmaxf(m, z[c]);
             float ssum = 0.f;
 #pragma unroll
-            for (int c = 0; c < CT; ++c) { z[c] = c < C ? exp_neg(z[c] - m) : 0.f; ssum += z[c]; }
+            for (int c = 0; c < CT; ++c) { z[c] = c < C ? exp2_unit(z[c] - m) : 0.f; ssum += z[c]; }
             const float inv = 1.f / ssum;
-            // ---- Eq. 9 with the Dirichlet posterior mean, Eq. 12's variance factor
+            // ---- Eq. 9 with the Dirichlet posterior mean; Eq. 12's variance from sums of differences to acc_0
             const int g0 = P.mfirst[a], M = P.mfirst[a + 1] - g0;
-            float accv[kMaxModelsPerApp], mean = 0.f;
+            float *dst = tb.acc32 + req * Mmax;
+            float *dst2 = prm.acc_out ? prm.acc_out + req * Mmax : nullptr;
+            float a0 = 0.f, s1 = 0.f, s2 = 0.f;
+#pragma unroll 1
+            for (int j = 0; j < Mmax; ++j) {
+                float aj = 0.f;
+                if (j < M) {
+                    const float *rr = recall_s + (g0 + j) * Cp;
+                    float p0 = 0.f, p1 = 0.f;
 #pragma unroll
-            for (int j = 0; j < kMaxModelsPerApp; ++j) {
-                accv[j] = 0.f;
-                if (j < Mmax) {
-                    if (j < M) {
-                        const float *rr = recall_s + (g0 + j) * C;
-                        float part = 0.f;
-                        if (vec4) {
-#pragma unroll
-                            for (int c = 0; c < CT; c += 4)
-                                if (c < C) {
-                                    const float4 rv = *reinterpret_cast<const float4 *>(rr + c);
-                                    part = fmaf(z[c], rv.x, part); part = fmaf(z[c + 1], rv.y, part);
-                                    part = fmaf(z[c + 2], rv.z, part); part = fmaf(z[c + 3], rv.w, part);
-                                }
-                        } else {
-#pragma unroll
-                            for (int c = 0; c < CT; ++c)
-                                if (c < C) part = fmaf(z[c], rr[c], part);
+                    for (int c = 0; c < CT; c += 4)
+                        if (c < C) {
+                            const float4 rv = *reinterpret_cast<const float4 *>(rr + c);
+                            p0 = fmaf(z[c], rv.x, p0); p1 = fmaf(z[c + 1], rv.y, p1);
+                            p0 = fmaf(z[c + 2], rv.z, p0); p1 = fmaf(z[c + 3], rv.w, p1);
                         }
-                        float aj = part * inv;
-                        if (P.prior) aj = (prior_s[g0 + j] + P.kappa * aj) / (prior_s[256 + a] + P.kappa);
-                        accv[j] = aj;
-                        mean += aj;
-                    }
+                    aj = (p0 + p1) * inv;
+                    if (P.prior) aj = (pdot_s[g0 + j] + P.kappa * aj) / (psum_s[a] + P.kappa);
+                    if (j == 0) a0 = aj;
+                    const float dj = aj - a0;
+                    s1 += dj; s2 = fmaf(dj, dj, s2);
+                }
+                if (valid) {
+                    dst[j] = aj;
+                    if (dst2) dst2[j] = aj;
                 }
             }
-            mean /= (float)M;
-            float var = 0.f;
-#pragma unroll
-            for (int j = 0; j < kMaxModelsPerApp; ++j)
-                if (j < M) var = fmaf(accv[j] - mean, accv[j] - mean, var);
             if (valid) {
-                float *dst = tb.acc32 + req * Mmax;
-#pragma unroll
-                for (int j = 0; j < kMaxModelsPerApp; ++j)
-                    if (j < Mmax) dst[j] = accv[j];
-                tb.v32[req] = 1.f + var / (float)M;
-                if (prm.acc_out) {
-                    float *o = prm.acc_out + req * Mmax;
-#pragma unroll
-                    for (int j = 0; j < kMaxModelsPerApp; ++j)
-                        if (j < Mmax) o[j] = accv[j];
-                }
+                const float invM = 1.f / (float)M, md = s1 * invM;
+                tb.v32[req] = 1.f + fmaxf(fmaf(s2, invM, -md * md), 0.f);
             }
         }
     }
