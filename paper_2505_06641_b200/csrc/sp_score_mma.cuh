@@ -13,8 +13,12 @@
 //   * fp32 accuracy from the tf32 unit: x = x_hi + x_lo and W = W_hi + W_lo with x_hi, W_hi the values
 //     truncated to tf32 (what the unit reads from a 32-bit container) and the remainders exact in fp32;
 //     z = x_hi [W_hi | W_lo] + x_lo W_hi accumulates in fp32 in tensor memory, the dropped x_lo W_lo term
-//     is below 2^-20 relative.  x_hi needs no conversion (it is the tile as loaded); converter warps
-//     write x_lo into a second ring of slabs and rebuild the W operand when the instance changes;
+//     is below 2^-20 relative;
+//   * shared-memory bandwidth is the scarce resource (every MMA re-reads its operands), so the A operand
+//     comes from tensor memory: converter warps (one row per thread) read each slab once, store the row as
+//     loaded (read as x_hi) and its remainder x_lo into a ring of tensor-memory columns, and the MMAs read
+//     only the small W operand from shared memory.  The converters also rebuild the W operand when the
+//     instance changes;
 //   * epilogue warps read the accumulator from tensor memory (one row per thread), add the bias, and do
 //     softmax, the recall contraction, the Dirichlet step and the variance in registers.
 // Every wait on an mbarrier is bounded; when a wait runs out the block raises kDevLimit and leaves.
@@ -34,29 +38,31 @@ constexpr int kSlabBytes = kRows * 128;    // 16 KB: 128 rows x 128 bytes
 constexpr int kMaxD = 128;
 constexpr int kMaxSlabs = kMaxD / kSlabK;
 constexpr int kCols = 64;                  // logit columns (sum over applications of the label count)
-constexpr int kHiStages = 6;               // ring of slabs filled by TMA (x, read as x_hi)
-constexpr int kLoStages = 3;               // ring of slabs written by the converter warps (x_lo)
-constexpr int kTmemCols = 512;             // whole tensor memory: 2 accumulators of 128 columns, reads may overhang
+constexpr int kXStages = 6;                // ring of slabs in shared memory filled by TMA
+constexpr int kASlots = 4;                 // ring of A operands in tensor memory: 32 columns x_hi + 32 columns x_lo each
+constexpr int kTmemCols = 512;             // whole tensor memory
 constexpr int kAccCols = 128;              // columns per accumulator: [x_hi W_hi + x_lo W_hi | x_hi W_lo]
+constexpr int kTmemA = 2 * kAccCols;       // accumulators first (epilogue reads may overhang into the A ring), then the ring
+constexpr int kSlotCols = 2 * kSlabK;
 constexpr int kProducerWarp = 0, kMmaWarp = 1, kConvWarp0 = 2, kEpiWarp0 = 6;
 constexpr int kEpiGroups = 2;              // epilogue warpgroups; group g takes every second tile and accumulator g
 constexpr int kThreads = 32 * (6 + 4 * kEpiGroups);
 constexpr int kConvThreads = 128, kEpiThreads = 128;
 constexpr float kLog2e = 1.44269502162933349609375f;   // folded into W and the bias: the softmax runs in base 2
-constexpr int kWRegs = (kCols * kMaxD / 4) / kConvThreads;   // float4 registers per converter thread holding a raw head
+constexpr int kWChunks = (kCols * kMaxD / 4) / kConvThreads;  // 4-feature pieces of the head operand per converter thread
 constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
 
 struct Smem {                               // byte offsets from the 1024-byte aligned base
     static constexpr int w = 0;                                        // kMaxSlabs slabs: rows 0..63 W_hi, 64..127 W_lo
-    static constexpr int hi = w + kMaxSlabs * kSlabBytes;
-    static constexpr int lo = hi + kHiStages * kSlabBytes;
+    static constexpr int wraw = w + kMaxSlabs * kSlabBytes;            // the next instance's heads as stored: W[a][d][c] fp32
+    static constexpr int x = wraw + kCols * kMaxD * 4;
     // per-instance tables, one copy per epilogue group, label rows padded with zeros to a multiple of 4 floats (Cp):
     // recall [sumM][Cp] (<= 1024 floats), bias * log2(e) [A][Cp] (<= 128), prior_dot [sumM] (<= 256), prior_sum [A] (<= 16)
     static constexpr int tab_recall = 0, tab_bias = 1024, tab_pdot = tab_bias + 2 * kCols, tab_psum = tab_pdot + 256;
     static constexpr int tab_floats = tab_psum + 16;
-    static constexpr int tabs = lo + kLoStages * kSlabBytes;
+    static constexpr int tabs = x + kXStages * kSlabBytes;
     static constexpr int bars = tabs + kEpiGroups * tab_floats * 4;
-    static constexpr int n_bars = 2 * kHiStages + 2 * kLoStages + 6 + 2 * kEpiGroups;
+    static constexpr int n_bars = 2 * kXStages + 2 * kASlots + 8 + 2 * kEpiGroups;
     static constexpr int misc = bars + n_bars * 8;                     // tmem base, abort flag
     static constexpr int end = misc + 16;
     static constexpr int bytes = end + 1024;                           // slack for the manual alignment
@@ -128,6 +134,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
         : "memory");
 }
 
+// Plain bulk copy global -> shared memory (no multicast); both addresses and the size are multiples of 16 bytes.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
     uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
@@ -147,6 +160,15 @@ __device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint
         "setp.ne.b32 p, %4, 0;\n"
         "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+// Same with the A operand in tensor memory (128 lanes x 8 columns of 32-bit containers per instruction).
+__device__ __forceinline__ void umma_tf32_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], [%1], %2, %3, p;\n}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(acc)
         : "memory");
 }
 // Arrives on the mbarrier once every MMA issued so far by this thread has completed.
@@ -221,6 +243,18 @@ __device__ __forceinline__ void tmem_ld<64>(uint32_t taddr, float (&r)[64]) {
 #pragma unroll
     for (int i = 0; i < 32; ++i) { r[i] = a[i]; r[32 + i] = b[i]; }
 }
+// 32 consecutive columns of this thread's lane.
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+          "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]),
+          "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]),
+          "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 // Value a tf32 operand takes from a 32-bit container: the low 13 mantissa bits are not read.
@@ -234,17 +268,18 @@ __device__ __forceinline__ float exp2_unit(float x) {
 }
 
 // Barrier indices
-__device__ __forceinline__ constexpr int bar_full(int h) { return h; }
-__device__ __forceinline__ constexpr int bar_hi_free(int h) { return kHiStages + h; }
-__device__ __forceinline__ constexpr int bar_lo_ready(int l) { return 2 * kHiStages + l; }
-__device__ __forceinline__ constexpr int bar_lo_free(int l) { return 2 * kHiStages + kLoStages + l; }
-__device__ __forceinline__ constexpr int bar_acc_full(int b) { return 2 * kHiStages + 2 * kLoStages + b; }
-__device__ __forceinline__ constexpr int bar_acc_empty(int b) { return 2 * kHiStages + 2 * kLoStages + 2 + b; }
-constexpr int kBarWReady = 2 * kHiStages + 2 * kLoStages + 4;
-constexpr int kBarDrain = 2 * kHiStages + 2 * kLoStages + 5;
+__device__ __forceinline__ constexpr int bar_full(int h) { return h; }                       // slab landed in shared memory
+__device__ __forceinline__ constexpr int bar_x_free(int h) { return kXStages + h; }          // converters are done with the slab
+__device__ __forceinline__ constexpr int bar_a_ready(int l) { return 2 * kXStages + l; }     // A operand slot written
+__device__ __forceinline__ constexpr int bar_a_free(int l) { return 2 * kXStages + kASlots + l; }   // its MMAs completed
+__device__ __forceinline__ constexpr int bar_acc_full(int b) { return 2 * kXStages + 2 * kASlots + b; }
+__device__ __forceinline__ constexpr int bar_acc_empty(int b) { return 2 * kXStages + 2 * kASlots + 2 + b; }
+constexpr int kBarDrain = 2 * kXStages + 2 * kASlots + 5;
+constexpr int kBarRawFull = 2 * kXStages + 2 * kASlots + 6;    // raw heads of an instance landed in shared memory
+constexpr int kBarRawFree = 2 * kXStages + 2 * kASlots + 7;    // converters have turned them into the operand
 // per epilogue group: A = every thread is done reading the old tables, B = the new tables are written
-__device__ __forceinline__ constexpr int bar_epi_a(int g) { return 2 * kHiStages + 2 * kLoStages + 6 + g; }
-__device__ __forceinline__ constexpr int bar_epi_b(int g) { return 2 * kHiStages + 2 * kLoStages + 6 + kEpiGroups + g; }
+__device__ __forceinline__ constexpr int bar_epi_a(int g) { return 2 * kXStages + 2 * kASlots + 8 + g; }
+__device__ __forceinline__ constexpr int bar_epi_b(int g) { return 2 * kXStages + 2 * kASlots + 8 + kEpiGroups + g; }
 
 // Warp-uniform outcome of a bounded wait done by every lane.
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
@@ -275,11 +310,12 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
 
     // ---- set-up: barriers, tensor memory, zeroed W operand (padding rows and features stay zero)
     if (tid == 0) {
-        for (int h = 0; h < kHiStages; ++h) { mbar_init(bar(bar_full(h)), 1); mbar_init(bar(bar_hi_free(h)), 1); }
-        for (int l = 0; l < kLoStages; ++l) { mbar_init(bar(bar_lo_ready(l)), kConvThreads); mbar_init(bar(bar_lo_free(l)), 1); }
+        for (int h = 0; h < kXStages; ++h) { mbar_init(bar(bar_full(h)), 1); mbar_init(bar(bar_x_free(h)), kConvThreads); }
+        for (int l = 0; l < kASlots; ++l) { mbar_init(bar(bar_a_ready(l)), kConvThreads); mbar_init(bar(bar_a_free(l)), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(bar(bar_acc_full(b)), 1); mbar_init(bar(bar_acc_empty(b)), kEpiThreads); }
-        mbar_init(bar(kBarWReady), kConvThreads);
         mbar_init(bar(kBarDrain), 1);
+        mbar_init(bar(kBarRawFull), 1);
+        mbar_init(bar(kBarRawFree), kConvThreads);
         for (int g = 0; g < kEpiGroups; ++g) { mbar_init(bar(bar_epi_a(g)), kEpiThreads); mbar_init(bar(bar_epi_b(g)), kEpiThreads); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -297,71 +333,88 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
+    if (tmem != 0 && tid == 0) *abort_flag = 1;                // cannot happen for a whole-memory allocation
+    __syncthreads();
+    const bool tmem_ok = *abort_flag == 0;
 
-    if (warp == kProducerWarp) {
+    if (!tmem_ok) {
+        // unexpected tensor-memory base: nothing runs, the block reports the error below
+    } else if (warp == kProducerWarp) {
         // ================================================================ TMA producer (one thread)
         if (lane == 0) {
-            uint32_t slab_seq = 0;
+            uint32_t slab_seq = 0, w_seq = 0;
+            int cur_inst = -1;
+            const uint32_t w_bytes = (uint32_t)(A * D * C) * 4u;
             bool ok = true;
+            int4 d_next = t_begin < t_end ? prm.tiles[t_begin] : make_int4(-1, 0, 0, 0);
             for (int t = t_begin; t < t_end && ok; ++t) {
-                const int4 d = prm.tiles[t];
+                const int4 d = d_next;
                 if (d.x < 0) break;                            // valid tiles form a prefix of the block's range
+                if (t + 1 < t_end) d_next = prm.tiles[t + 1];
+                if (d.x != cur_inst) {                         // stage the heads of the instance this tile starts
+                    if (w_seq > 0 && !mbar_wait(bar(kBarRawFree), (w_seq - 1) & 1, abort_flag)) break;
+                    mbar_arrive_expect_tx(bar(kBarRawFull), w_bytes);
+                    bulk_load(base + Smem::wraw, (const float *)P.W + (int64_t)d.x * A * D * C, w_bytes, bar(kBarRawFull));
+                    ++w_seq; cur_inst = d.x;
+                }
                 const int row0 = (int)(tb.gstart[(int64_t)d.x * A] + d.y);
                 for (int s = 0; s < n_slabs; ++s, ++slab_seq) {
-                    const int h = slab_seq % kHiStages;
-                    const uint32_t use = slab_seq / kHiStages;
-                    if (use > 0 && !mbar_wait(bar(bar_hi_free(h)), (use - 1) & 1, abort_flag)) { ok = false; break; }
+                    const int h = slab_seq % kXStages;
+                    const uint32_t use = slab_seq / kXStages;
+                    if (use > 0 && !mbar_wait(bar(bar_x_free(h)), (use - 1) & 1, abort_flag)) { ok = false; break; }
                     mbar_arrive_expect_tx(bar(bar_full(h)), kSlabBytes);
-                    tma_load_2d(base + Smem::hi + h * kSlabBytes, &x_map, s * kSlabK, row0, bar(bar_full(h)));
+                    tma_load_2d(base + Smem::x + h * kSlabBytes, &x_map, s * kSlabK, row0, bar(bar_full(h)));
                 }
             }
-            if (!ok) {
+            if (!ok || *abort_flag) {
                 // copies already issued still land in shared memory: give them a bounded time to finish
-                const uint32_t first = slab_seq > (uint32_t)kHiStages ? slab_seq - kHiStages : 0;
+                if (w_seq > 0) {
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(bar(kBarRawFull), (w_seq - 1) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+                }
+                const uint32_t first = slab_seq > (uint32_t)kXStages ? slab_seq - kXStages : 0;
                 for (uint32_t q = first; q < slab_seq; ++q) {
                     const unsigned long long t0 = global_ns();
-                    while (!mbar_try_wait(bar(bar_full(q % kHiStages)), (q / kHiStages) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+                    while (!mbar_try_wait(bar(bar_full(q % kXStages)), (q / kXStages) & 1) && global_ns() - t0 < kWaitLimitNs) {}
                 }
             }
         }
     } else if (warp == kMmaWarp) {
         // ================================================================ MMA issuer (one thread)
+        // All tensor-memory addresses below are compile-time offsets: the allocation covers the whole tensor
+        // memory, so its base is column 0 (checked after the allocation).
         if (lane == 0) {
             constexpr uint32_t idesc_hi = instr_desc(2 * kCols), idesc_lo = instr_desc(kCols);
-            uint32_t slab_seq = 0, tile_seq = 0, w_seq = 0;
-            int cur_inst = -1;
+            const uint64_t w_desc = smem_desc(base + Smem::w);
+            uint32_t slab_seq = 0;
             bool ok = true;
+            int4 d_next = t_begin < t_end ? prm.tiles[t_begin] : make_int4(-1, 0, 0, 0);
             for (int t = t_begin; t < t_end && ok; ++t) {
-                const int4 d = prm.tiles[t];
+                const int4 d = d_next;
                 if (d.x < 0) break;                            // valid tiles form a prefix of the block's range
-                if (d.x != cur_inst) {                         // operand of the new instance's heads
-                    if (!mbar_wait(bar(kBarWReady), w_seq & 1, abort_flag)) break;
-                    ++w_seq; cur_inst = d.x;
-                }
-                const int b = tile_seq & 1;
-                const uint32_t acc_use = tile_seq >> 1;
+                if (t + 1 < t_end) d_next = prm.tiles[t + 1];
+                const uint32_t tile_seq = (uint32_t)(t - t_begin);
+                const uint32_t b = tile_seq & 1, acc_use = tile_seq >> 1;
                 if (acc_use > 0 && !mbar_wait(bar(bar_acc_empty(b)), (acc_use - 1) & 1, abort_flag)) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem + (uint32_t)(b * kAccCols);
+                const uint32_t d_tmem = b * kAccCols;
                 for (int s = 0; s < n_slabs; ++s, ++slab_seq) {
-                    const int h = slab_seq % kHiStages, l = slab_seq % kLoStages;
-                    if (!mbar_wait(bar(bar_full(h)), (slab_seq / kHiStages) & 1, abort_flag)) { ok = false; break; }
+                    const uint32_t l = slab_seq % kASlots;
+                    // the slot holds the rows of this slab; the same arrival says that the head operand of the
+                    // slab's features is in place (the converters rebuild it before they arrive)
+                    if (!mbar_wait(bar(bar_a_ready(l)), (slab_seq / kASlots) & 1, abort_flag)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_hi = base + Smem::hi + h * kSlabBytes, a_lo = base + Smem::lo + l * kSlabBytes;
-                    const uint32_t b_w = base + Smem::w + s * kSlabBytes;
+                    const uint32_t a_hi = kTmemA + l * kSlotCols, a_lo = a_hi + kSlabK;
+                    const uint64_t b_w = w_desc + (uint64_t)((s * kSlabBytes) >> 4);
 #pragma unroll
                     for (int k = 0; k < kSlabK / 8; ++k)       // x_hi [W_hi | W_lo] -> all 128 columns
-                        umma_tf32(d_tmem, smem_desc(a_hi + k * 32), smem_desc(b_w + k * 32), idesc_hi, (s | k) != 0);
-                    if (!mbar_wait(bar(bar_lo_ready(l)), (slab_seq / kLoStages) & 1, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
+                        umma_tf32_ts(d_tmem, a_hi + k * 8, b_w + (uint64_t)(k * 2), idesc_hi, (s | k) != 0);
 #pragma unroll
                     for (int k = 0; k < kSlabK / 8; ++k)       // x_lo W_hi -> the first 64 columns
-                        umma_tf32(d_tmem, smem_desc(a_lo + k * 32), smem_desc(b_w + k * 32), idesc_lo, 1u);
-                    umma_commit(bar(bar_hi_free(h)));
-                    umma_commit(bar(bar_lo_free(l)));
+                        umma_tf32_ts(d_tmem, a_lo + k * 8, b_w + (uint64_t)(k * 2), idesc_lo, 1u);
+                    umma_commit(bar(bar_a_free(l)));
                 }
                 if (ok) umma_commit(bar(bar_acc_full(b)));
-                ++tile_seq;
             }
             if (*abort_flag) {                                 // leaving early: let the issued MMAs finish first
                 umma_commit(bar(kBarDrain));
@@ -372,77 +425,81 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
     } else if (warp < kEpiWarp0) {
         // ================================================================ converter warps
         const int ct = tid - kConvWarp0 * 32;                  // 0..127
-        uint32_t slab_seq = 0, tile_seq = 0;
-        int cur_inst = -1, pre_inst = -1;
-        // Head operand: this thread owns logit column wn (= operand row) and half of the feature chunks.
-        // Its raw weights W[a][d][c] are gathered into registers ahead of time (consecutive threads read
-        // consecutive labels, so the loads coalesce) and written as 16-byte pieces of the swizzled rows.
-        const int wn = ct & (kCols - 1), wq0 = (ct >> 6) * (kMaxD / 8);   // 16 chunks of 4 features per thread
+        const int cquad = warp & 3, crow = cquad * 32 + lane;  // tensor-memory lanes this warp may write = its rows
+        uint32_t slab_seq = 0, w_seq = 0;
+        int cur_inst = -1;
+        // Head operand: this thread owns logit column wn (= operand row) and, per slab, 4 of its 8 chunks of 4
+        // features.  The raw heads W[a][d][c] of the instance were staged in shared memory by the producer;
+        // consecutive threads read consecutive labels (distinct banks) and write 16-byte pieces of the swizzled
+        // operand rows.  The operand is rebuilt slab by slab during the first tile of an instance: slab s as soon
+        // as the MMAs of the previous tile's slab s have completed, so the pipeline never drains.
+        const int wn = ct & (kCols - 1), wq0 = (ct >> 6) * 4;
         const int wa = wn / C, wc = wn - wa * C;
         const bool w_row = wn < A * C;
-        float wreg[kWRegs * 4];
-        auto fetch_w = [&](int inst) {
-            const float *src = (const float *)P.W + ((int64_t)inst * A + wa) * D * C + wc;
-#pragma unroll
-            for (int q = 0; q < kWRegs; ++q)
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int dd = (wq0 + q) * 4 + u;
-                    wreg[q * 4 + u] = (w_row && dd < D) ? src[(int64_t)dd * C] : 0.f;
-                }
-            pre_inst = inst;
-        };
+        const float *wraw = reinterpret_cast<const float *>(sm + Smem::wraw) + wa * D * C + wc;
         bool ok = true;
+        int4 d_next = t_begin < t_end ? prm.tiles[t_begin] : make_int4(-1, 0, 0, 0);
         for (int t = t_begin; t < t_end && ok; ++t) {
-            const int4 d = prm.tiles[t];
-            if (d.x < 0) break;                            // valid tiles form a prefix of the block's range
-            if (d.x != cur_inst) {
-                if (pre_inst != d.x) fetch_w(d.x);
-                // every MMA that reads the previous operand belongs to the previous tile: wait for its accumulator
-                if (tile_seq > 0) {
-                    const uint32_t pt = tile_seq - 1;
-                    if (!warp_wait(bar(bar_acc_full(pt & 1)), (pt >> 1) & 1, abort_flag)) break;
-                }
-                if (w_row) {
+            const int4 d = d_next;
+            if (d.x < 0) break;                                // valid tiles form a prefix of the block's range
+            if (t + 1 < t_end) d_next = prm.tiles[t + 1];
+            const bool new_inst = d.x != cur_inst;
+            cur_inst = d.x;
+            if (new_inst && !warp_wait(bar(kBarRawFull), w_seq & 1, abort_flag)) break;
+            for (int s = 0; s < n_slabs; ++s, ++slab_seq) {
+                const int h = slab_seq % kXStages, l = slab_seq % kASlots;
+                const uint32_t a_use = slab_seq / kASlots;
+                if (new_inst) {
+                    if (slab_seq >= (uint32_t)n_slabs) {       // MMAs of the previous tile's slab s read the old operand
+                        const uint32_t ps = slab_seq - (uint32_t)n_slabs;
+                        if (!warp_wait(bar(bar_a_free(ps % kASlots)), (ps / kASlots) & 1, abort_flag)) { ok = false; break; }
+                    }
+                    if (w_row) {
 #pragma unroll
-                    for (int q = 0; q < kWRegs; ++q) {
-                        const int j = wq0 + q;                 // chunk of 4 features: slab j / 8, 16-byte piece j % 8
-                        if (j * 4 < D) {
-                            const uint32_t off = (uint32_t)((j >> 3) * kSlabBytes + wn * 128 + (((j & 7) ^ (wn & 7)) << 4));
-                            const float w0 = wreg[q * 4 + 0] * kLog2e, w1 = wreg[q * 4 + 1] * kLog2e;
-                            const float w2 = wreg[q * 4 + 2] * kLog2e, w3 = wreg[q * 4 + 3] * kLog2e;
-                            float4 hi, lo;
-                            hi.x = tf32_part(w0); lo.x = w0 - hi.x;
-                            hi.y = tf32_part(w1); lo.y = w1 - hi.y;
-                            hi.z = tf32_part(w2); lo.z = w2 - hi.z;
-                            hi.w = tf32_part(w3); lo.w = w3 - hi.w;
-                            *reinterpret_cast<float4 *>(sm + Smem::w + off) = hi;
-                            *reinterpret_cast<float4 *>(sm + Smem::w + off + kCols * 128) = lo;
+                        for (int q = 0; q < 4; ++q) {
+                            const int j = wq0 + q, dd = s * kSlabK + j * 4;   // 16-byte piece j of the operand row
+                            if (dd < D) {
+                                const uint32_t off = (uint32_t)(s * kSlabBytes + wn * 128 + ((j ^ (wn & 7)) << 4));
+                                const float *src = wraw + dd * C;
+                                const float w0 = src[0] * kLog2e, w1 = src[C] * kLog2e;
+                                const float w2 = src[2 * C] * kLog2e, w3 = src[3 * C] * kLog2e;
+                                float4 hi, lo;
+                                hi.x = tf32_part(w0); lo.x = w0 - hi.x;
+                                hi.y = tf32_part(w1); lo.y = w1 - hi.y;
+                                hi.z = tf32_part(w2); lo.z = w2 - hi.z;
+                                hi.w = tf32_part(w3); lo.w = w3 - hi.w;
+                                *reinterpret_cast<float4 *>(sm + Smem::w + off) = hi;
+                                *reinterpret_cast<float4 *>(sm + Smem::w + off + kCols * 128) = lo;
+                            }
                         }
                     }
+                    fence_proxy_async();
+                    if (s == n_slabs - 1) { mbar_arrive(bar(kBarRawFree)); ++w_seq; }
                 }
-                fence_proxy_async();
-                mbar_arrive(bar(kBarWReady));
-                cur_inst = d.x;
-                if (d.x + 1 < P.I) fetch_w(d.x + 1);           // the next instance's heads, in flight while this one runs
-            }
-            for (int s = 0; s < n_slabs; ++s, ++slab_seq) {
-                const int h = slab_seq % kHiStages, l = slab_seq % kLoStages;
-                const uint32_t lo_use = slab_seq / kLoStages;
-                if (!warp_wait(bar(bar_full(h)), (slab_seq / kHiStages) & 1, abort_flag)) { ok = false; break; }
-                if (lo_use > 0 && !warp_wait(bar(bar_lo_free(l)), (lo_use - 1) & 1, abort_flag)) { ok = false; break; }
-                const float4 *src = reinterpret_cast<const float4 *>(sm + Smem::hi + h * kSlabBytes);
-                float4 *dst = reinterpret_cast<float4 *>(sm + Smem::lo + l * kSlabBytes);
+                if (!warp_wait(bar(bar_full(h)), (slab_seq / kXStages) & 1, abort_flag)) { ok = false; break; }
+                // this thread's row of the slab: 8 pieces of 16 bytes, un-swizzled into feature order
+                const unsigned char *xrow = sm + Smem::x + h * kSlabBytes + crow * 128;
+                uint32_t v[kSlabK];
 #pragma unroll
-                for (int q = 0; q < kSlabBytes / 16 / kConvThreads; ++q) {
-                    const float4 x = src[q * kConvThreads + ct];
-                    dst[q * kConvThreads + ct] = make_float4(x.x - tf32_part(x.x), x.y - tf32_part(x.y),
-                                                             x.z - tf32_part(x.z), x.w - tf32_part(x.w));
+                for (int j = 0; j < 8; ++j) {
+                    const uint4 q = *reinterpret_cast<const uint4 *>(xrow + ((j ^ (crow & 7)) << 4));
+                    v[4 * j] = q.x; v[4 * j + 1] = q.y; v[4 * j + 2] = q.z; v[4 * j + 3] = q.w;
                 }
-                fence_proxy_async();
-                mbar_arrive(bar(bar_lo_ready(l)));
+                if (a_use > 0 && !warp_wait(bar(bar_a_free(l)), (a_use - 1) & 1, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t a_hi = ((uint32_t)(cquad * 32) << 16) + (uint32_t)(kTmemA + l * kSlotCols);
+                tmem_st32(a_hi, v);                            // read as x_hi: the unit drops the low mantissa bits
+#pragma unroll
+                for (int k = 0; k < kSlabK; ++k) {
+                    const float x = __uint_as_float(v[k]);
+                    v[k] = __float_as_uint(x - tf32_part(x));
+                }
+                tmem_st32(a_hi + kSlabK, v);
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(bar(bar_a_ready(l)));
+                mbar_arrive(bar(bar_x_free(h)));
             }
-            ++tile_seq;
         }
     } else {
         // ================================================================ epilogue warps (one row per thread)
