@@ -46,7 +46,8 @@ constexpr int kTmemA = 2 * kAccCols;       // accumulators first (epilogue reads
 constexpr int kSlotCols = 2 * kSlabK;
 constexpr int kProducerWarp = 0, kMmaWarp = 1, kConvWarp0 = 2, kEpiWarp0 = 6;
 constexpr int kEpiGroups = 2;              // epilogue warpgroups; group g takes every second tile and accumulator g
-constexpr int kThreads = 32 * (6 + 4 * kEpiGroups);
+constexpr int kMmaWarp2 = 6 + 4 * kEpiGroups;   // second MMA issuer: the two take alternate tiles (and accumulators)
+constexpr int kThreads = 32 * (7 + 4 * kEpiGroups);
 constexpr int kConvThreads = 128, kEpiThreads = 128;
 constexpr float kLog2e = 1.44269502162933349609375f;   // folded into W and the bias: the softmax runs in base 2
 constexpr int kWChunks = (kCols * kMaxD / 4) / kConvThreads;  // 4-feature pieces of the head operand per converter thread
@@ -62,7 +63,7 @@ struct Smem {                               // byte offsets from the 1024-byte a
     static constexpr int tab_floats = tab_psum + 16;
     static constexpr int tabs = x + kXStages * kSlabBytes;
     static constexpr int bars = tabs + kEpiGroups * tab_floats * 4;
-    static constexpr int n_bars = 2 * kXStages + 2 * kASlots + 8 + 2 * kEpiGroups;
+    static constexpr int n_bars = 2 * kXStages + 3 * kASlots + 9 + 2 * kEpiGroups;
     static constexpr int misc = bars + n_bars * 8;                     // tmem base, abort flag
     static constexpr int end = misc + 16;
     static constexpr int bytes = end + 1024;                           // slack for the manual alignment
@@ -268,18 +269,22 @@ __device__ __forceinline__ float exp2_unit(float x) {
 }
 
 // Barrier indices
+constexpr int kBarBase2 = 2 * kXStages + 3 * kASlots;
 __device__ __forceinline__ constexpr int bar_full(int h) { return h; }                       // slab landed in shared memory
 __device__ __forceinline__ constexpr int bar_x_free(int h) { return kXStages + h; }          // converters are done with the slab
-__device__ __forceinline__ constexpr int bar_a_ready(int l) { return 2 * kXStages + l; }     // A operand slot written
-__device__ __forceinline__ constexpr int bar_a_free(int l) { return 2 * kXStages + kASlots + l; }   // its MMAs completed
-__device__ __forceinline__ constexpr int bar_acc_full(int b) { return 2 * kXStages + 2 * kASlots + b; }
-__device__ __forceinline__ constexpr int bar_acc_empty(int b) { return 2 * kXStages + 2 * kASlots + 2 + b; }
-constexpr int kBarDrain = 2 * kXStages + 2 * kASlots + 5;
-constexpr int kBarRawFull = 2 * kXStages + 2 * kASlots + 6;    // raw heads of an instance landed in shared memory
-constexpr int kBarRawFree = 2 * kXStages + 2 * kASlots + 7;    // converters have turned them into the operand
+// A operand slot l written for MMA issuer g (each issuer waits on its own barriers: a waiter that is a whole
+// phase ahead of another one would pass a shared barrier early)
+__device__ __forceinline__ constexpr int bar_a_ready(int g, int l) { return 2 * kXStages + g * kASlots + l; }
+__device__ __forceinline__ constexpr int bar_a_free(int l) { return 2 * kXStages + 2 * kASlots + l; }   // its MMAs completed
+__device__ __forceinline__ constexpr int bar_acc_full(int b) { return kBarBase2 + b; }
+__device__ __forceinline__ constexpr int bar_acc_empty(int b) { return kBarBase2 + 2 + b; }
+constexpr int kBarDrain = kBarBase2 + 5;
+constexpr int kBarRawFull = kBarBase2 + 6;    // raw heads of an instance landed in shared memory
+constexpr int kBarRawFree = kBarBase2 + 7;    // converters have turned them into the operand
+constexpr int kBarDrain2 = kBarBase2 + 8;     // drain barrier of the second MMA issuer
 // per epilogue group: A = every thread is done reading the old tables, B = the new tables are written
-__device__ __forceinline__ constexpr int bar_epi_a(int g) { return 2 * kXStages + 2 * kASlots + 8 + g; }
-__device__ __forceinline__ constexpr int bar_epi_b(int g) { return 2 * kXStages + 2 * kASlots + 8 + kEpiGroups + g; }
+__device__ __forceinline__ constexpr int bar_epi_a(int g) { return kBarBase2 + 9 + g; }
+__device__ __forceinline__ constexpr int bar_epi_b(int g) { return kBarBase2 + 9 + kEpiGroups + g; }
 
 // Warp-uniform outcome of a bounded wait done by every lane.
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
@@ -311,9 +316,13 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
     // ---- set-up: barriers, tensor memory, zeroed W operand (padding rows and features stay zero)
     if (tid == 0) {
         for (int h = 0; h < kXStages; ++h) { mbar_init(bar(bar_full(h)), 1); mbar_init(bar(bar_x_free(h)), kConvThreads); }
-        for (int l = 0; l < kASlots; ++l) { mbar_init(bar(bar_a_ready(l)), kConvThreads); mbar_init(bar(bar_a_free(l)), 1); }
+        for (int l = 0; l < kASlots; ++l) {
+            mbar_init(bar(bar_a_ready(0, l)), kConvThreads); mbar_init(bar(bar_a_ready(1, l)), kConvThreads);
+            mbar_init(bar(bar_a_free(l)), 1);
+        }
         for (int b = 0; b < 2; ++b) { mbar_init(bar(bar_acc_full(b)), 1); mbar_init(bar(bar_acc_empty(b)), kEpiThreads); }
         mbar_init(bar(kBarDrain), 1);
+        mbar_init(bar(kBarDrain2), 1);
         mbar_init(bar(kBarRawFull), 1);
         mbar_init(bar(kBarRawFree), kConvThreads);
         for (int g = 0; g < kEpiGroups; ++g) { mbar_init(bar(bar_epi_a(g)), kEpiThreads); mbar_init(bar(bar_epi_b(g)), kEpiThreads); }
@@ -379,21 +388,25 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
                 }
             }
         }
-    } else if (warp == kMmaWarp) {
-        // ================================================================ MMA issuer (one thread)
+    } else if (warp == kMmaWarp || warp == kMmaWarp2) {
+        // ================================================================ MMA issuers (one thread each)
+        // Issuing an MMA costs about as much time as the tensor pipe needs for it at this tile shape, so two
+        // threads issue: issuer g takes tiles g, g + 2, ... and accumulator g; their MMAs interleave in the pipe.
         // All tensor-memory addresses below are compile-time offsets: the allocation covers the whole tensor
         // memory, so its base is column 0 (checked after the allocation).
         if (lane == 0) {
             constexpr uint32_t idesc_hi = instr_desc(2 * kCols), idesc_lo = instr_desc(kCols);
             const uint64_t w_desc = smem_desc(base + Smem::w);
-            uint32_t slab_seq = 0;
+            const int mg = warp == kMmaWarp ? 0 : 1;
             bool ok = true;
-            int4 d_next = t_begin < t_end ? prm.tiles[t_begin] : make_int4(-1, 0, 0, 0);
-            for (int t = t_begin; t < t_end && ok; ++t) {
+            uint32_t rdy_par = 0;                              // bit l: parity of this issuer's next wait on slot l
+            int4 d_next = t_begin + mg < t_end ? prm.tiles[t_begin + mg] : make_int4(-1, 0, 0, 0);
+            for (int t = t_begin + mg; t < t_end && ok; t += 2) {
                 const int4 d = d_next;
                 if (d.x < 0) break;                            // valid tiles form a prefix of the block's range
-                if (t + 1 < t_end) d_next = prm.tiles[t + 1];
+                if (t + 2 < t_end) d_next = prm.tiles[t + 2];
                 const uint32_t tile_seq = (uint32_t)(t - t_begin);
+                uint32_t slab_seq = tile_seq * (uint32_t)n_slabs;
                 const uint32_t b = tile_seq & 1, acc_use = tile_seq >> 1;
                 if (acc_use > 0 && !mbar_wait(bar(bar_acc_empty(b)), (acc_use - 1) & 1, abort_flag)) break;
                 tc_fence_after();
@@ -402,7 +415,8 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
                     const uint32_t l = slab_seq % kASlots;
                     // the slot holds the rows of this slab; the same arrival says that the head operand of the
                     // slab's features is in place (the converters rebuild it before they arrive)
-                    if (!mbar_wait(bar(bar_a_ready(l)), (slab_seq / kASlots) & 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(bar(bar_a_ready(mg, l)), (rdy_par >> l) & 1, abort_flag)) { ok = false; break; }
+                    rdy_par ^= 1u << l;
                     tc_fence_after();
                     const uint32_t a_hi = kTmemA + l * kSlotCols, a_lo = a_hi + kSlabK;
                     const uint64_t b_w = w_desc + (uint64_t)((s * kSlabBytes) >> 4);
@@ -417,9 +431,10 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
                 if (ok) umma_commit(bar(bar_acc_full(b)));
             }
             if (*abort_flag) {                                 // leaving early: let the issued MMAs finish first
-                umma_commit(bar(kBarDrain));
+                const uint32_t drain = bar(mg ? kBarDrain2 : kBarDrain);
+                umma_commit(drain);
                 const unsigned long long t0 = global_ns();
-                while (!mbar_try_wait(bar(kBarDrain), 0) && global_ns() - t0 < kWaitLimitNs) {}
+                while (!mbar_try_wait(drain, 0) && global_ns() - t0 < kWaitLimitNs) {}
             }
         }
     } else if (warp < kEpiWarp0) {
@@ -443,6 +458,7 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
             const int4 d = d_next;
             if (d.x < 0) break;                                // valid tiles form a prefix of the block's range
             if (t + 1 < t_end) d_next = prm.tiles[t + 1];
+            const int mg = (t - t_begin) & 1;                  // MMA issuer of this tile
             const bool new_inst = d.x != cur_inst;
             cur_inst = d.x;
             if (new_inst && !warp_wait(bar(kBarRawFull), w_seq & 1, abort_flag)) break;
@@ -497,7 +513,7 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
                 tmem_st32(a_hi + kSlabK, v);
                 tmem_wait_st();
                 tc_fence_before();
-                mbar_arrive(bar(bar_a_ready(l)));
+                mbar_arrive(bar(bar_a_ready(mg, l)));
                 mbar_arrive(bar(bar_x_free(h)));
             }
         }
