@@ -250,7 +250,7 @@ def main():
         tj = json.load(open(tpath)).get(args.workload)
         if tj and tj.get("kernel_version") == KERNEL_VERSION:
             traffic = tj["dram_bytes_per_request"] * n
-    roofline = {"bound": "hbm", "kernel": "k_score_small" if ses_small(w) else "k_score_tiled", "achieved": achieved,
+    roofline = {"bound": "hbm", "kernel": ("k_score_tiled", "k_score_small", "k_score_mma")[int(st.get("score_kernel", 0))], "achieved": achieved,
                 "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak if achieved else None,
                 "traffic": traffic, "algorithmic_bytes": bytes_per_launch, "kernel_ms": score_ms}
 
@@ -305,11 +305,7 @@ def main():
         dist.destroy_process_group()
 
 
-KERNEL_VERSION = 1     # bump when the scoring kernel changes: stale ncu traffic figures are then ignored
-
-
-def ses_small(w):
-    return int(w.feat_dtype) == 0 and int(w.feat_dim) % 4 == 0 and int(w.n_classes) <= 64
+KERNEL_VERSION = 4     # bump when the scoring kernel changes: stale ncu traffic figures are then ignored
 
 
 if __name__ == "__main__":

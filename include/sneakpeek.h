@@ -109,6 +109,8 @@ typedef struct {
      * calls since the previous sp_get_stats() (at most 512 calls are kept), and the number of calls summed. */
     int64_t score_calls, sched_calls;
     double score_kernel_ms, sched_kernel_ms;
+    /* Scoring kernel the loaded profiles select: 0 = tiled FP32, 1 = small-head FP32, 2 = tensor-core (tcgen05). */
+    int32_t score_kernel, pad_;
 } sp_stats;
 
 /* Creates a context on CUDA device `device` that enqueues on `cuda_stream` (a cudaStream_t; NULL = the

@@ -57,7 +57,8 @@ class _Options(C.Structure):
 class _Stats(C.Structure):
     _fields_ = [("kernel_launches", C.c_int64), ("rounds", C.c_int64), ("exact_utility", C.c_int64),
                 ("exact_priority", C.c_int64), ("exact_rows", C.c_int64), ("score_calls", C.c_int64),
-                ("sched_calls", C.c_int64), ("score_kernel_ms", C.c_double), ("sched_kernel_ms", C.c_double)]
+                ("sched_calls", C.c_int64), ("score_kernel_ms", C.c_double), ("sched_kernel_ms", C.c_double),
+                ("score_kernel", C.c_int32), ("pad_", C.c_int32)]
 
 
 class _StaticHead(C.Structure):

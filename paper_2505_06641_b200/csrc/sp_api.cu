@@ -610,6 +610,8 @@ sp_status sp_get_stats(sp_ctx *c, sp_stats *out) {
     out->exact_rows = (int64_t)s[3];
     out->score_kernel_ms = drain_events(c->ev_score, &out->score_calls);
     out->sched_kernel_ms = drain_events(c->ev_sched, &out->sched_calls);
+    out->score_kernel = c->mma_ct ? 2 : c->small_ct ? 1 : 0;
+    out->pad_ = 0;
     return SP_OK;
 }
 
