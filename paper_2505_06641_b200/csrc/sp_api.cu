@@ -12,6 +12,7 @@
 #include "sp_score_tiled.cuh"
 #include "sp_score_mma.cuh"
 #include "sp_sched.cuh"
+#include "sp_sched_warp.cuh"
 
 using namespace sp;
 
@@ -34,6 +35,7 @@ struct sp_ctx {
     std::string err;
     bool have_profiles = false;
     bool have_table = false;
+    bool sched_started = false;  // a scheduling call has run on the current request table
     HostProfiles hp;
     DevProfiles P{};
     DevTable tb{};
@@ -239,8 +241,8 @@ sp_status sp_create(sp_ctx **out, int device, void *cuda_stream) {
     c->device = device;
     c->stream = (cudaStream_t)cuda_stream;
     if (cudaDeviceGetAttribute(&c->n_sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || c->n_sms < 1) c->n_sms = 1;
-    if (ensure(c, c->flags, 2 * sizeof(int)) != SP_OK || ensure(c, c->stats, 4 * sizeof(unsigned long long)) != SP_OK ||
-        cudaMemsetAsync(c->flags.p, 0, 2 * sizeof(int), c->stream) != cudaSuccess ||
+    if (ensure(c, c->flags, 4 * sizeof(int)) != SP_OK || ensure(c, c->stats, 4 * sizeof(unsigned long long)) != SP_OK ||
+        cudaMemsetAsync(c->flags.p, 0, 4 * sizeof(int), c->stream) != cudaSuccess ||
         cudaMemsetAsync(c->stats.p, 0, 4 * sizeof(unsigned long long), c->stream) != cudaSuccess) {
         delete c;
         return SP_ECUDA;
@@ -439,6 +441,7 @@ sp_status sp_reset(sp_ctx *c) {
     SP_CUDA(c, cudaMemsetAsync((int *)c->flags.p + 1, 0, sizeof(int), c->stream));
     SP_CUDA(c, cudaMemsetAsync(c->stats.p, 0, 4 * sizeof(unsigned long long), c->stream));
     c->have_table = false;
+    c->sched_started = false;
     c->tb.n = 0;
     return SP_OK;
 }
@@ -534,6 +537,7 @@ sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, 
         SP_TRY(mark(c, c->ev_score));
     }
     c->have_table = true;
+    c->sched_started = false;
     return SP_OK;
 }
 
@@ -578,9 +582,25 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
     int sort_cap = P.I > 1 ? 1024 : 8192;
     while (sort_cap > 64 && sort_cap / 2 >= per_inst) sort_cap /= 2;
     sp.sort_cap = sort_cap;
+    sp.zbuf_warps = c->sched_threads / 32;
     const SchedSmem L(sort_cap, P.Mmax, sp.bmax, kMaxModelsPerApp * kMaxBatchSizes);
     SP_CUDA(c, cudaFuncSetAttribute(k_sched, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.end));
     SP_TRY(mark(c, c->ev_sched));
+    // Batched mode, first call on a fresh table: one warp per instance takes every instance that fits its slice of
+    // shared memory; k_sched follows for the rest (it returns at once when nothing is left).
+    if (P.I > 1 && !c->opt.trace_mode && !c->sched_started && c->tb.n > 0) {
+        int64_t wcap = 32;
+        while (wcap < (c->tb.n + P.I - 1) / P.I) wcap <<= 1;
+        const WarpSchedSmem W((int)wcap, P.Mmax, sp.bmax);
+        if (wcap <= 2048 && W.end * kWarpSchedWarps <= 200 * 1024) {
+            SP_CUDA(c, cudaMemsetAsync((int *)c->flags.p + 2, 0, sizeof(int), c->stream));
+            SP_CUDA(c, cudaFuncSetAttribute(k_sched_warp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(W.end * kWarpSchedWarps)));
+            k_sched_warp<<<(P.I + kWarpSchedWarps - 1) / kWarpSchedWarps, kWarpSchedWarps * 32, W.end * kWarpSchedWarps, c->stream>>>(sp, (int)wcap);
+            SP_TRY(launched(c, "k_sched_warp"));
+            sp.only_unstarted = 1;
+        }
+    }
+    c->sched_started = true;
     k_sched<<<P.I, c->sched_threads, L.end, c->stream>>>(sp);
     SP_TRY(launched(c, "k_sched"));
     return mark(c, c->ev_sched);

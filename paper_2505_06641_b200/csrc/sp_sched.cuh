@@ -45,6 +45,8 @@ struct SchedParams {
     int32_t *n_done;
     int sort_cap;               // SortKey entries available in shared memory
     int bmax;                   // largest allowed batch size
+    int zbuf_warps;             // zbuf rows per instance
+    int only_unstarted;         // 1: k_sched runs after k_sched_warp and takes only what that kernel left (flags[2])
 };
 
 __device__ __forceinline__ bool key_less(const SortKey &a, const SortKey &b) {
@@ -258,6 +260,7 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
         if (tid == 0 && sp.n_done) sp.n_done[inst] = 0;
         return;
     }
+    if (sp.only_unstarted && (!sp.flags[2] || sp.state[inst].started)) return;   // the warp kernel has done it
     const int64_t r0 = tb.gstart[(int64_t)inst * A], r1 = tb.gstart[(int64_t)(inst + 1) * A];
     const int64_t n_inst = r1 - r0;
     if (tid == 0) st = sp.state[inst];

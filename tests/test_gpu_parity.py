@@ -164,3 +164,52 @@ def test_errors_are_reported_not_crashes():
         api.sp_load_profiles(ses.ctx, w)
     assert e.value.status == api.SP_EINVAL
     ses.close()
+
+
+def _drop_requests(w, keep):
+    for f in ("feats", "app", "arrival_ns", "deadline_ns", "instance"):
+        setattr(w, f, np.ascontiguousarray(getattr(w, f)[keep]))
+    return w
+
+
+def test_batched_rounds_resume_after_a_partial_call():
+    """Batched mode: a call that stops after one round per instance leaves a state the next calls continue from."""
+    from oracle import oracle
+    from paper_2505_06641_b200 import api, runner
+    w = synth.make_workload("C4", n_instances=6, n_requests=200)
+    s = oracle.score(w)
+    od = oracle.drain(w, s.acc, s.v)
+    ses = runner.Session(w)
+    ses.upload(); ses.alloc_outputs(4); ses.score()
+    got = [[] for _ in range(6)]
+    for _ in range(64):
+        ses.schedule(1)
+        api.sp_check(ses.ctx)
+        nd = ses.n_done.cpu().numpy()
+        rr = ses.rounds.cpu().numpy().reshape(6, -1).view(api.ROUND_DTYPE)
+        for k in range(6):
+            got[k].extend(rr[k, :nd[k]].copy())
+        if nd.sum() == 0:
+            break
+    for k in range(6):
+        n = int(od.n_rounds[k])
+        assert len(got[k]) == n
+        for f in ("round", "app", "model", "batch", "n_members", "n_expired", "t_start_ns", "t_end_ns"):
+            assert [int(r[f]) for r in got[k]] == [int(x) for x in od.rounds[k, :n][f]], (k, f)
+    api.sp_get_requests(ses.ctx, 0, ses.n, ses.recs)
+    reqs = ses.recs.cpu().numpy().reshape(-1).view(api.REQ_DTYPE)[:ses.n]
+    for f in ("status", "round", "model", "order"):
+        assert np.array_equal(reqs[f], od.reqs[f]), f
+    ses.close()
+
+
+def test_batched_instances_of_very_different_sizes():
+    """One instance far above the average size is left to the block-per-instance kernel in the same call."""
+    w = synth.make_workload("C4", n_instances=8, n_requests=512)
+    inst = np.asarray(w.instance)
+    rank = np.arange(len(inst)) - np.searchsorted(inst, inst)      # position inside the instance
+    keep = (inst == 3) | (rank < 40)
+    w = _drop_requests(w, keep)
+    s, od, res = _both(w)
+    check_scores(res, s)
+    check_schedule(w, res, od)
