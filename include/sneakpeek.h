@@ -95,8 +95,8 @@ typedef struct {
 typedef struct {
     int32_t trace_mode;   /* 0: every scored request is pending at once; 1: a request joins when arrival <= clock */
     int32_t timing;       /* 1: bracket the scoring and the scheduling kernel with CUDA events (see sp_stats) */
-    double guard_utility; /* relative margin under which candidate utilities are re-evaluated in fp64 (default 1e-4) */
-    double guard_priority;/* same for group priorities (default 2e-5) */
+    double guard_utility; /* relative margin under which candidate utilities are re-evaluated in fp64 (default 2e-5) */
+    double guard_priority;/* same for group priorities (default 2e-6) */
 } sp_options;
 
 typedef struct {

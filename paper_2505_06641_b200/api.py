@@ -161,8 +161,8 @@ def sp_load_profiles(ctx: int, w) -> None:
     _ok(ctx, load_library().sp_load_profiles(ctx, C.byref(p)))
 
 
-def sp_set_options(ctx: int, trace_mode: bool = False, guard_utility: float = 1e-4,
-                   guard_priority: float = 2e-5, timing: bool = False) -> None:
+def sp_set_options(ctx: int, trace_mode: bool = False, guard_utility: float = 2e-5,
+                   guard_priority: float = 2e-6, timing: bool = False) -> None:
     o = _Options(int(bool(trace_mode)), int(bool(timing)), float(guard_utility), float(guard_priority))
     _ok(ctx, load_library().sp_set_options(ctx, C.byref(o)))
 

@@ -39,7 +39,7 @@ struct sp_ctx {
     HostProfiles hp;
     DevProfiles P{};
     DevTable tb{};
-    sp_options opt{0, 0, 1e-4, 2e-5};
+    sp_options opt{0, 0, 2e-5, 2e-6};
     std::vector<cudaEvent_t> ev_score, ev_sched;   // start/stop pairs recorded since the last sp_get_stats
     int64_t launches = 0;
     int sched_threads = 1024;
@@ -50,7 +50,7 @@ struct sp_ctx {
     // profile buffers
     Buf W, bias, recall, prior, prior_dot, prior_sum, lat_alpha, lat_beta, swap;
     // per-instance state and scratch
-    Buf state, zbuf, flags, stats, cnt, gstart, cursor, small_start, tiled_start, small_tiles;
+    Buf state, zbuf, flags, stats, cnt, gstart, cursor, small_start, tiled_start, small_tiles, scan_partial;
     // per-request buffers
     Buf acc32, v32, acc64, v64, exact, recs, perm, q_id0, q_id1, q_dl0, q_dl1, q_pw0, q_pw1, sort_scratch;
     // staging of sp_run_host
@@ -115,7 +115,7 @@ __global__ void k_state_reset(InstState *st, int n_inst, int mode) {
     if (i >= n_inst) return;
     InstState s = st[i];
     if (mode == 0) { s.T = 0; s.L = -1; }
-    s.next_order = 1; s.Tref = 0; s.inserted = 0; s.round = 0; s.exp_since = 0; s.started = 0;
+    s.next_order = 1; s.Tref = 0; s.inserted = 0; s.round = 0; s.exp_since = 0; s.started = 0; s.handed = 0; s.pad_ = 0;
     for (int a = 0; a < kMaxApps; ++a) { s.head[a] = 0; s.tail[a] = 0; s.cur[a] = 0; }
     st[i] = s;
 }
@@ -260,7 +260,7 @@ void sp_destroy(sp_ctx *c) {
     drain_events(c->ev_sched, &dummy);
     Buf *all[] = {&c->W, &c->bias, &c->recall, &c->prior, &c->prior_dot, &c->prior_sum, &c->lat_alpha, &c->lat_beta,
                   &c->swap, &c->state, &c->zbuf, &c->flags, &c->stats, &c->cnt, &c->gstart, &c->cursor,
-                  &c->small_start, &c->tiled_start, &c->small_tiles, &c->acc32, &c->v32, &c->acc64, &c->v64, &c->exact, &c->recs,
+                  &c->small_start, &c->tiled_start, &c->small_tiles, &c->scan_partial, &c->acc32, &c->v32, &c->acc64, &c->v64, &c->exact, &c->recs,
                   &c->perm, &c->q_id0, &c->q_id1, &c->q_dl0, &c->q_dl1, &c->q_pw0, &c->q_pw1, &c->sort_scratch,
                   &c->h_feats, &c->h_app, &c->h_arrival, &c->h_deadline, &c->h_instance, &c->h_t0, &c->h_loaded,
                   &c->h_rounds, &c->h_ndone};
@@ -489,9 +489,19 @@ sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, 
         k_group_count<<<gb, 256, 0, c->stream>>>(P, tb, c->opt.trace_mode, (int *)c->flags.p);
         SP_TRY(launched(c, "k_group_count"));
     }
-    k_group_scan<<<1, 1024, 0, c->stream>>>((int)nkeys, P.A, tb.cnt, tb.gstart, (int32_t *)c->tiled_start.p,
-                                            (int32_t *)c->small_start.p);
-    SP_TRY(launched(c, "k_group_scan"));
+    if (nkeys <= 4 * (size_t)kScanChunk) {
+        k_group_scan<<<1, 1024, 0, c->stream>>>((int)nkeys, P.A, tb.cnt, tb.gstart, (int32_t *)c->tiled_start.p,
+                                                (int32_t *)c->small_start.p);
+        SP_TRY(launched(c, "k_group_scan"));
+    } else {                                           // many keys: per-block totals, then one scan block per chunk
+        const int nblk = (int)(nkeys / kScanChunk + 1);    // covers index nkeys (the grand total) as well
+        SP_TRY(ensure(c, c->scan_partial, (size_t)3 * nblk * sizeof(long long)));
+        k_group_partials<<<nblk, kScanChunk, 0, c->stream>>>((int)nkeys, P.A, tb.cnt, (long long *)c->scan_partial.p);
+        SP_TRY(launched(c, "k_group_partials"));
+        k_group_scan_blocks<<<nblk, kScanChunk, 0, c->stream>>>((int)nkeys, P.A, tb.cnt, (const long long *)c->scan_partial.p,
+                                                              tb.gstart, (int32_t *)c->tiled_start.p, (int32_t *)c->small_start.p);
+        SP_TRY(launched(c, "k_group_scan_blocks"));
+    }
     if (n > 0) {
         int grid = 0;
         if (c->small_ct || c->mma_ct) {
@@ -592,10 +602,12 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
         int64_t wcap = 32;
         while (wcap < (c->tb.n + P.I - 1) / P.I) wcap <<= 1;
         const WarpSchedSmem W((int)wcap, P.Mmax, sp.bmax);
-        if (wcap <= 2048 && W.end * kWarpSchedWarps <= 200 * 1024) {
+        if (wcap <= 2048 && P.sumM <= 32 && W.end * kWarpSchedWarps <= 200 * 1024) {
+            const int wgrid = (P.I + kWarpSchedWarps - 1) / kWarpSchedWarps;
+            const size_t wsmem = W.end * kWarpSchedWarps;
             SP_CUDA(c, cudaMemsetAsync((int *)c->flags.p + 2, 0, sizeof(int), c->stream));
-            SP_CUDA(c, cudaFuncSetAttribute(k_sched_warp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(W.end * kWarpSchedWarps)));
-            k_sched_warp<<<(P.I + kWarpSchedWarps - 1) / kWarpSchedWarps, kWarpSchedWarps * 32, W.end * kWarpSchedWarps, c->stream>>>(sp, (int)wcap);
+            SP_CUDA(c, cudaFuncSetAttribute(k_sched_warp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)wsmem));
+            k_sched_warp<<<wgrid, kWarpSchedWarps * 32, wsmem, c->stream>>>(sp, (int)wcap);
             SP_TRY(launched(c, "k_sched_warp"));
             sp.only_unstarted = 1;
         }

@@ -20,7 +20,8 @@ namespace sp {
 
 struct InstState {
     int64_t T, next_order, Tref, inserted;   // inserted: requests of the instance that have joined a queue
-    int32_t L, round, exp_since, started;
+    int32_t L, round, exp_since, started;   // started: 0 fresh, 1 running, 2 handed over by k_sched_warp within this call
+    int32_t handed, pad_;                    // rounds of this call done before the hand-over
     int32_t head[kMaxApps], tail[kMaxApps], cur[kMaxApps];   // queue positions relative to the region start
 };
 
@@ -260,7 +261,7 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
         if (tid == 0 && sp.n_done) sp.n_done[inst] = 0;
         return;
     }
-    if (sp.only_unstarted && (!sp.flags[2] || sp.state[inst].started)) return;   // the warp kernel has done it
+    if (sp.only_unstarted && (!sp.flags[2] || sp.state[inst].started == 1)) return;   // the warp kernel has done it
     const int64_t r0 = tb.gstart[(int64_t)inst * A], r1 = tb.gstart[(int64_t)(inst + 1) * A];
     const int64_t n_inst = r1 - r0;
     if (tid == 0) st = sp.state[inst];
@@ -270,7 +271,11 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
     const int64_t *al = P.lat_alpha + (int64_t)inst * P.sumM;
     const int64_t *be = P.lat_beta + (int64_t)inst * P.sumM;
     const int64_t *sw = P.swap + (int64_t)inst * P.sumM;
-    int rounds_done = 0;
+    const int rounds_init = st.started == 2 ? st.handed : 0;   // rounds k_sched_warp ran in this call before handing over
+    int rounds_done = rounds_init;
+    __syncthreads();
+    if (tid == 0 && st.started == 2) st.started = 1;
+    __syncthreads();
     unsigned long long n_exact_u = 0, n_exact_p = 0;
     const int64_t max_iter = (int64_t)sp.max_rounds + 2 * n_inst + 8;
     bool finished = false;
@@ -569,7 +574,7 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
         if (!finished && rounds_done < sp.max_rounds) dev_error(&sp.flags[0], kDevLimit);
         sp.state[inst] = st;
         if (sp.n_done) sp.n_done[inst] = rounds_done;
-        if (rounds_done) atomicAdd(&sp.stats[0], (unsigned long long)rounds_done);
+        if (rounds_done > rounds_init) atomicAdd(&sp.stats[0], (unsigned long long)(rounds_done - rounds_init));
         if (n_exact_u) atomicAdd(&sp.stats[1], n_exact_u);
         if (n_exact_p) atomicAdd(&sp.stats[2], n_exact_p);
     }
