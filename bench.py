@@ -250,7 +250,7 @@ def main():
         tj = json.load(open(tpath)).get(args.workload)
         if tj and tj.get("kernel_version") == KERNEL_VERSION:
             traffic = tj["dram_bytes_per_request"] * n
-    roofline = {"bound": "hbm", "kernel": ("k_score_tiled", "k_score_small", "k_score_mma")[int(st.get("score_kernel", 0))], "achieved": achieved,
+    roofline = {"bound": "hbm", "kernel": ("k_score_tiled", "k_score_small", "k_score_mma", "k_score_gemm_bf16")[int(st.get("score_kernel", 0))], "achieved": achieved,
                 "peak": peak, "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak if achieved else None,
                 "traffic": traffic, "algorithmic_bytes": bytes_per_launch, "kernel_ms": score_ms}
 

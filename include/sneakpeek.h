@@ -109,7 +109,8 @@ typedef struct {
      * calls since the previous sp_get_stats() (at most 512 calls are kept), and the number of calls summed. */
     int64_t score_calls, sched_calls;
     double score_kernel_ms, sched_kernel_ms;
-    /* Scoring kernel the loaded profiles select: 0 = tiled FP32, 1 = small-head FP32, 2 = tensor-core (tcgen05). */
+    /* Scoring kernel the loaded profiles select: 0 = tiled FP32, 1 = small-head FP32, 2 = tensor-core small heads
+     * (tcgen05, tf32 split), 3 = tensor-core bf16 GEMM (tcgen05). */
     int32_t score_kernel, pad_;
 } sp_stats;
 

@@ -11,6 +11,7 @@
 #include "sp_score_small.cuh"
 #include "sp_score_tiled.cuh"
 #include "sp_score_mma.cuh"
+#include "sp_score_gemm.cuh"
 #include "sp_sched.cuh"
 #include "sp_sched_warp.cuh"
 
@@ -46,11 +47,14 @@ struct sp_ctx {
     int small_ct = 0;            // labels per lane of the small-head kernel, 0 = use the tiled kernel
     size_t small_smem = 0;
     int mma_ct = 0;              // logit columns per epilogue thread of the tensor-core kernel, 0 = not used
+    bool gemm_bf16 = false;      // the bf16 GEMM-shaped tensor-core kernel scores this context's requests
+    int gemm_cp = 0;             // labels per head in the transposed image
+    CUtensorMap wt_map, r_map, b_map;
     int n_sms = 1;
     // profile buffers
     Buf W, bias, recall, prior, prior_dot, prior_sum, lat_alpha, lat_beta, swap;
     // per-instance state and scratch
-    Buf state, zbuf, flags, stats, cnt, gstart, cursor, small_start, tiled_start, small_tiles, scan_partial;
+    Buf state, zbuf, flags, stats, cnt, gstart, cursor, small_start, tiled_start, small_tiles, scan_partial, wt_image, gemm_tiles, gemm_counter;
     // per-request buffers
     Buf acc32, v32, acc64, v64, exact, recs, perm, q_id0, q_id1, q_dl0, q_dl1, q_pw0, q_pw1, sort_scratch;
     // staging of sp_run_host
@@ -216,6 +220,21 @@ sp_status feature_map(sp_ctx *c, CUtensorMap *map, const void *feats, int64_t n,
     return SP_OK;
 }
 
+// Plain 2-D tensor map over a row-major matrix [rows][cols] of `esz`-byte elements, boxes of box_rows x box_cols.
+sp_status matrix_map(sp_ctx *c, CUtensorMap *map, const void *ptr, CUtensorMapDataType dt, int esz, int64_t rows, int64_t cols,
+                     int box_rows, int box_cols, CUtensorMapSwizzle swz) {
+    EncodeTiledFn enc = encode_tiled_fn();
+    if (!enc) return fail(c, SP_ECUDA, "cuTensorMapEncodeTiled is not available from this driver");
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * esz};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = enc(map, dt, 2, const_cast<void *>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(c, SP_ECUDA, "cuTensorMapEncodeTiled failed with code " + std::to_string((int)r));
+    return SP_OK;
+}
+
 template <int CT>
 sp_status launch_mma(sp_ctx *c, const CUtensorMap &map, const mma::Params &prm) {
     auto kern = mma::k_score_mma<CT>;
@@ -260,7 +279,7 @@ void sp_destroy(sp_ctx *c) {
     drain_events(c->ev_sched, &dummy);
     Buf *all[] = {&c->W, &c->bias, &c->recall, &c->prior, &c->prior_dot, &c->prior_sum, &c->lat_alpha, &c->lat_beta,
                   &c->swap, &c->state, &c->zbuf, &c->flags, &c->stats, &c->cnt, &c->gstart, &c->cursor,
-                  &c->small_start, &c->tiled_start, &c->small_tiles, &c->scan_partial, &c->acc32, &c->v32, &c->acc64, &c->v64, &c->exact, &c->recs,
+                  &c->small_start, &c->tiled_start, &c->small_tiles, &c->scan_partial, &c->wt_image, &c->gemm_tiles, &c->gemm_counter, &c->acc32, &c->v32, &c->acc64, &c->v64, &c->exact, &c->recs,
                   &c->perm, &c->q_id0, &c->q_id1, &c->q_dl0, &c->q_dl1, &c->q_pw0, &c->q_pw1, &c->sort_scratch,
                   &c->h_feats, &c->h_app, &c->h_arrival, &c->h_deadline, &c->h_instance, &c->h_t0, &c->h_loaded,
                   &c->h_rounds, &c->h_ndone};
@@ -371,7 +390,29 @@ sp_status sp_load_profiles(sp_ctx *c, const sp_profiles *p) {
     c->sched_threads = I > 1 ? 128 : 1024;
     c->small_ct = 0;
     c->mma_ct = 0;
-    if (p->feat_dtype == SP_F32 && D % 4 == 0 && D <= mma::kMaxD && A * C <= mma::kCols && sumM * ((C + 3) & ~3) <= 1024) {
+    c->gemm_bf16 = false;
+    if (p->feat_dtype == SP_BF16 && D % 8 == 0 && C % 4 == 0 && C >= 32 && (int64_t)I * A * ((C + 15) & ~15) < (1 << 30)) {
+        // GEMM-shaped head: transpose it once into the K-major image the tensor-core kernel streams from
+        const int Cp = (C + 15) & ~15;
+        const int64_t heads = (int64_t)I * A;
+        SP_TRY(ensure(c, c->wt_image, (size_t)heads * Cp * D * 2));
+        const dim3 tg((unsigned)((Cp + 31) / 32), (unsigned)((D + 31) / 32), (unsigned)heads);
+        if (heads <= 65535) {
+            gemm::k_transpose_head_bf16<<<tg, 256, 0, c->stream>>>((const unsigned short *)c->W.p, (unsigned short *)c->wt_image.p,
+                                                                   heads, D, C, Cp);
+            SP_TRY(launched(c, "k_transpose_head_bf16"));
+            SP_TRY(matrix_map(c, &c->wt_map, c->wt_image.p, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads * Cp, D, gemm::kNC, gemm::kKSlab,
+                              CU_TENSOR_MAP_SWIZZLE_128B));
+            SP_TRY(matrix_map(c, &c->r_map, c->recall.p, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, (int64_t)I * sumM, C, kMaxModelsPerApp,
+                              gemm::kNC, CU_TENSOR_MAP_SWIZZLE_NONE));
+            SP_TRY(matrix_map(c, &c->b_map, c->bias.p, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, heads, C, 1, gemm::kNC,
+                              CU_TENSOR_MAP_SWIZZLE_NONE));
+            c->gemm_bf16 = true;
+            c->gemm_cp = Cp;
+        }
+    }
+    if (c->gemm_bf16) {
+    } else if (p->feat_dtype == SP_F32 && D % 4 == 0 && D <= mma::kMaxD && A * C <= mma::kCols && sumM * ((C + 3) & ~3) <= 1024) {
         c->mma_ct = C <= 8 ? 8 : C <= 16 ? 16 : C <= 24 ? 24 : C <= 32 ? 32 : C <= 48 ? 48 : 64;
     } else if (p->feat_dtype == SP_F32 && D % 4 == 0 && C <= 64) {
         const int ct = small_ct_for(C);
@@ -512,6 +553,20 @@ sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, 
                                                                      (int4 *)c->small_tiles.p, (const int *)c->flags.p);
             SP_TRY(launched(c, "k_small_tiles"));
         }
+        int n_tiles = 0;
+        if (c->gemm_bf16) {
+            k_group_scatter<<<gb, 256, 0, c->stream>>>(P, tb, (const int *)c->flags.p);
+            SP_TRY(launched(c, "k_group_scatter"));
+            if (n / gemm::kGRows + (int64_t)nkeys > 0x3fffffff) return fail(c, SP_EINVAL, "too many requests for one call");
+            n_tiles = (int)(n / gemm::kGRows + (int64_t)nkeys);
+            SP_TRY(ensure(c, c->gemm_tiles, (size_t)n_tiles * sizeof(int4)));
+            SP_TRY(ensure(c, c->gemm_counter, 16));
+            SP_CUDA(c, cudaMemsetAsync(c->gemm_tiles.p, 0xFF, (size_t)n_tiles * sizeof(int4), c->stream));
+            SP_CUDA(c, cudaMemsetAsync(c->gemm_counter.p, 0, 16, c->stream));
+            gemm::k_gemm_tiles<<<(unsigned)((nkeys + 255) / 256), 256, 0, c->stream>>>((int)nkeys, tb.cnt, tb.gstart, (int4 *)c->gemm_tiles.p,
+                                                                                    (int *)c->gemm_counter.p, (const int *)c->flags.p);
+            SP_TRY(launched(c, "k_gemm_tiles"));
+        }
         CUtensorMap x_map;
         if (c->mma_ct) SP_TRY(feature_map(c, &x_map, feats, n, P.D));
         SP_TRY(mark(c, c->ev_score));
@@ -532,6 +587,12 @@ sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, 
                 case 16: SP_TRY(launch_small<16>(c, grid, acc_out)); break;
                 default: SP_TRY(launch_small<32>(c, grid, acc_out)); break;
             }
+        } else if (c->gemm_bf16) {
+            gemm::GParams gp{P, tb, (const int4 *)c->gemm_tiles.p, n_tiles, c->gemm_cp, acc_out, (int *)c->flags.p};
+            SP_CUDA(c, cudaFuncSetAttribute(gemm::k_score_gemm_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::GSmem::bytes));
+            gemm::k_score_gemm_bf16<<<n_tiles < c->n_sms ? n_tiles : c->n_sms, gemm::kGThreads, gemm::GSmem::bytes, c->stream>>>(
+                c->wt_map, c->r_map, c->b_map, gp);
+            SP_TRY(launched(c, "k_score_gemm_bf16"));
         } else {
             k_group_scatter<<<gb, 256, 0, c->stream>>>(P, tb, (const int *)c->flags.p);
             SP_TRY(launched(c, "k_group_scatter"));
@@ -642,7 +703,7 @@ sp_status sp_get_stats(sp_ctx *c, sp_stats *out) {
     out->exact_rows = (int64_t)s[3];
     out->score_kernel_ms = drain_events(c->ev_score, &out->score_calls);
     out->sched_kernel_ms = drain_events(c->ev_sched, &out->sched_calls);
-    out->score_kernel = c->mma_ct ? 2 : c->small_ct ? 1 : 0;
+    out->score_kernel = c->gemm_bf16 ? 3 : c->mma_ct ? 2 : c->small_ct ? 1 : 0;
     out->pad_ = 0;
     return SP_OK;
 }

@@ -1,0 +1,416 @@
+// Tensor-core scoring kernel for large heads with bf16 features and weights (the head is a real GEMM:
+// thousands of requests x hundreds of labels x D up to thousands).
+//
+// Per request (Section 4.1 + Eq. 9 + Eq. 12 of the paper):
+//   z = x W_a + b_a;  p = softmax(z);  theta = Dirichlet posterior mean;  acc_j = sum_c theta_c recall_j(c);
+//   v = 1 + population variance_j(acc_j).
+// Shape of the computation: a tile is 128 requests of one (instance, application) group (gathered through the
+// grouping permutation), the labels are swept in chunks of 256 logit columns, and for every chunk the logits
+// Z[128 x 256] = X[128 x D] W^T[256 x D]^T accumulate over 64-feature slabs in tensor memory (tcgen05 bf16 MMAs,
+// both operands K-major with 128-byte swizzle in shared memory).  Neither logits nor posterior leave the SM:
+// epilogue warps read each finished chunk from tensor memory and fold it into an online softmax (running max,
+// running sum) with the recall contraction fused (running sum of 2^z * recall_j), flash-attention style; the two
+// accumulators alternate so the epilogue of a chunk overlaps the MMAs of the next one.
+//   * A operand: requests of a group are not contiguous, so 4 producer warps gather their rows with 16-byte
+//     cp.async copies into the swizzled slab (thread = row).
+//   * B operand: the head is transposed once, when the profiles are loaded, into a K-major image
+//     Wt[(instance, application, label)][feature]; TMA tiles of 256 labels x 64 features stream from it (L2
+//     resident).  The chunk's recall rows and bias arrive by TMA as well.
+//   * Epilogue: 2 groups of 4 warps split the 256 columns of a chunk; each keeps its own running state for the
+//     row and the two are merged at the end of the tile.
+// Every wait on an mbarrier is bounded; when one runs out the block raises kDevLimit and leaves.
+#pragma once
+
+#include <cuda.h>
+
+#include "sp_common.cuh"
+#include "sp_score_mma.cuh"   // mbarrier / TMA / tcgen05 helpers
+
+namespace sp {
+namespace gemm {
+
+using namespace sp::mma;
+
+constexpr int kGRows = 128;                 // requests per tile = MMA M
+constexpr int kNC = 256;                    // logit columns per chunk = MMA N
+constexpr int kKSlab = 64;                  // bf16 features per slab row (128 bytes)
+constexpr int kASlabBytes = kGRows * 128;   // 16 KB
+constexpr int kBSlabBytes = kNC * 128;      // 32 KB
+constexpr int kStageBytes = kASlabBytes + kBSlabBytes;
+constexpr int kGStages = 3;
+constexpr int kRBytes = kMaxModelsPerApp * kNC * 4;   // recall rows of a chunk: 16 models x 256 labels fp32
+constexpr int kBiasBytes = kNC * 4;
+constexpr int kGBProducerWarp = 0, kGMmaWarp = 1, kGAWarp0 = 2, kGEpiWarp0 = 6;
+constexpr int kGThreads = 32 * 14;
+constexpr int kGAThreads = 128, kGEpiThreads = 256;
+constexpr int kMergeFloats = 2 + kMaxModelsPerApp;    // running max, running sum, running sums per model
+
+struct GSmem {                               // byte offsets from the 1024-byte aligned base
+    static constexpr int stages = 0;                                      // [kGStages][A slab | B slab]
+    static constexpr int rtab = stages + kGStages * kStageBytes;          // [2][16][256] floats
+    static constexpr int bias = rtab + 2 * kRBytes;                       // [2][256] floats
+    static constexpr int merge = bias + 2 * kBiasBytes;                   // [128][kMergeFloats]
+    static constexpr int bars = merge + kGRows * kMergeFloats * 4;
+    static constexpr int n_bars = 3 * kGStages + 8 + 3;
+    static constexpr int misc = bars + n_bars * 8;
+    static constexpr int end = misc + 16;
+    static constexpr int bytes = end + 1024;
+};
+__device__ __forceinline__ constexpr int gbar_full_a(int s) { return s; }
+__device__ __forceinline__ constexpr int gbar_full_b(int s) { return kGStages + s; }
+__device__ __forceinline__ constexpr int gbar_free(int s) { return 2 * kGStages + s; }
+__device__ __forceinline__ constexpr int gbar_acc_full(int b) { return 3 * kGStages + b; }
+__device__ __forceinline__ constexpr int gbar_acc_empty(int b) { return 3 * kGStages + 2 + b; }
+__device__ __forceinline__ constexpr int gbar_r_full(int b) { return 3 * kGStages + 4 + b; }
+__device__ __forceinline__ constexpr int gbar_r_free(int b) { return 3 * kGStages + 6 + b; }
+constexpr int kGBarMergeReady = 3 * kGStages + 8;
+constexpr int kGBarMergeDone = 3 * kGStages + 9;
+constexpr int kGBarDrain = 3 * kGStages + 10;
+
+struct GParams {
+    DevProfiles P;
+    DevTable tb;
+    const int4 *tiles;       // (key = instance * A + application, first position in perm, rows, -); key -1 = unused entry
+    int n_tiles;
+    int Cp;                  // labels per application in the transposed head image (C rounded up to 16)
+    float *acc_out;
+    int *flags;
+};
+
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
+__host__ __device__ constexpr uint32_t instr_desc_bf16(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kGRows >> 4) << 24);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n.reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(acc)
+        : "memory");
+}
+// 16-byte async copy that reads only src_bytes (0..16) from global memory and fills the rest with zeros.
+__device__ __forceinline__ void cp_async16_zfill(uint32_t dst, const void *src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Transposes the heads into the K-major image Wt[(i * A + a) * Cp + c][d] (bf16 bit patterns), labels c >= C zero.
+__global__ void k_transpose_head_bf16(const unsigned short *__restrict__ W, unsigned short *__restrict__ Wt, int64_t n_heads,
+                                      int D, int C, int Cp) {
+    __shared__ unsigned short tile[32][33];
+    const int64_t head = blockIdx.z;
+    const int d0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;          // 32 x 8 threads
+    for (int r = ty; r < 32; r += 8) {
+        const int d = d0 + r, c = c0 + tx;
+        tile[r][tx] = (d < D && c < C) ? W[(head * D + d) * C + c] : (unsigned short)0;
+    }
+    __syncthreads();
+    for (int r = ty; r < 32; r += 8) {
+        const int c = c0 + r, d = d0 + tx;
+        if (c < Cp && d < D) Wt[(head * Cp + c) * D + d] = tile[tx][r];
+    }
+}
+
+// Tile table: every (instance, application) group is cut into tiles of 128 requests; the order of the entries is
+// arbitrary (slots are handed out by an atomic counter), unused entries keep key -1.
+__global__ void k_gemm_tiles(int n_keys, const int32_t *__restrict__ cnt, const int64_t *__restrict__ gstart,
+                             int4 *__restrict__ tiles, int *__restrict__ counter, const int *__restrict__ flags) {
+    const int key = blockIdx.x * blockDim.x + threadIdx.x;
+    if (key >= n_keys || flags[1]) return;
+    const int n = cnt[key];
+    if (n <= 0) return;
+    const int nt = (n + kGRows - 1) / kGRows;
+    const int base = atomicAdd(counter, nt);
+    for (int i = 0; i < nt; ++i) {
+        const int rows = n - i * kGRows < kGRows ? n - i * kGRows : kGRows;
+        tiles[base + i] = make_int4(key, (int)(gstart[key] + (int64_t)i * kGRows), rows, 0);
+    }
+}
+
+__global__ void __launch_bounds__(kGThreads, 1)
+k_score_gemm_bf16(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__ CUtensorMap r_map,
+                  const __grid_constant__ CUtensorMap b_map, const GParams prm) {
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw_u32 = smem_u32(smem_raw);
+    const uint32_t base = (raw_u32 + 1023u) & ~1023u;
+    unsigned char *sm = smem_raw + (base - raw_u32);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(sm + GSmem::misc);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(sm + GSmem::misc + 4);
+    auto bar = [&](int i) -> uint32_t { return base + GSmem::bars + 8u * (uint32_t)i; };
+
+    const DevProfiles &P = prm.P;
+    const DevTable &tb = prm.tb;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int A = P.A, C = P.C, D = P.D, Cp = prm.Cp;
+    const int n_ks = (D + kKSlab - 1) / kKSlab;            // feature slabs
+    const int n_ch = (C + kNC - 1) / kNC;                  // label chunks
+
+    if (tid == 0) {
+        for (int s = 0; s < kGStages; ++s) {
+            mbar_init(bar(gbar_full_a(s)), kGAThreads); mbar_init(bar(gbar_full_b(s)), 1); mbar_init(bar(gbar_free(s)), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar(gbar_acc_full(b)), 1); mbar_init(bar(gbar_acc_empty(b)), kGEpiThreads);
+            mbar_init(bar(gbar_r_full(b)), 1); mbar_init(bar(gbar_r_free(b)), kGEpiThreads);
+        }
+        mbar_init(bar(kGBarMergeReady), kGEpiThreads / 2);
+        mbar_init(bar(kGBarMergeDone), kGEpiThreads / 2);
+        mbar_init(bar(kGBarDrain), 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kGMmaWarp) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+    if (tmem != 0 && tid == 0) *abort_flag = 1;                // cannot happen for a whole-memory allocation
+    __syncthreads();
+    const bool tmem_ok = *abort_flag == 0;
+
+    if (!tmem_ok) {
+        // unexpected tensor-memory base: nothing runs, the block reports the error below
+    } else if (warp == kGBProducerWarp) {
+        // ================================================================ TMA producer of W^T slabs, recall rows, bias
+        if (lane == 0) {
+            uint32_t slab_seq = 0, chunk_seq = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < prm.n_tiles && ok; t += gridDim.x) {
+                const int4 d = prm.tiles[t];
+                if (d.x < 0) continue;
+                const int inst = d.x / A, a = d.x - inst * A;
+                const int wrow0 = d.x * Cp;                              // first row of this head in the image
+                for (int ch = 0; ch < n_ch && ok; ++ch, ++chunk_seq) {
+                    const int rb = chunk_seq & 1;
+                    const uint32_t ruse = chunk_seq >> 1;
+                    if (ruse > 0 && !mbar_wait(bar(gbar_r_free(rb)), (ruse - 1) & 1, abort_flag)) { ok = false; break; }
+                    mbar_arrive_expect_tx(bar(gbar_r_full(rb)), kRBytes + kBiasBytes);
+                    tma_load_2d(base + GSmem::rtab + rb * kRBytes, &r_map, ch * kNC, inst * P.sumM + P.mfirst[a], bar(gbar_r_full(rb)));
+                    tma_load_2d(base + GSmem::bias + rb * kBiasBytes, &b_map, ch * kNC, d.x, bar(gbar_r_full(rb)));
+                    for (int ks = 0; ks < n_ks; ++ks, ++slab_seq) {
+                        const int s = slab_seq % kGStages;
+                        const uint32_t use = slab_seq / kGStages;
+                        if (use > 0 && !mbar_wait(bar(gbar_free(s)), (use - 1) & 1, abort_flag)) { ok = false; break; }
+                        mbar_arrive_expect_tx(bar(gbar_full_b(s)), kBSlabBytes);
+                        tma_load_2d(base + GSmem::stages + s * kStageBytes + kASlabBytes, &wt_map, ks * kKSlab, wrow0 + ch * kNC,
+                                    bar(gbar_full_b(s)));
+                    }
+                }
+            }
+        }
+    } else if (warp == kGMmaWarp) {
+        // ================================================================ MMA issuer (one thread)
+        if (lane == 0) {
+            uint32_t slab_seq = 0, chunk_seq = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < prm.n_tiles && ok; t += gridDim.x) {
+                const int4 d = prm.tiles[t];
+                if (d.x < 0) continue;
+                for (int ch = 0; ch < n_ch && ok; ++ch, ++chunk_seq) {
+                    const uint32_t b = chunk_seq & 1, acc_use = chunk_seq >> 1;
+                    if (acc_use > 0 && !mbar_wait(bar(gbar_acc_empty(b)), (acc_use - 1) & 1, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const int ncols = min(kNC, ((C - ch * kNC) + 15) & ~15);
+                    const uint32_t idesc = instr_desc_bf16(ncols);
+                    const uint32_t d_tmem = b * kNC;
+                    for (int ks = 0; ks < n_ks; ++ks, ++slab_seq) {
+                        const int s = slab_seq % kGStages;
+                        const uint32_t par = (slab_seq / kGStages) & 1;
+                        if (!mbar_wait(bar(gbar_full_a(s)), par, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(bar(gbar_full_b(s)), par, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        const uint64_t a_desc = smem_desc(base + GSmem::stages + s * kStageBytes);
+                        const uint64_t b_desc = smem_desc(base + GSmem::stages + s * kStageBytes + kASlabBytes);
+#pragma unroll
+                        for (int k = 0; k < kKSlab / 16; ++k)
+                            umma_bf16(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 2), idesc, (ks | k) != 0);
+                        umma_commit(bar(gbar_free(s)));
+                    }
+                    if (ok) umma_commit(bar(gbar_acc_full(b)));
+                }
+            }
+            if (*abort_flag) {                                 // leaving early: let the issued MMAs finish first
+                umma_commit(bar(kGBarDrain));
+                const unsigned long long t0 = global_ns();
+                while (!mbar_try_wait(bar(kGBarDrain), 0) && global_ns() - t0 < kWaitLimitNs) {}
+            }
+        }
+    } else if (warp < kGEpiWarp0) {
+        // ================================================================ A producers: gather the rows of the tile
+        const int row = tid - kGAWarp0 * 32;                   // 0..127
+        uint32_t slab_seq = 0;
+        bool ok = true;
+        int pending = -1;                                      // stage whose copies are issued but not signalled
+        for (int t = blockIdx.x; t < prm.n_tiles && ok; t += gridDim.x) {
+            const int4 d = prm.tiles[t];
+            if (d.x < 0) continue;
+            const int64_t req = tb.perm[d.y + (row < d.z ? row : 0)];
+            const unsigned short *src = (const unsigned short *)tb.feats + req * D;
+            for (int ch = 0; ch < n_ch && ok; ++ch) {
+                for (int ks = 0; ks < n_ks; ++ks, ++slab_seq) {
+                    const int s = slab_seq % kGStages;
+                    const uint32_t use = slab_seq / kGStages;
+                    if (use > 0 && !warp_wait(bar(gbar_free(s)), (use - 1) & 1, abort_flag)) { ok = false; break; }
+                    const uint32_t dst = base + GSmem::stages + s * kStageBytes + row * 128;
+                    const int k0 = ks * kKSlab;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int kk = k0 + j * 8;
+                        const int left = (D - kk) * 2;         // bytes of the row that exist from this piece on
+                        cp_async16_zfill(dst + ((j ^ (row & 7)) << 4), src + (kk < D ? kk : 0), left >= 16 ? 16u : left > 0 ? (uint32_t)left : 0u);
+                    }
+                    cp_async_commit();
+                    if (pending >= 0) {                        // the copies of the previous slab have landed by now
+                        cp_async_wait<1>();
+                        fence_proxy_async();
+                        mbar_arrive(bar(gbar_full_a(pending)));
+                    }
+                    pending = s;
+                }
+            }
+        }
+        cp_async_wait<0>();
+        if (pending >= 0 && ok) {
+            fence_proxy_async();
+            mbar_arrive(bar(gbar_full_a(pending)));
+        }
+    } else {
+        // ================================================================ epilogue warps (one row per thread, half the columns)
+        const int eg = (warp - kGEpiWarp0) >> 2;               // column half of every chunk this group reads
+        const int quad = warp & 3, row = quad * 32 + lane;
+        const float *rtab = reinterpret_cast<const float *>(sm + GSmem::rtab);
+        const float *btab = reinterpret_cast<const float *>(sm + GSmem::bias);
+        float *merge = reinterpret_cast<float *>(sm + GSmem::merge) + row * kMergeFloats;
+        uint32_t chunk_seq = 0, tile_seq = 0;
+        const int Mmax = P.Mmax;
+        bool ok = true;
+        for (int t = blockIdx.x; t < prm.n_tiles && ok; t += gridDim.x) {
+            const int4 d = prm.tiles[t];
+            if (d.x < 0) continue;
+            const int inst = d.x / A, a = d.x - inst * A;
+            const int g0 = P.mfirst[a], M = P.mfirst[a + 1] - g0;
+            float run_m = -INFINITY, run_s = 0.f, racc[kMaxModelsPerApp];
+#pragma unroll
+            for (int j = 0; j < kMaxModelsPerApp; ++j) racc[j] = 0.f;
+            for (int ch = 0; ch < n_ch && ok; ++ch, ++chunk_seq) {
+                const uint32_t b = chunk_seq & 1, par = (chunk_seq >> 1) & 1;
+                if (!warp_wait(bar(gbar_r_full(b)), par, abort_flag)) { ok = false; break; }
+                if (!warp_wait(bar(gbar_acc_full(b)), par, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const float *rt = rtab + b * (kRBytes / 4), *bt = btab + b * kNC;
+                const int c_base = ch * kNC;
+                for (int sb = 0; sb < 4; ++sb) {
+                    const int col0 = eg * 128 + sb * 32;                   // column of the chunk
+                    if (c_base + col0 >= C) break;                         // uniform: nothing valid from here on
+                    float z[32];
+                    tmem_ld<32>(((uint32_t)(quad * 32) << 16) + b * kNC + col0, z);
+                    tmem_wait_ld();
+                    float bm = -INFINITY;
+#pragma unroll
+                    for (int c = 0; c < 32; c += 4) {
+                        const float4 bv = *reinterpret_cast<const float4 *>(bt + col0 + c);
+                        z[c] = (z[c] + bv.x) * kLog2e; z[c + 1] = (z[c + 1] + bv.y) * kLog2e;
+                        z[c + 2] = (z[c + 2] + bv.z) * kLog2e; z[c + 3] = (z[c + 3] + bv.w) * kLog2e;
+                    }
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        if (c_base + col0 + c >= C) z[c] = -INFINITY;
+                        bm = fmaxf(bm, z[c]);
+                    }
+                    if (bm > run_m) {                                      // rescale what has been summed so far
+                        const float sc = exp2_unit(run_m - bm);            // 0 for the first block (run_m = -inf)
+                        run_s *= sc;
+#pragma unroll
+                        for (int j = 0; j < kMaxModelsPerApp; ++j) racc[j] *= sc;
+                        run_m = bm;
+                    }
+                    float ps = 0.f;
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) { z[c] = exp2_unit(z[c] - run_m); ps += z[c]; }
+                    run_s += ps;
+#pragma unroll
+                    for (int j = 0; j < kMaxModelsPerApp; ++j) {
+                        if (j < M) {
+                            const float *rr = rt + j * kNC + col0;
+                            float p0 = 0.f, p1 = 0.f;
+#pragma unroll
+                            for (int c = 0; c < 32; c += 4) {
+                                const float4 rv = *reinterpret_cast<const float4 *>(rr + c);
+                                p0 = fmaf(z[c], rv.x, p0); p1 = fmaf(z[c + 1], rv.y, p1);
+                                p0 = fmaf(z[c + 2], rv.z, p0); p1 = fmaf(z[c + 3], rv.w, p1);
+                            }
+                            racc[j] += p0 + p1;
+                        }
+                    }
+                }
+                tc_fence_before();
+                mbar_arrive(bar(gbar_acc_empty(b)));
+                mbar_arrive(bar(gbar_r_free(b)));
+            }
+            if (!ok) break;
+            // ---- merge the two column halves of the row, finish Eq. 9 / Eq. 12, store
+            if (eg == 1) {
+                if (tile_seq > 0 && !warp_wait(bar(kGBarMergeDone), (tile_seq - 1) & 1, abort_flag)) break;
+                merge[0] = run_m; merge[1] = run_s;
+#pragma unroll
+                for (int j = 0; j < kMaxModelsPerApp; ++j) merge[2 + j] = racc[j];
+                mbar_arrive(bar(kGBarMergeReady));
+            } else {
+                if (!warp_wait(bar(kGBarMergeReady), tile_seq & 1, abort_flag)) break;
+                const float om = merge[0], os = merge[1];
+                const float mm = fmaxf(run_m, om);
+                const float s0 = run_m == -INFINITY ? 0.f : exp2_unit(run_m - mm);
+                const float s1 = om == -INFINITY ? 0.f : exp2_unit(om - mm);
+                const float inv = 1.f / (run_s * s0 + os * s1);
+                const bool valid = row < d.z;
+                const int64_t req = tb.perm[d.y + (valid ? row : 0)];
+                float *dst = tb.acc32 + req * Mmax;
+                float *dst2 = prm.acc_out ? prm.acc_out + req * Mmax : nullptr;
+                float a0 = 0.f, q1 = 0.f, q2 = 0.f;
+#pragma unroll
+                for (int j = 0; j < kMaxModelsPerApp; ++j) {
+                    if (j < Mmax) {
+                        float aj = 0.f;
+                        if (j < M) {
+                            aj = (racc[j] * s0 + merge[2 + j] * s1) * inv;
+                            if (P.prior)
+                                aj = (P.prior_dot[(int64_t)inst * P.sumM + g0 + j] + P.kappa * aj) / (P.prior_sum[d.x] + P.kappa);
+                            if (j == 0) a0 = aj;
+                            const float dj = aj - a0;
+                            q1 += dj; q2 = fmaf(dj, dj, q2);
+                        }
+                        if (valid) {
+                            dst[j] = aj;
+                            if (dst2) dst2[j] = aj;
+                        }
+                    }
+                }
+                if (valid) {
+                    const float invM = 1.f / (float)M, md = q1 * invM;
+                    tb.v32[req] = 1.f + fmaxf(fmaf(q2, invM, -md * md), 0.f);
+                }
+                mbar_arrive(bar(kGBarMergeDone));
+            }
+            ++tile_seq;
+        }
+    }
+
+    // ---- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (tid == 0 && *abort_flag) dev_error(&prm.flags[0], kDevLimit);
+    if (warp == kGMmaWarp) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+    }
+}
+
+}  // namespace gemm
+}  // namespace sp
