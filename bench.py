@@ -239,7 +239,7 @@ def main():
     # ---- roofline of the dominant kernel (the scoring kernel), from CUDA events recorded around it
     score_ms = st["score_kernel_ms"] / max(1, st["score_calls"])
     sched_ms = st["sched_kernel_ms"] / max(1, st["sched_calls"])
-    kernel = ("k_score_tiled", "k_score_small", "k_score_mma", "k_score_gemm_bf16")[int(st.get("score_kernel", 0))]
+    kernel = ("k_score_tiled", "k_score_small", "k_score_mma", "k_score_gemm<bf16>", "k_score_gemm<f32>")[int(st.get("score_kernel", 0))]
     peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     peaks = json.load(open(peaks_path)) if os.path.exists(peaks_path) else None
     traffic = None
@@ -248,16 +248,21 @@ def main():
         tj = json.load(open(tpath)).get(args.workload)
         if tj and tj.get("kernel_version") == KERNEL_VERSION:
             traffic = tj["dram_bytes_per_request"] * n
-    if kernel == "k_score_gemm_bf16":
-        # the head is a dense bf16 contraction far above the HBM ridge: bound by the tensor pipe.  The kernel is
-        # short and timed by its own events, so the burst figure of the measured peak applies.
+    if kernel.startswith("k_score_gemm"):
+        # the head is a dense contraction far above the HBM ridge: bound by the tensor pipe.  The kernel is short and
+        # timed by its own events, so the burst figure of the measured bf16 peak applies; the fp32 flavour runs on the
+        # tf32 unit (nominal ratio to bf16: 0.5) and needs three MMA passes for fp32 accuracy, but the algorithmic
+        # flops (2 n D C) are what is counted.
+        f32 = kernel.endswith("<f32>")
         flops = 2.0 * n * int(w.feat_dim) * int(w.n_classes)
         peak, peak_src = (float(peaks["bf16_tflops"]), "measured") if peaks else (1590.0, "fallback")
+        if f32:
+            peak, peak_src = peak * 0.5, peak_src + " bf16 x 0.5 (tf32)"
         achieved = flops / (score_ms * 1e-3) / 1e12 if score_ms > 0 else None
         roofline = {"bound": "tensor", "kernel": kernel, "achieved": achieved, "peak": peak, "peak_source": peak_src,
                     "unit": "TFLOP/s", "frac": achieved / peak if achieved else None, "traffic": traffic,
-                    "algorithmic_flops": flops, "algorithmic_bytes": algorithmic_bytes_per_request(w) * n,
-                    "kernel_ms": score_ms}
+                    "algorithmic_flops": flops, "mma_passes": 3 if f32 else 1,
+                    "algorithmic_bytes": algorithmic_bytes_per_request(w) * n, "kernel_ms": score_ms}
     else:
         bytes_per_launch = algorithmic_bytes_per_request(w) * n
         peak, peak_src = (float(peaks["hbm_gbs"]), "measured") if peaks else (6650.0, "fallback")

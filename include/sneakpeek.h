@@ -110,7 +110,7 @@ typedef struct {
     int64_t score_calls, sched_calls;
     double score_kernel_ms, sched_kernel_ms;
     /* Scoring kernel the loaded profiles select: 0 = tiled FP32, 1 = small-head FP32, 2 = tensor-core small heads
-     * (tcgen05, tf32 split), 3 = tensor-core bf16 GEMM (tcgen05). */
+     * (tcgen05, tf32 split), 3 = tensor-core bf16 GEMM (tcgen05), 4 = tensor-core fp32 GEMM (tcgen05, tf32 split). */
     int32_t score_kernel, pad_;
 } sp_stats;
 

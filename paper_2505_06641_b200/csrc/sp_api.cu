@@ -47,7 +47,8 @@ struct sp_ctx {
     int small_ct = 0;            // labels per lane of the small-head kernel, 0 = use the tiled kernel
     size_t small_smem = 0;
     int mma_ct = 0;              // logit columns per epilogue thread of the tensor-core kernel, 0 = not used
-    bool gemm_bf16 = false;      // the bf16 GEMM-shaped tensor-core kernel scores this context's requests
+    bool gemm_on = false;      // a GEMM-shaped tensor-core kernel scores this context's requests (either flavour)
+    bool gemm_f32 = false;       // ... the fp32 (tf32 split) flavour
     int gemm_cp = 0;             // labels per head in the transposed image
     CUtensorMap wt_map, r_map, b_map;
     int n_sms = 1;
@@ -390,28 +391,39 @@ sp_status sp_load_profiles(sp_ctx *c, const sp_profiles *p) {
     c->sched_threads = I > 1 ? 128 : 1024;
     c->small_ct = 0;
     c->mma_ct = 0;
-    c->gemm_bf16 = false;
-    if (p->feat_dtype == SP_BF16 && D % 8 == 0 && C % 4 == 0 && C >= 32 && (int64_t)I * A * ((C + 15) & ~15) < (1 << 30)) {
+    c->gemm_on = false;
+    c->gemm_f32 = false;
+    const bool small_head = p->feat_dtype == SP_F32 && D % 4 == 0 && D <= mma::kMaxD && A * C <= mma::kCols && sumM * ((C + 3) & ~3) <= 1024;
+    const bool want_bf16 = p->feat_dtype == SP_BF16 && D % 8 == 0;
+    const bool want_f32 = p->feat_dtype == SP_F32 && D % 4 == 0 && !small_head;
+    if ((want_bf16 || want_f32) && C % 4 == 0 && C >= 32 && (int64_t)I * A * ((C + 15) & ~15) < (1 << 29) && (int64_t)I * A <= 65535) {
         // GEMM-shaped head: transpose it once into the K-major image the tensor-core kernel streams from
         const int Cp = (C + 15) & ~15;
         const int64_t heads = (int64_t)I * A;
-        SP_TRY(ensure(c, c->wt_image, (size_t)heads * Cp * D * 2));
         const dim3 tg((unsigned)((Cp + 31) / 32), (unsigned)((D + 31) / 32), (unsigned)heads);
-        if (heads <= 65535) {
+        if (want_bf16) {
+            SP_TRY(ensure(c, c->wt_image, (size_t)heads * Cp * D * 2));
             gemm::k_transpose_head_bf16<<<tg, 256, 0, c->stream>>>((const unsigned short *)c->W.p, (unsigned short *)c->wt_image.p,
                                                                    heads, D, C, Cp);
             SP_TRY(launched(c, "k_transpose_head_bf16"));
-            SP_TRY(matrix_map(c, &c->wt_map, c->wt_image.p, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads * Cp, D, gemm::kNC, gemm::kKSlab,
-                              CU_TENSOR_MAP_SWIZZLE_128B));
-            SP_TRY(matrix_map(c, &c->r_map, c->recall.p, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, (int64_t)I * sumM, C, kMaxModelsPerApp,
-                              gemm::kNC, CU_TENSOR_MAP_SWIZZLE_NONE));
-            SP_TRY(matrix_map(c, &c->b_map, c->bias.p, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, heads, C, 1, gemm::kNC,
-                              CU_TENSOR_MAP_SWIZZLE_NONE));
-            c->gemm_bf16 = true;
-            c->gemm_cp = Cp;
+            SP_TRY(matrix_map(c, &c->wt_map, c->wt_image.p, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, heads * Cp, D, gemm::GCfg<false>::NC,
+                              gemm::GCfg<false>::KSlab, CU_TENSOR_MAP_SWIZZLE_128B));
+        } else {
+            SP_TRY(ensure(c, c->wt_image, (size_t)2 * heads * Cp * D * 4));
+            gemm::k_transpose_head_f32<<<tg, 256, 0, c->stream>>>((const float *)c->W.p, (float *)c->wt_image.p, heads, D, C, Cp);
+            SP_TRY(launched(c, "k_transpose_head_f32"));
+            SP_TRY(matrix_map(c, &c->wt_map, c->wt_image.p, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, 2 * heads * Cp, D, gemm::GCfg<true>::NC,
+                              gemm::GCfg<true>::KSlab, CU_TENSOR_MAP_SWIZZLE_128B));
         }
+        const int nc = want_bf16 ? gemm::GCfg<false>::NC : gemm::GCfg<true>::NC;
+        SP_TRY(matrix_map(c, &c->r_map, c->recall.p, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, (int64_t)I * sumM, C, kMaxModelsPerApp, nc,
+                          CU_TENSOR_MAP_SWIZZLE_NONE));
+        SP_TRY(matrix_map(c, &c->b_map, c->bias.p, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, heads, C, 1, nc, CU_TENSOR_MAP_SWIZZLE_NONE));
+        c->gemm_on = true;
+        c->gemm_f32 = want_f32;
+        c->gemm_cp = Cp;
     }
-    if (c->gemm_bf16) {
+    if (c->gemm_on) {
     } else if (p->feat_dtype == SP_F32 && D % 4 == 0 && D <= mma::kMaxD && A * C <= mma::kCols && sumM * ((C + 3) & ~3) <= 1024) {
         c->mma_ct = C <= 8 ? 8 : C <= 16 ? 16 : C <= 24 ? 24 : C <= 32 ? 32 : C <= 48 ? 48 : 64;
     } else if (p->feat_dtype == SP_F32 && D % 4 == 0 && C <= 64) {
@@ -554,7 +566,7 @@ sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, 
             SP_TRY(launched(c, "k_small_tiles"));
         }
         int n_tiles = 0;
-        if (c->gemm_bf16) {
+        if (c->gemm_on) {
             k_group_scatter<<<gb, 256, 0, c->stream>>>(P, tb, (const int *)c->flags.p);
             SP_TRY(launched(c, "k_group_scatter"));
             if (n / gemm::kGRows + (int64_t)nkeys > 0x3fffffff) return fail(c, SP_EINVAL, "too many requests for one call");
@@ -587,12 +599,17 @@ sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, 
                 case 16: SP_TRY(launch_small<16>(c, grid, acc_out)); break;
                 default: SP_TRY(launch_small<32>(c, grid, acc_out)); break;
             }
-        } else if (c->gemm_bf16) {
-            gemm::GParams gp{P, tb, (const int4 *)c->gemm_tiles.p, n_tiles, c->gemm_cp, acc_out, (int *)c->flags.p};
-            SP_CUDA(c, cudaFuncSetAttribute(gemm::k_score_gemm_bf16, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::GSmem::bytes));
-            gemm::k_score_gemm_bf16<<<n_tiles < c->n_sms ? n_tiles : c->n_sms, gemm::kGThreads, gemm::GSmem::bytes, c->stream>>>(
-                c->wt_map, c->r_map, c->b_map, gp);
-            SP_TRY(launched(c, "k_score_gemm_bf16"));
+        } else if (c->gemm_on) {
+            gemm::GParams gp{P, tb, (const int4 *)c->gemm_tiles.p, n_tiles, c->gemm_cp, P.I * P.A * c->gemm_cp, acc_out, (int *)c->flags.p};
+            const int ggrid = n_tiles < c->n_sms ? n_tiles : c->n_sms;
+            if (c->gemm_f32) {
+                SP_CUDA(c, cudaFuncSetAttribute(gemm::k_score_gemm<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::GCfg<true>::bytes));
+                gemm::k_score_gemm<true><<<ggrid, gemm::kGThreads, gemm::GCfg<true>::bytes, c->stream>>>(c->wt_map, c->r_map, c->b_map, gp);
+            } else {
+                SP_CUDA(c, cudaFuncSetAttribute(gemm::k_score_gemm<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::GCfg<false>::bytes));
+                gemm::k_score_gemm<false><<<ggrid, gemm::kGThreads, gemm::GCfg<false>::bytes, c->stream>>>(c->wt_map, c->r_map, c->b_map, gp);
+            }
+            SP_TRY(launched(c, "k_score_gemm"));
         } else {
             k_group_scatter<<<gb, 256, 0, c->stream>>>(P, tb, (const int *)c->flags.p);
             SP_TRY(launched(c, "k_group_scatter"));
@@ -703,7 +720,7 @@ sp_status sp_get_stats(sp_ctx *c, sp_stats *out) {
     out->exact_rows = (int64_t)s[3];
     out->score_kernel_ms = drain_events(c->ev_score, &out->score_calls);
     out->sched_kernel_ms = drain_events(c->ev_sched, &out->sched_calls);
-    out->score_kernel = c->gemm_bf16 ? 3 : c->mma_ct ? 2 : c->small_ct ? 1 : 0;
+    out->score_kernel = c->gemm_f32 ? 4 : c->gemm_on ? 3 : c->mma_ct ? 2 : c->small_ct ? 1 : 0;
     out->pad_ = 0;
     return SP_OK;
 }

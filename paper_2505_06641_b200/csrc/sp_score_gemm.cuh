@@ -1,23 +1,29 @@
-// Tensor-core scoring kernel for large heads with bf16 features and weights (the head is a real GEMM:
-// thousands of requests x hundreds of labels x D up to thousands).
+// Tensor-core scoring kernel for large heads (the head is a real GEMM: thousands of requests x hundreds of
+// labels x D up to thousands), in two flavours: bf16 features and weights, and fp32 features and weights.
 //
 // Per request (Section 4.1 + Eq. 9 + Eq. 12 of the paper):
 //   z = x W_a + b_a;  p = softmax(z);  theta = Dirichlet posterior mean;  acc_j = sum_c theta_c recall_j(c);
 //   v = 1 + population variance_j(acc_j).
 // Shape of the computation: a tile is 128 requests of one (instance, application) group (gathered through the
-// grouping permutation), the labels are swept in chunks of 256 logit columns, and for every chunk the logits
-// Z[128 x 256] = X[128 x D] W^T[256 x D]^T accumulate over 64-feature slabs in tensor memory (tcgen05 bf16 MMAs,
-// both operands K-major with 128-byte swizzle in shared memory).  Neither logits nor posterior leave the SM:
-// epilogue warps read each finished chunk from tensor memory and fold it into an online softmax (running max,
-// running sum) with the recall contraction fused (running sum of 2^z * recall_j), flash-attention style; the two
-// accumulators alternate so the epilogue of a chunk overlaps the MMAs of the next one.
+// grouping permutation), the labels are swept in chunks of NC logit columns, and for every chunk the logits
+// Z[128 x NC] = X[128 x D] W^T[NC x D]^T accumulate over 128-byte feature slabs in tensor memory (tcgen05 MMAs,
+// operands K-major with 128-byte swizzle).  Neither logits nor posterior leave the SM: epilogue warps read each
+// finished chunk from tensor memory and fold it into an online softmax (running max, running sum) with the recall
+// contraction fused (running sum of 2^z * recall_j), flash-attention style; the two accumulators alternate so the
+// epilogue of a chunk overlaps the MMAs of the next one.
 //   * A operand: requests of a group are not contiguous, so 4 producer warps gather their rows with 16-byte
 //     cp.async copies into the swizzled slab (thread = row).
 //   * B operand: the head is transposed once, when the profiles are loaded, into a K-major image
-//     Wt[(instance, application, label)][feature]; TMA tiles of 256 labels x 64 features stream from it (L2
-//     resident).  The chunk's recall rows and bias arrive by TMA as well.
-//   * Epilogue: 2 groups of 4 warps split the 256 columns of a chunk; each keeps its own running state for the
-//     row and the two are merged at the end of the tile.
+//     Wt[(instance, application, label)][feature]; TMA tiles of NC labels x one slab of features stream from it
+//     (L2 resident).  The chunk's recall rows and bias arrive by TMA as well.
+//   * bf16: NC = 256, 64 features per slab, one MMA pass (bf16 products are exact in the fp32 accumulator).
+//   * fp32: NC = 208, 32 features per slab, tf32 MMAs with the split x = x_hi + x_lo, W = W_hi + W_lo (hi = value
+//     truncated to tf32, lo = exact remainder): x_hi W_hi + x_hi W_lo + x_lo W_hi, the dropped term is below 2^-20
+//     relative.  The image holds W_hi and W_lo (log2(e) folded in); x_hi is the gathered slab as it is (the unit
+//     reads the truncated value), x_lo is computed by the producer threads from their own row and stored into a
+//     32-column slot of tensor memory, from where the third MMA takes its A operand.
+//   * Epilogue: 2 groups of 4 warps split the columns of a chunk; each keeps its own running state for the row and
+//     the two are merged at the end of the tile.
 // Every wait on an mbarrier is bounded; when one runs out the block raises kDevLimit and leaves.
 #pragma once
 
@@ -32,40 +38,47 @@ namespace gemm {
 using namespace sp::mma;
 
 constexpr int kGRows = 128;                 // requests per tile = MMA M
-constexpr int kNC = 256;                    // logit columns per chunk = MMA N
-constexpr int kKSlab = 64;                  // bf16 features per slab row (128 bytes)
-constexpr int kASlabBytes = kGRows * 128;   // 16 KB
-constexpr int kBSlabBytes = kNC * 128;      // 32 KB
-constexpr int kStageBytes = kASlabBytes + kBSlabBytes;
-constexpr int kGStages = 3;
-constexpr int kRBytes = kMaxModelsPerApp * kNC * 4;   // recall rows of a chunk: 16 models x 256 labels fp32
-constexpr int kBiasBytes = kNC * 4;
+constexpr int kASlabBytes = kGRows * 128;   // 16 KB: 128 rows x 128 bytes
 constexpr int kGBProducerWarp = 0, kGMmaWarp = 1, kGAWarp0 = 2, kGEpiWarp0 = 6;
 constexpr int kGThreads = 32 * 14;
 constexpr int kGAThreads = 128, kGEpiThreads = 256;
 constexpr int kMergeFloats = 2 + kMaxModelsPerApp;    // running max, running sum, running sums per model
+constexpr int kGMaxStages = 3;
 
-struct GSmem {                               // byte offsets from the 1024-byte aligned base
-    static constexpr int stages = 0;                                      // [kGStages][A slab | B slab]
-    static constexpr int rtab = stages + kGStages * kStageBytes;          // [2][16][256] floats
-    static constexpr int bias = rtab + 2 * kRBytes;                       // [2][256] floats
-    static constexpr int merge = bias + 2 * kBiasBytes;                   // [128][kMergeFloats]
-    static constexpr int bars = merge + kGRows * kMergeFloats * 4;
-    static constexpr int n_bars = 3 * kGStages + 8 + 3;
+template <bool F32>
+struct GCfg {
+    static constexpr int NC = F32 ? 208 : 256;                 // logit columns per chunk = MMA N (2 accumulators <= 512 columns)
+    static constexpr int KSlab = F32 ? 32 : 64;                // features per slab row (128 bytes)
+    static constexpr int KStep = F32 ? 8 : 16;                 // features per MMA
+    static constexpr int BSlabBytes = NC * 128 * (F32 ? 2 : 1);   // fp32: W_hi rows, then W_lo rows
+    static constexpr int StageBytes = kASlabBytes + ((BSlabBytes + 1023) & ~1023);
+    static constexpr int Stages = F32 ? 2 : 3;
+    static constexpr int RBytes = kMaxModelsPerApp * NC * 4;   // recall rows of a chunk
+    static constexpr int BiasBytes = NC * 4;
+    static constexpr int BiasSlot = (BiasBytes + 127) & ~127;     // TMA destinations are 128-byte aligned
+    static_assert(RBytes % 128 == 0, "recall buffers must keep the 128-byte alignment of TMA destinations");
+    static constexpr int TmemLo = 2 * NC;                      // fp32: x_lo slots (32 columns per stage) after the accumulators
+    // byte offsets from the 1024-byte aligned base
+    static constexpr int stages = 0;                                          // [Stages][A slab | B slab]
+    static constexpr int rtab = stages + Stages * StageBytes;                 // [2][16][NC] floats
+    static constexpr int bias = rtab + 2 * RBytes;                            // [2][NC] floats
+    static constexpr int merge = bias + 2 * BiasSlot;                        // [128][kMergeFloats]
+    static constexpr int bars = (merge + kGRows * kMergeFloats * 4 + 15) & ~15;
+    static constexpr int n_bars = 3 * kGMaxStages + 8 + 3;
     static constexpr int misc = bars + n_bars * 8;
     static constexpr int end = misc + 16;
     static constexpr int bytes = end + 1024;
 };
 __device__ __forceinline__ constexpr int gbar_full_a(int s) { return s; }
-__device__ __forceinline__ constexpr int gbar_full_b(int s) { return kGStages + s; }
-__device__ __forceinline__ constexpr int gbar_free(int s) { return 2 * kGStages + s; }
-__device__ __forceinline__ constexpr int gbar_acc_full(int b) { return 3 * kGStages + b; }
-__device__ __forceinline__ constexpr int gbar_acc_empty(int b) { return 3 * kGStages + 2 + b; }
-__device__ __forceinline__ constexpr int gbar_r_full(int b) { return 3 * kGStages + 4 + b; }
-__device__ __forceinline__ constexpr int gbar_r_free(int b) { return 3 * kGStages + 6 + b; }
-constexpr int kGBarMergeReady = 3 * kGStages + 8;
-constexpr int kGBarMergeDone = 3 * kGStages + 9;
-constexpr int kGBarDrain = 3 * kGStages + 10;
+__device__ __forceinline__ constexpr int gbar_full_b(int s) { return kGMaxStages + s; }
+__device__ __forceinline__ constexpr int gbar_free(int s) { return 2 * kGMaxStages + s; }
+__device__ __forceinline__ constexpr int gbar_acc_full(int b) { return 3 * kGMaxStages + b; }
+__device__ __forceinline__ constexpr int gbar_acc_empty(int b) { return 3 * kGMaxStages + 2 + b; }
+__device__ __forceinline__ constexpr int gbar_r_full(int b) { return 3 * kGMaxStages + 4 + b; }
+__device__ __forceinline__ constexpr int gbar_r_free(int b) { return 3 * kGMaxStages + 6 + b; }
+constexpr int kGBarMergeReady = 3 * kGMaxStages + 8;
+constexpr int kGBarMergeDone = 3 * kGMaxStages + 9;
+constexpr int kGBarDrain = 3 * kGMaxStages + 10;
 
 struct GParams {
     DevProfiles P;
@@ -73,6 +86,7 @@ struct GParams {
     const int4 *tiles;       // (key = instance * A + application, first position in perm, rows, -); key -1 = unused entry
     int n_tiles;
     int Cp;                  // labels per application in the transposed head image (C rounded up to 16)
+    int lo_row0;             // fp32: first row of the W_lo half of the image (= number of W_hi rows)
     float *acc_out;
     int *flags;
 };
@@ -115,6 +129,28 @@ __global__ void k_transpose_head_bf16(const unsigned short *__restrict__ W, unsi
     }
 }
 
+// fp32 heads: K-major images of W * log2(e) split for the tf32 unit: rows [0, n_heads * Cp) hold the value truncated to
+// tf32, rows [n_heads * Cp, 2 n_heads * Cp) the exact remainder; labels c >= C zero.
+__global__ void k_transpose_head_f32(const float *__restrict__ W, float *__restrict__ Wt, int64_t n_heads, int D, int C, int Cp) {
+    __shared__ float tile[32][33];
+    const int64_t head = blockIdx.z;
+    const int d0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;          // 32 x 8 threads
+    for (int r = ty; r < 32; r += 8) {
+        const int d = d0 + r, c = c0 + tx;
+        tile[r][tx] = (d < D && c < C) ? W[(head * D + d) * C + c] : 0.f;
+    }
+    __syncthreads();
+    for (int r = ty; r < 32; r += 8) {
+        const int c = c0 + r, d = d0 + tx;
+        if (c < Cp && d < D) {
+            const float w = tile[tx][r] * kLog2e, hi = tf32_part(w);
+            Wt[(head * Cp + c) * D + d] = hi;
+            Wt[((n_heads + head) * Cp + c) * D + d] = w - hi;
+        }
+    }
+}
+
 // Tile table: every (instance, application) group is cut into tiles of 128 requests; the order of the entries is
 // arbitrary (slots are handed out by an atomic counter), unused entries keep key -1.
 __global__ void k_gemm_tiles(int n_keys, const int32_t *__restrict__ cnt, const int64_t *__restrict__ gstart,
@@ -131,9 +167,14 @@ __global__ void k_gemm_tiles(int n_keys, const int32_t *__restrict__ cnt, const 
     }
 }
 
+template <bool F32>
 __global__ void __launch_bounds__(kGThreads, 1)
-k_score_gemm_bf16(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__ CUtensorMap r_map,
-                  const __grid_constant__ CUtensorMap b_map, const GParams prm) {
+k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__ CUtensorMap r_map,
+             const __grid_constant__ CUtensorMap b_map, const GParams prm) {
+    using G = GCfg<F32>;
+    constexpr int kNC = G::NC, kKSlab = G::KSlab, kGStages = G::Stages, kStageBytes = G::StageBytes;
+    constexpr int kBSlabBytes = G::BSlabBytes, kRBytes = G::RBytes, kBiasBytes = G::BiasBytes;
+    using GSmem = G;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw_u32 = smem_u32(smem_raw);
     const uint32_t base = (raw_u32 + 1023u) & ~1023u;
@@ -193,14 +234,15 @@ k_score_gemm_bf16(const __grid_constant__ CUtensorMap wt_map, const __grid_const
                     if (ruse > 0 && !mbar_wait(bar(gbar_r_free(rb)), (ruse - 1) & 1, abort_flag)) { ok = false; break; }
                     mbar_arrive_expect_tx(bar(gbar_r_full(rb)), kRBytes + kBiasBytes);
                     tma_load_2d(base + GSmem::rtab + rb * kRBytes, &r_map, ch * kNC, inst * P.sumM + P.mfirst[a], bar(gbar_r_full(rb)));
-                    tma_load_2d(base + GSmem::bias + rb * kBiasBytes, &b_map, ch * kNC, d.x, bar(gbar_r_full(rb)));
+                    tma_load_2d(base + GSmem::bias + rb * G::BiasSlot, &b_map, ch * kNC, d.x, bar(gbar_r_full(rb)));
                     for (int ks = 0; ks < n_ks; ++ks, ++slab_seq) {
                         const int s = slab_seq % kGStages;
                         const uint32_t use = slab_seq / kGStages;
                         if (use > 0 && !mbar_wait(bar(gbar_free(s)), (use - 1) & 1, abort_flag)) { ok = false; break; }
                         mbar_arrive_expect_tx(bar(gbar_full_b(s)), kBSlabBytes);
-                        tma_load_2d(base + GSmem::stages + s * kStageBytes + kASlabBytes, &wt_map, ks * kKSlab, wrow0 + ch * kNC,
-                                    bar(gbar_full_b(s)));
+                        const uint32_t bdst = base + GSmem::stages + s * kStageBytes + kASlabBytes;
+                        tma_load_2d(bdst, &wt_map, ks * kKSlab, wrow0 + ch * kNC, bar(gbar_full_b(s)));
+                        if (F32) tma_load_2d(bdst + kNC * 128, &wt_map, ks * kKSlab, prm.lo_row0 + wrow0 + ch * kNC, bar(gbar_full_b(s)));
                     }
                 }
             }
@@ -218,7 +260,7 @@ k_score_gemm_bf16(const __grid_constant__ CUtensorMap wt_map, const __grid_const
                     if (acc_use > 0 && !mbar_wait(bar(gbar_acc_empty(b)), (acc_use - 1) & 1, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     const int ncols = min(kNC, ((C - ch * kNC) + 15) & ~15);
-                    const uint32_t idesc = instr_desc_bf16(ncols);
+                    const uint32_t idesc = F32 ? instr_desc(ncols) : instr_desc_bf16(ncols);
                     const uint32_t d_tmem = b * kNC;
                     for (int ks = 0; ks < n_ks; ++ks, ++slab_seq) {
                         const int s = slab_seq % kGStages;
@@ -228,9 +270,20 @@ k_score_gemm_bf16(const __grid_constant__ CUtensorMap wt_map, const __grid_const
                         tc_fence_after();
                         const uint64_t a_desc = smem_desc(base + GSmem::stages + s * kStageBytes);
                         const uint64_t b_desc = smem_desc(base + GSmem::stages + s * kStageBytes + kASlabBytes);
+                        if (F32) {
+                            const uint64_t bl_desc = b_desc + (uint64_t)((kNC * 128) >> 4);      // W_lo rows
+                            const uint32_t a_lo = (uint32_t)(G::TmemLo + s * 32);                  // x_lo of this stage
 #pragma unroll
-                        for (int k = 0; k < kKSlab / 16; ++k)
-                            umma_bf16(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 2), idesc, (ks | k) != 0);
+                            for (int k = 0; k < kKSlab / 8; ++k) {
+                                umma_tf32(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 2), idesc, (ks | k) != 0);
+                                umma_tf32(d_tmem, a_desc + (uint64_t)(k * 2), bl_desc + (uint64_t)(k * 2), idesc, 1u);
+                                umma_tf32_ts(d_tmem, a_lo + k * 8, b_desc + (uint64_t)(k * 2), idesc, 1u);
+                            }
+                        } else {
+#pragma unroll
+                            for (int k = 0; k < kKSlab / 16; ++k)
+                                umma_bf16(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 2), idesc, (ks | k) != 0);
+                        }
                         umma_commit(bar(gbar_free(s)));
                     }
                     if (ok) umma_commit(bar(gbar_acc_full(b)));
@@ -244,15 +297,40 @@ k_score_gemm_bf16(const __grid_constant__ CUtensorMap wt_map, const __grid_const
         }
     } else if (warp < kGEpiWarp0) {
         // ================================================================ A producers: gather the rows of the tile
-        const int row = tid - kGAWarp0 * 32;                   // 0..127
+        const int aquad = warp & 3, row = aquad * 32 + lane;  // fp32: the thread's row is also its tensor-memory lane
+        constexpr int kEsz = F32 ? 4 : 2, kPiece = 16 / kEsz; // bytes per feature, features per 16-byte piece
         uint32_t slab_seq = 0;
         bool ok = true;
         int pending = -1;                                      // stage whose copies are issued but not signalled
+        // The copies of stage ps have landed: (fp32) store this row's x_lo into the stage's tensor-memory slot, then
+        // tell the MMA issuer that the A operand of the stage is complete.
+        auto signal = [&](int ps) {
+            if (F32) {
+                const unsigned char *xrow = sm + GSmem::stages + ps * kStageBytes + row * 128;
+                uint32_t v[32];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const uint4 q = *reinterpret_cast<const uint4 *>(xrow + ((j ^ (row & 7)) << 4));
+                    v[4 * j] = q.x; v[4 * j + 1] = q.y; v[4 * j + 2] = q.z; v[4 * j + 3] = q.w;
+                }
+#pragma unroll
+                for (int k = 0; k < 32; ++k) {
+                    const float x = __uint_as_float(v[k]);
+                    v[k] = __float_as_uint(x - tf32_part(x));
+                }
+                tc_fence_after();
+                tmem_st32(((uint32_t)(aquad * 32) << 16) + (uint32_t)(G::TmemLo + ps * 32), v);
+                tmem_wait_st();
+                tc_fence_before();
+            }
+            fence_proxy_async();
+            mbar_arrive(bar(gbar_full_a(ps)));
+        };
         for (int t = blockIdx.x; t < prm.n_tiles && ok; t += gridDim.x) {
             const int4 d = prm.tiles[t];
             if (d.x < 0) continue;
             const int64_t req = tb.perm[d.y + (row < d.z ? row : 0)];
-            const unsigned short *src = (const unsigned short *)tb.feats + req * D;
+            const unsigned char *src = (const unsigned char *)tb.feats + req * D * kEsz;
             for (int ch = 0; ch < n_ch && ok; ++ch) {
                 for (int ks = 0; ks < n_ks; ++ks, ++slab_seq) {
                     const int s = slab_seq % kGStages;
@@ -262,25 +340,22 @@ k_score_gemm_bf16(const __grid_constant__ CUtensorMap wt_map, const __grid_const
                     const int k0 = ks * kKSlab;
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
-                        const int kk = k0 + j * 8;
-                        const int left = (D - kk) * 2;         // bytes of the row that exist from this piece on
-                        cp_async16_zfill(dst + ((j ^ (row & 7)) << 4), src + (kk < D ? kk : 0), left >= 16 ? 16u : left > 0 ? (uint32_t)left : 0u);
+                        const int kk = k0 + j * kPiece;
+                        const int left = (D - kk) * kEsz;      // bytes of the row that exist from this piece on
+                        cp_async16_zfill(dst + ((j ^ (row & 7)) << 4), src + (kk < D ? kk : 0) * kEsz,
+                                         left >= 16 ? 16u : left > 0 ? (uint32_t)left : 0u);
                     }
                     cp_async_commit();
                     if (pending >= 0) {                        // the copies of the previous slab have landed by now
                         cp_async_wait<1>();
-                        fence_proxy_async();
-                        mbar_arrive(bar(gbar_full_a(pending)));
+                        signal(pending);
                     }
                     pending = s;
                 }
             }
         }
         cp_async_wait<0>();
-        if (pending >= 0 && ok) {
-            fence_proxy_async();
-            mbar_arrive(bar(gbar_full_a(pending)));
-        }
+        if (pending >= 0 && ok) signal(pending);
     } else {
         // ================================================================ epilogue warps (one row per thread, half the columns)
         const int eg = (warp - kGEpiWarp0) >> 2;               // column half of every chunk this group reads
@@ -304,10 +379,12 @@ k_score_gemm_bf16(const __grid_constant__ CUtensorMap wt_map, const __grid_const
                 if (!warp_wait(bar(gbar_r_full(b)), par, abort_flag)) { ok = false; break; }
                 if (!warp_wait(bar(gbar_acc_full(b)), par, abort_flag)) { ok = false; break; }
                 tc_fence_after();
-                const float *rt = rtab + b * (kRBytes / 4), *bt = btab + b * kNC;
+                const float *rt = rtab + b * (kRBytes / 4), *bt = btab + b * (G::BiasSlot / 4);
                 const int c_base = ch * kNC;
-                for (int sb = 0; sb < 4; ++sb) {
-                    const int col0 = eg * 128 + sb * 32;                   // column of the chunk
+                constexpr int kHalf = kNC / 2;                             // columns of a chunk per epilogue group
+                for (int sb = 0; sb < (kHalf + 31) / 32; ++sb) {
+                    const int col0 = eg * kHalf + sb * 32;                 // column of the chunk
+                    const int col_end = (eg + 1) * kHalf;                  // this group's columns end here
                     if (c_base + col0 >= C) break;                         // uniform: nothing valid from here on
                     float z[32];
                     tmem_ld<32>(((uint32_t)(quad * 32) << 16) + b * kNC + col0, z);
@@ -315,13 +392,20 @@ k_score_gemm_bf16(const __grid_constant__ CUtensorMap wt_map, const __grid_const
                     float bm = -INFINITY;
 #pragma unroll
                     for (int c = 0; c < 32; c += 4) {
-                        const float4 bv = *reinterpret_cast<const float4 *>(bt + col0 + c);
-                        z[c] = (z[c] + bv.x) * kLog2e; z[c + 1] = (z[c + 1] + bv.y) * kLog2e;
-                        z[c + 2] = (z[c + 2] + bv.z) * kLog2e; z[c + 3] = (z[c + 3] + bv.w) * kLog2e;
+                        if (col0 + c < kNC) {                              // the bias row has NC entries
+                            const float4 bv = *reinterpret_cast<const float4 *>(bt + col0 + c);
+                            if (F32) {                                     // log2(e) is already in the head image
+                                z[c] = fmaf(bv.x, kLog2e, z[c]); z[c + 1] = fmaf(bv.y, kLog2e, z[c + 1]);
+                                z[c + 2] = fmaf(bv.z, kLog2e, z[c + 2]); z[c + 3] = fmaf(bv.w, kLog2e, z[c + 3]);
+                            } else {
+                                z[c] = (z[c] + bv.x) * kLog2e; z[c + 1] = (z[c + 1] + bv.y) * kLog2e;
+                                z[c + 2] = (z[c + 2] + bv.z) * kLog2e; z[c + 3] = (z[c + 3] + bv.w) * kLog2e;
+                            }
+                        }
                     }
 #pragma unroll
                     for (int c = 0; c < 32; ++c) {
-                        if (c_base + col0 + c >= C) z[c] = -INFINITY;
+                        if (c_base + col0 + c >= C || col0 + c >= col_end) z[c] = -INFINITY;
                         bm = fmaxf(bm, z[c]);
                     }
                     if (bm > run_m) {                                      // rescale what has been summed so far
@@ -342,9 +426,11 @@ k_score_gemm_bf16(const __grid_constant__ CUtensorMap wt_map, const __grid_const
                             float p0 = 0.f, p1 = 0.f;
 #pragma unroll
                             for (int c = 0; c < 32; c += 4) {
-                                const float4 rv = *reinterpret_cast<const float4 *>(rr + c);
-                                p0 = fmaf(z[c], rv.x, p0); p1 = fmaf(z[c + 1], rv.y, p1);
-                                p0 = fmaf(z[c + 2], rv.z, p0); p1 = fmaf(z[c + 3], rv.w, p1);
+                                if (col0 + c < kNC) {                      // a recall row has NC entries; z is 0 past the group's end
+                                    const float4 rv = *reinterpret_cast<const float4 *>(rr + c);
+                                    p0 = fmaf(z[c], rv.x, p0); p1 = fmaf(z[c + 1], rv.y, p1);
+                                    p0 = fmaf(z[c + 2], rv.z, p0); p1 = fmaf(z[c + 3], rv.w, p1);
+                                }
                             }
                             racc[j] += p0 + p1;
                         }
