@@ -237,7 +237,9 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
     __shared__ double s_P[kMaxApps];
     __shared__ int s_seg[kMaxApps + 2];
     __shared__ int s_newhead[kMaxApps];
-    __shared__ int64_t s_nnew;
+    __shared__ int64_t s_emin[kMaxApps];
+    __shared__ unsigned s_ballot[32];
+    __shared__ double s_part[32 * kMaxApps];
     __shared__ int s_best_app, s_exactP, s_best_ci, s_nclose, s_maxbp;
     __shared__ double s_best_u, s_best_p;
     __shared__ unsigned char s_contend[kMaxApps];
@@ -283,19 +285,21 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
     for (int64_t iter = 0; iter < max_iter; ++iter) {
         if (rounds_done >= sp.max_rounds) { finished = true; break; }
         // ---------------------------------------------------------------- 1. arrivals join their queues
-        if (tid == 0) {
-            if (!st.started) { st.started = 1; st.Tref = st.T; }
-            int64_t lo = st.inserted, hi = n_inst;
-            if (sp.trace_mode) {              // first request (in arrival order) that has not arrived yet
-                while (lo < hi) {
-                    const int64_t mid = (lo + hi) >> 1;
-                    if (tb.arrival[r0 + mid] <= st.T) lo = mid + 1; else hi = mid;
-                }
-            } else lo = n_inst;
-            s_nnew = lo - st.inserted;
-        }
+        if (tid == 0 && !st.started) { st.started = 1; st.Tref = st.T; }
         __syncthreads();
-        const int64_t nnew = s_nnew;
+        int64_t arrived_upto = n_inst;
+        if (sp.trace_mode) {
+            // Requests are in arrival order: the whole block looks at the next NT arrival times at once (one
+            // memory round trip instead of a binary search of dependent loads) and counts those that have passed.
+            arrived_upto = st.inserted;
+            for (;;) {
+                const int64_t k = arrived_upto + tid;
+                const int cnt = __syncthreads_count(k < n_inst && tb.arrival[r0 + k] <= st.T);
+                arrived_upto += cnt;
+                if (cnt < NT) break;
+            }
+        }
+        const int64_t nnew = arrived_upto - st.inserted;
         if (nnew > 0) {
             const int64_t ap = st.inserted;
             SortKey *keys = nnew <= sp.sort_cap ? smem_keys : sp.sort_scratch + r0 + ap;
@@ -389,18 +393,43 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
             __syncthreads();
         }
         // ---------------------------------------------------------------- 2. retire hopeless requests
+        if (tid < A) {                        // earliest completion any candidate of the application can reach
+            const int a = tid;
+            int64_t emin = INT64_MAX;
+            for (int g = P.mfirst[a]; g < P.mfirst[a + 1]; ++g) {
+                const int64_t e = st.T + (g != st.L ? sw[g] : 0) + al[g] + be[g] * (int64_t)P.batch[0];
+                emin = e < emin ? e : emin;
+            }
+            s_emin[a] = emin;
+        }
+        __syncthreads();
+        {
+            // The queues are sorted by deadline, so the late requests of a queue are a prefix.  Every application
+            // gets NT / 16 threads that look at the head of its queue at once (one memory round trip); only a queue
+            // whose whole window is late continues with a binary search behind it.
+            const int per = NT / kMaxApps, a = tid / per, j = tid - a * per;
+            bool late = false;
+            if (a < A) {
+                const int k = st.head[a] + j;
+                late = k < st.tail[a] && (sp.q_dl[st.cur[a]] + tb.gstart[(int64_t)inst * A + a])[k] < s_emin[a];
+            }
+            const unsigned bal = __ballot_sync(0xffffffffu, late);
+            if (lane == 0) s_ballot[warp] = bal;
+        }
+        __syncthreads();
         if (tid < A) {
-            const int a = tid, head = st.head[a], tail = st.tail[a];
-            int nh = head;
-            if (tail > head) {
-                int64_t emin = INT64_MAX;
-                for (int g = P.mfirst[a]; g < P.mfirst[a + 1]; ++g) {
-                    const int64_t e = st.T + (g != st.L ? sw[g] : 0) + al[g] + be[g] * (int64_t)P.batch[0];
-                    emin = e < emin ? e : emin;
-                }
+            const int a = tid, per = NT / kMaxApps, head = st.head[a], tail = st.tail[a];
+            int cnt = 0;                      // leading late requests inside the window
+            for (int j = 0; j < per; ++j) {
+                const int t2 = a * per + j;
+                if (!((s_ballot[t2 >> 5] >> (t2 & 31)) & 1u)) break;
+                ++cnt;
+            }
+            int nh = head + cnt;
+            if (cnt == per && nh < tail) {
                 const int64_t *dl = sp.q_dl[st.cur[a]] + tb.gstart[(int64_t)inst * A + a];
-                int lo = head, hi = tail;
-                while (lo < hi) { const int mid = (lo + hi) >> 1; if (dl[mid] < emin) lo = mid + 1; else hi = mid; }
+                int lo = nh, hi = tail;
+                while (lo < hi) { const int mid = (lo + hi) >> 1; if (dl[mid] < s_emin[a]) lo = mid + 1; else hi = mid; }
                 nh = lo;
             }
             s_newhead[a] = nh;
@@ -421,14 +450,33 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
         for (int a = 0; a < A; ++a) live += st.tail[a] - st.head[a];
         if (live == 0) continue;
         // ---------------------------------------------------------------- 3. group priorities (Eq. 14)
-        for (int a = 0; a < A; ++a) {
-            const int na = st.tail[a] - st.head[a];
-            if (na == 0) { if (tid == 0) s_P[a] = -INFINITY; continue; }
-            const double *pw = sp.q_pw[st.cur[a]] + tb.gstart[(int64_t)inst * A + a];
-            double part = 0.0;
-            for (int k = st.head[a] + tid; k < st.tail[a]; k += NT) part += pw[k];
-            const double S = block_sum(part, red);
-            if (tid == 0) s_P[a] = S / (double)na;
+        {
+            // partial sums of every application first (their loads are in flight together), then one reduction
+            double part[kMaxApps];
+#pragma unroll
+            for (int a = 0; a < kMaxApps; ++a) {
+                part[a] = 0.0;
+                if (a < A) {
+                    const double *pw = sp.q_pw[st.cur[a]] + tb.gstart[(int64_t)inst * A + a];
+                    for (int k = st.head[a] + tid; k < st.tail[a]; k += NT) part[a] += pw[k];
+                }
+            }
+#pragma unroll
+            for (int a = 0; a < kMaxApps; ++a) {
+                if (a < A) {
+                    double v = part[a];
+#pragma unroll
+                    for (int o = 16; o >= 1; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+                    if (lane == 0) s_part[warp * kMaxApps + a] = v;
+                }
+            }
+            __syncthreads();
+            if (tid < A) {
+                const int na = st.tail[tid] - st.head[tid];
+                double S = 0.0;
+                for (int w2 = 0; w2 < nwarps; ++w2) S += s_part[w2 * kMaxApps + tid];
+                s_P[tid] = na > 0 ? S / (double)na : -INFINITY;
+            }
         }
         __syncthreads();
         if (tid == 0) {
