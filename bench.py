@@ -54,9 +54,11 @@ def make(args, rank, n_instances=None):
         kw["n_requests"] = args.requests
     ni = n_instances if n_instances is not None else args.instances
     if args.workload == "C4":
+        from paper_2505_06641_b200 import shard
         full = synth._SPECS["C4"][2]
         ni = ni if ni is not None else full
-        return synth.make_workload("C4", n_instances=ni, first_instance=rank * full, **kw)
+        first, _ = shard.instance_shard(rank, max(rank + 1, int(os.environ.get("WORLD_SIZE", "1"))), full)
+        return synth.make_workload("C4", n_instances=ni, first_instance=first, **kw)
     return synth.make_workload(args.workload, **kw)
 
 
@@ -224,15 +226,8 @@ def main():
     st = api.sp_get_stats(ses.ctx)
     launches = st["kernel_launches"] - launches0
     n_rounds = int(ses.n_done.sum().item())
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-        cnt = torch.tensor([n, launches, n_rounds], dtype=torch.int64, device="cuda")
-        dist.all_reduce(cnt, op=dist.ReduceOp.SUM)
-        n_total, launches, n_rounds_total = int(cnt[0]), int(cnt[1]), int(cnt[2])
-    else:
-        n_total, n_rounds_total = n, n_rounds
+    from paper_2505_06641_b200 import shard
+    ms, (n_total, launches, n_rounds_total) = shard.reduce_step_stats(ms, [n, launches, n_rounds], "cuda")
     ms_per_step = ms / args.steps
     value = n_total / (ms_per_step * 1e-3)
 
@@ -293,10 +288,7 @@ def main():
             call()
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([dt], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
+        dt, _ = shard.reduce_step_stats(dt, [], "cuda")
         h2d = hf.nbytes + ha.nbytes + harr.nbytes + hdl.nbytes + (hinst.nbytes if hinst is not None else 0) + ht0.nbytes + hl0.nbytes
         d2h = reqs.nbytes + rounds.nbytes + nd.nbytes
         e2e = {"value": n_total / (dt / e2e_steps), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
