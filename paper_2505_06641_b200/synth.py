@@ -262,3 +262,36 @@ def make_workload(name: str, n_requests: Optional[int] = None, n_instances: Opti
         t0_ns=np.asarray([p["t0"] for p in parts], dtype=np.int64), trace_mode=spec.trace_mode,
         meta=dict(base_seed=base_seed, first_instance=first_instance, requests_per_instance=n),
     )
+
+
+def with_short_circuit(w: Workload, static_acc) -> Workload:
+    """Adds the short-circuit candidate of the paper's Section 4.3 to every application of ``w``.
+
+    The candidate is one more model variant per application, placed after the application's own variants: it
+    answers at once (latency alpha = beta = 0, no swap time) and its accuracy is the profiled, static accuracy
+    ``static_acc[a]`` whatever the request looks like.  In the profile format that is a recall row that holds the
+    same value for every label.  Only profile arrays change; requests, heads and seeds stay as they are.
+    """
+    a, ni = int(w.n_apps), int(w.n_instances)
+    acc = np.broadcast_to(np.asarray(static_acc, dtype=np.float32), (a,))
+    old_m = np.asarray(w.models_per_app, dtype=np.int64)
+    first = np.concatenate([[0], np.cumsum(old_m)])
+    c = int(w.n_classes)
+
+    def grow(arr, fill_rows):
+        out = []
+        for app in range(a):
+            out.append(arr[:, first[app]:first[app + 1]])
+            out.append(fill_rows[app])
+        return np.ascontiguousarray(np.concatenate(out, axis=1))
+
+    recall = grow(w.recall, [np.full((ni, 1, c), acc[app], dtype=np.float32) for app in range(a)])
+    zeros = [np.zeros((ni, 1), dtype=np.int64) for _ in range(a)]
+    out = Workload(**{**w.__dict__})
+    out.models_per_app = (old_m + 1).astype(np.int32)
+    out.recall = recall
+    out.lat_alpha_ns = grow(w.lat_alpha_ns, zeros)
+    out.lat_beta_ns = grow(w.lat_beta_ns, zeros)
+    out.swap_ns = grow(w.swap_ns, zeros)
+    out.meta = dict(w.meta, short_circuit=[float(x) for x in acc])
+    return out

@@ -253,3 +253,17 @@ def test_full_size_batched_workload_on_sampled_instances():
     per_inst = np.add.reduceat(sched.astype(np.int64), starts[:-1])
     max_order = np.maximum.reduceat(np.where(sched, res.reqs["order"], 0), starts[:-1])
     assert np.array_equal(per_inst, max_order)
+
+
+@pytest.mark.parametrize("name,kw,tight", [("C1", {}, False), ("C4", dict(n_instances=10), False),
+                                           ("C1", dict(n_requests=200), True), ("C5", dict(n_requests=3000), False)])
+def test_short_circuit_candidate(name, kw, tight):
+    """Section 4.3's zero-latency candidate with static accuracy, added to every application's variants."""
+    w = synth.with_short_circuit(synth.make_workload(name, **kw), [0.55, 0.6, 0.65])
+    if tight:                             # nothing but the zero-latency candidate can meet these deadlines
+        w.deadline_ns = np.maximum(w.deadline_ns, w.t0_ns[0]) * 0 + int(w.t0_ns[0]) + synth.MS
+    s, od, res = _both(w)
+    check_scores(res, s)
+    check_schedule(w, res, od)
+    if tight:
+        assert np.all(res.reqs["status"] == 1) and np.all(res.rounds[0, :int(res.n_rounds[0])]["t_end_ns"] == w.t0_ns[0])

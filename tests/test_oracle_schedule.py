@@ -264,3 +264,25 @@ def test_max_rounds_stops_early_and_leaves_the_rest_pending():
     full = oracle.drain(w, s.acc, s.v)
     assert d.n_rounds[0] == 2 and np.array_equal(d.rounds[0, :2], full.rounds[0, :2])
     assert np.sum(d.reqs["status"] == oracle.PENDING) > 0
+
+
+def test_short_circuit_candidate_is_static_and_wins_when_nothing_else_is_in_time():
+    """Section 4.3: the SneakPeek model as one more candidate with zero latency and its profiled (static) accuracy.
+    In the profile format it is a recall row with one value for every label, so Eq. 9 gives that value for every
+    request; with deadlines that no real variant can meet it is the only candidate with non-zero utility."""
+    from oracle import oracle
+    from paper_2505_06641_b200 import synth
+    w = synth.with_short_circuit(synth.make_workload("C1", n_requests=60), [0.55, 0.6, 0.65])
+    assert list(w.models_per_app) == [5, 5, 5] and w.recall.shape[1] == 15
+    s = oracle.score(w)
+    for a in range(3):
+        np.testing.assert_allclose(s.acc[w.app == a, 4], [0.55, 0.6, 0.65][a], rtol=1e-6)
+    # every deadline 1 ms after the starting clock: real variants need at least 2.5 ms
+    w.deadline_ns = np.full_like(w.deadline_ns, int(w.t0_ns[0]) + synth.MS)
+    d = oracle.drain(w, s.acc, s.v)
+    assert np.all(d.reqs["status"] == 1)
+    first = np.concatenate([[0], np.cumsum(w.models_per_app)])
+    assert np.all(d.reqs["model"] == first[w.app + 1] - 1)            # the short-circuit variant of its application
+    nr = int(d.n_rounds[0])
+    assert np.all(d.rounds[0, :nr]["t_end_ns"] == w.t0_ns[0])           # zero latency: the clock does not move
+    np.testing.assert_allclose(d.rounds[0, :nr]["utility"].sum(), s.acc[np.arange(60), 4].astype(np.float64).sum(), rtol=1e-12)
