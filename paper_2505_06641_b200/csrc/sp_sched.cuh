@@ -237,6 +237,7 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
     __shared__ double s_P[kMaxApps];
     __shared__ int s_seg[kMaxApps + 2];
     __shared__ int s_newhead[kMaxApps];
+    __shared__ int s_lstart[kMaxApps + 1];
     __shared__ int64_t s_emin[kMaxApps];
     __shared__ unsigned s_ballot[32];
     __shared__ double s_part[32 * kMaxApps];
@@ -316,45 +317,54 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
                 s_seg[tid] = lo;
             }
             __syncthreads();
-            for (int a = 0; a < A; ++a) {
-                const int nn = s_seg[a + 1] - s_seg[a];
-                if (nn == 0) continue;
+            // Merge of every application's new keys into its live queue, all applications at once (one thread per
+            // element, so the dependent loads of the binary searches are paid once per call, not once per application).
+            if (tid == 0) {                       // live elements of the queues that get new members, flattened
+                int tot = 0;
+                for (int a = 0; a < A; ++a) {
+                    s_lstart[a] = tot;
+                    if (s_seg[a + 1] - s_seg[a] > 0) tot += st.tail[a] - st.head[a];
+                }
+                s_lstart[A] = tot;
+            }
+            __syncthreads();
+            for (int t = tid; t < (int)nnew; t += NT) {      // new element: count live elements before it
+                const int a = keys[t].app, tl = t - s_seg[a];
                 const int64_t base = tb.gstart[(int64_t)inst * A + a];
                 const int head = st.head[a], tail = st.tail[a], nl = tail - head, c = st.cur[a];
-                const SortKey *nk = keys + s_seg[a];
-                if (nl == 0) {
-                    for (int t = tid; t < nn; t += NT) {
-                        const int64_t id = r0 + nk[t].id_rel, pos = base + tail + t;
-                        sp.q_id[c][pos] = id; sp.q_dl[c][pos] = nk[t].dl;
-                        sp.q_pw[c][pos] = prio_weight((double)tb.v32[id], nk[t].dl, st.Tref, tau);
-                    }
-                } else {
-                    const int d = 1 - c;
+                const int64_t dl = keys[t].dl, idr = keys[t].id_rel, id = r0 + idr;
+                int lo = 0, buf = c;
+                if (nl > 0) {
                     const int64_t *lid = sp.q_id[c] + base + head, *ldl = sp.q_dl[c] + base + head;
-                    for (int k = tid; k < nl; k += NT) {        // live element: count new elements before it
-                        const int64_t dl = ldl[k], idr = lid[k] - r0;
-                        int lo = 0, hi = nn;
-                        while (lo < hi) {
-                            const int mid = (lo + hi) >> 1;
-                            const bool less = nk[mid].dl < dl || (nk[mid].dl == dl && nk[mid].id_rel < idr);
-                            if (less) lo = mid + 1; else hi = mid;
-                        }
-                        const int64_t pos = base + head + k + lo;
-                        sp.q_id[d][pos] = lid[k]; sp.q_dl[d][pos] = dl; sp.q_pw[d][pos] = sp.q_pw[c][base + head + k];
+                    int hi = nl;
+                    while (lo < hi) {
+                        const int mid = (lo + hi) >> 1;
+                        const int64_t md = ldl[mid];
+                        const bool less = md < dl || (md == dl && (lid[mid] - r0) < idr);
+                        if (less) lo = mid + 1; else hi = mid;
                     }
-                    for (int t = tid; t < nn; t += NT) {        // new element: count live elements before it
-                        const int64_t dl = nk[t].dl, idr = nk[t].id_rel;
-                        int lo = 0, hi = nl;
-                        while (lo < hi) {
-                            const int mid = (lo + hi) >> 1;
-                            const bool less = ldl[mid] < dl || (ldl[mid] == dl && (lid[mid] - r0) < idr);
-                            if (less) lo = mid + 1; else hi = mid;
-                        }
-                        const int64_t id = r0 + idr, pos = base + head + t + lo;
-                        sp.q_id[d][pos] = id; sp.q_dl[d][pos] = dl;
-                        sp.q_pw[d][pos] = prio_weight((double)tb.v32[id], dl, st.Tref, tau);
-                    }
+                    buf = 1 - c;
                 }
+                const int64_t pos = base + (nl > 0 ? head : tail) + tl + lo;
+                sp.q_id[buf][pos] = id; sp.q_dl[buf][pos] = dl;
+                sp.q_pw[buf][pos] = prio_weight((double)tb.v32[id], dl, st.Tref, tau);
+            }
+            for (int f = tid; f < s_lstart[A]; f += NT) {     // live element: count new elements before it
+                int a = 0;
+                while (f >= s_lstart[a + 1]) ++a;
+                const int k = f - s_lstart[a], nn = s_seg[a + 1] - s_seg[a];
+                const int64_t base = tb.gstart[(int64_t)inst * A + a];
+                const int head = st.head[a], c = st.cur[a], d = 1 - c;
+                const SortKey *nk = keys + s_seg[a];
+                const int64_t lidk = sp.q_id[c][base + head + k], dl = sp.q_dl[c][base + head + k], idr = lidk - r0;
+                int lo = 0, hi = nn;
+                while (lo < hi) {
+                    const int mid = (lo + hi) >> 1;
+                    const bool less = nk[mid].dl < dl || (nk[mid].dl == dl && nk[mid].id_rel < idr);
+                    if (less) lo = mid + 1; else hi = mid;
+                }
+                const int64_t pos = base + head + k + lo;
+                sp.q_id[d][pos] = lidk; sp.q_dl[d][pos] = dl; sp.q_pw[d][pos] = sp.q_pw[c][base + head + k];
             }
             __syncthreads();
             if (tid == 0) {
