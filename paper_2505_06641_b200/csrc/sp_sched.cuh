@@ -415,9 +415,9 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
         __syncthreads();
         {
             // The queues are sorted by deadline, so the late requests of a queue are a prefix.  Every application
-            // gets NT / 16 threads that look at the head of its queue at once (one memory round trip); only a queue
+            // gets NT / A threads that look at the head of its queue at once (one memory round trip); only a queue
             // whose whole window is late continues with a binary search behind it.
-            const int per = NT / kMaxApps, a = tid / per, j = tid - a * per;
+            const int per = NT / A, a = tid / per, j = tid - a * per;
             bool late = false;
             if (a < A) {
                 const int k = st.head[a] + j;
@@ -428,7 +428,7 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
         }
         __syncthreads();
         if (tid < A) {
-            const int a = tid, per = NT / kMaxApps, head = st.head[a], tail = st.tail[a];
+            const int a = tid, per = NT / A, head = st.head[a], tail = st.tail[a];
             int cnt = 0;                      // leading late requests inside the window
             for (int j = 0; j < per; ++j) {
                 const int t2 = a * per + j;
