@@ -42,7 +42,7 @@ class _Profiles(C.Structure):
         ("prior_alpha", C.c_void_p), ("evidence_k", C.c_double), ("recall", C.c_void_p),
         ("lat_alpha_ns", C.c_void_p), ("lat_beta_ns", C.c_void_p), ("swap_ns", C.c_void_p),
         ("batch_sizes", C.c_void_p), ("n_batch_sizes", C.c_int32),
-        ("prio_time_scale_s", C.c_double),
+        ("prio_time_scale_s", C.c_double), ("penalty_kind", C.c_void_p),
     ]
 
 
@@ -67,12 +67,19 @@ def _load():
         lib.orc_drain.argtypes = ([C.POINTER(_Profiles), C.c_int64] + [C.c_void_p] * 8 +
                                   [C.c_int, C.c_int64, C.c_void_p, C.c_int64] + [C.c_void_p] * 4)
         lib.orc_num_threads.restype = C.c_int
+        lib.orc_penalty.restype = C.c_double
+        lib.orc_penalty.argtypes = [C.c_int, C.c_int64, C.c_int64, C.c_int64]
         _lib = lib
     return _lib
 
 
 def num_threads() -> int:
     return int(_load().orc_num_threads())
+
+
+def penalty(kind: int, deadline_ns: int, arrival_ns: int, completion_ns: int) -> float:
+    """gamma of Eq. 2 under the stated reading of Section 5.1 (0 step, 1 linear, 2 sigmoid)."""
+    return float(_load().orc_penalty(int(kind), int(deadline_ns), int(arrival_ns), int(completion_ns)))
 
 
 def _ptr(a: Optional[np.ndarray]):
@@ -89,13 +96,14 @@ class _Bound:
             mpa=f(w.models_per_app, np.int32), head_w=f(w.head_w, wdt), head_b=f(w.head_b, np.float32),
             prior=None if w.prior_alpha is None else f(w.prior_alpha, np.float32),
             recall=f(w.recall, np.float32), al=f(w.lat_alpha_ns, np.int64), be=f(w.lat_beta_ns, np.int64),
-            sw=f(w.swap_ns, np.int64), bs=f(w.batch_sizes, np.int32))
+            sw=f(w.swap_ns, np.int64), bs=f(w.batch_sizes, np.int32),
+            pen=f(w.penalty_kind, np.int32))
         k = self.keep
         self.struct = _Profiles(
             int(w.n_instances), int(w.n_apps), int(w.n_classes), int(w.feat_dim), int(w.feat_dtype),
             _ptr(k["mpa"]), _ptr(k["head_w"]), _ptr(k["head_b"]), _ptr(k["prior"]), float(w.evidence_k),
             _ptr(k["recall"]), _ptr(k["al"]), _ptr(k["be"]), _ptr(k["sw"]), _ptr(k["bs"]),
-            int(k["bs"].shape[0]), float(w.prio_time_scale_s))
+            int(k["bs"].shape[0]), float(w.prio_time_scale_s), _ptr(k["pen"]))
 
 
 @dataclass

@@ -15,7 +15,10 @@
  * literal Algorithm 1 on one-batch groups, brute force over all pick sequences on tiny queues.
  * Parity UNPINNED by the paper (readings of points it leaves open, pinned only by their
  * stated definition): the purge rule for hopeless requests, deadline order inside a group,
- * batch-size candidates with l(m,b) = alpha + beta*b and a separate swap cost.
+ * batch-size candidates with l(m,b) = alpha + beta*b and a separate swap cost, and the linear
+ * and sigmoid penalties (Section 5.1 prints them garbled; orc_penalty() states the reading and
+ * is pinned only at gamma(e = d) = 0, gamma(half way) = 1/2, gamma(>= relative deadline late) = 1
+ * and monotonicity).
  */
 #include <math.h>
 #include <stdint.h>
@@ -27,6 +30,7 @@
 
 enum { ORC_F32 = 0, ORC_BF16 = 1 };
 enum { ORC_PENDING = 0, ORC_SCHEDULED = 1, ORC_EXPIRED = 2 };
+enum { ORC_PEN_STEP = 0, ORC_PEN_LINEAR = 1, ORC_PEN_SIGMOID = 2 };
 
 typedef struct {
     int32_t n_instances, n_apps, n_classes, feat_dim, feat_dtype;
@@ -40,6 +44,7 @@ typedef struct {
     const int32_t *batch_sizes;      /* [nB] ascending */
     int32_t n_batch_sizes;
     double prio_time_scale_s;        /* tau of exp(-(d - T)/tau) */
+    const int32_t *penalty_kind;     /* [A] ORC_PEN_*, or NULL = step for every application */
 } orc_profiles;
 
 typedef struct {
@@ -158,6 +163,34 @@ int orc_score(const orc_profiles *p, int64_t n, const void *feats, const int32_t
 }
 
 /* ---------------------------------------------------------------------------------------------
+ * Penalty gamma of Eq. 2 for a request with deadline d that arrived at `arrival` and would complete at e
+ * (Section 5.1).  step: 1 when the deadline is missed, else 0.  The linear and sigmoid forms are printed
+ * with max(1, .) and a ratio to "d"; read literally they never fall below 1 once late, so they are read as
+ *   x = (e - d) / delta,  delta = d - arrival (the relative deadline),
+ *   linear : gamma = min(max(x, 0), 1)
+ *   sigmoid: gamma = 0 for x <= 0, 1 for x >= 1, else 1 / (1 + ((1 - x) / x)^3)
+ * so that the utility degrades from the deadline on and is gone once the request is late by its whole relative
+ * deadline.  A request whose deadline is not after its arrival falls back to the step form.
+ * ------------------------------------------------------------------------------------------- */
+double orc_penalty(int kind, int64_t d, int64_t arrival, int64_t e)
+{
+    const int64_t delta = d - arrival;
+    if (kind == ORC_PEN_STEP || delta <= 0) return d < e ? 1.0 : 0.0;
+    if (e <= d) return 0.0;
+    if (e - d >= delta) return 1.0;
+    const double x = (double)(e - d) / (double)delta;
+    if (kind == ORC_PEN_LINEAR) return x;
+    const double r = (1.0 - x) / x;
+    return 1.0 / (1.0 + r * r * r);
+}
+
+/* A request is hopeless when even the earliest completion `emin` its group can reach leaves it no utility. */
+static int hopeless(int kind, int64_t d, int64_t arrival, int64_t emin)
+{
+    return orc_penalty(kind, d, arrival, emin) >= 1.0;
+}
+
+/* ---------------------------------------------------------------------------------------------
  * Scheduling rounds of one instance (Section 4.2: groups = applications, Eq. 14 group priority,
  * Eq. 13 applied to the group with summed member utilities (Eq. 2), Algorithm 1's greedy branch
  * taken one batch at a time).  Readings of points the paper leaves open:
@@ -165,9 +198,11 @@ int orc_score(const orc_profiles *p, int64_t n, const void *feats, const int32_t
  *   - a candidate is (model m, allowed batch size b): the first b' = min(b, n_a) live requests
  *     of the group run as one batch that completes at e = T + swap_m*[m != loaded] + alpha_m
  *     + beta_m*b' (Eq. 1 with the swap time kept separate from the inference latency);
- *   - step penalty (Section 5.1): a member with deadline < e contributes 0, else acc[member][m];
- *   - a request whose deadline precedes the earliest completion any candidate of its group
- *     could reach from the current state can never earn utility: it is retired as EXPIRED;
+ *   - a member contributes acc[member][m] * (1 - gamma) with the application's penalty gamma of
+ *     orc_penalty() (step penalty: 0 when its deadline < e, else acc[member][m]);
+ *   - a request at the head of its group's queue whose penalty is already 1 at the earliest
+ *     completion any candidate of the group could reach from the current state can never earn
+ *     utility: it is retired as EXPIRED (for the step penalty: every request with deadline < that time);
  *   - group priorities are re-evaluated every round over the live members, with d measured
  *     from the current clock in seconds and scaled by tau;
  *   - ties: lowest application index; lowest model index, then smallest batch size.
@@ -248,7 +283,8 @@ static void drain_instance(const orc_profiles *p, int inst, int64_t lo, int64_t 
                 const int64_t e = T + (g != L ? sw[g] : 0) + al[g] + be[g] * bmin;
                 if (e < emin) emin = e;
             }
-            while (head[a] < tail[a] && q[a][head[a]].deadline < emin) {
+            const int pk = p->penalty_kind ? p->penalty_kind[a] : ORC_PEN_STEP;
+            while (head[a] < tail[a] && hopeless(pk, q[a][head[a]].deadline, arrival[q[a][head[a]].id], emin)) {
                 orc_req_rec *r = &reqs[q[a][head[a]].id];
                 r->status = ORC_EXPIRED; r->round = (int32_t)round;
                 ++head[a]; ++exp_since;
@@ -276,6 +312,7 @@ static void drain_instance(const orc_profiles *p, int inst, int64_t lo, int64_t 
         /* 5./6. every (model, batch size) candidate of the chosen group; best summed utility */
         const int a = best_a, g0 = first_model(p, a), M = p->models_per_app[a];
         const int64_t na = tail[a] - head[a];
+        const int pen = p->penalty_kind ? p->penalty_kind[a] : ORC_PEN_STEP;
         int best_j = -1, best_b = 0;
         int64_t best_bp = 0, best_e = 0;
         double best_u = 0.0, second_u = -INFINITY;
@@ -287,7 +324,8 @@ static void drain_instance(const orc_profiles *p, int inst, int64_t lo, int64_t 
                 double u = 0.0;
                 for (int64_t k = 0; k < bp; ++k) {
                     const qkey *m = &q[a][head[a] + k];
-                    if (!(m->deadline < e)) u += acc[m->id * MM + j];
+                    if (pen == ORC_PEN_STEP) { if (!(m->deadline < e)) u += acc[m->id * MM + j]; }
+                    else u += acc[m->id * MM + j] * (1.0 - orc_penalty(pen, m->deadline, arrival[m->id], e));
                 }
                 if (best_j < 0) { best_j = j; best_b = (int)b; best_bp = bp; best_e = e; best_u = u; }
                 else if (u > best_u) { second_u = best_u; best_j = j; best_b = (int)b; best_bp = bp; best_e = e; best_u = u; }

@@ -106,8 +106,17 @@ def replay_schedule(w, acc, reqs, rounds, n_rounds, loaded0=-1, inst=0):
         end = start + (int(sw[g]) if g != prev_model else 0) + int(al[g]) + int(be[g]) * len(members)
         assert end == rec["t_end_ns"]
         j = g - first_model(w, a)
-        u = sum(float(acc[i, j]) for i in members if not (w.deadline_ns[i] < end))
-        assert abs(u - rec["utility"]) <= 1e-12 * max(1.0, abs(u))
+        kind = int(w.penalty_kind[a])
+        if kind == 0:
+            u = sum(float(acc[i, j]) for i in members if not (w.deadline_ns[i] < end))
+        else:                              # utility degrades over the relative deadline after the deadline (Section 5.1)
+            u = 0.0
+            for i in members:
+                d, delta = int(w.deadline_ns[i]), int(w.deadline_ns[i]) - int(w.arrival_ns[i])
+                late = min(max((end - d) / delta, 0.0), 1.0) if delta > 0 else float(d < end)
+                gamma = late if kind == 1 else (0.0 if late <= 0 else 1.0 if late >= 1 else 1.0 / (1.0 + ((1.0 - late) / late) ** 3))
+                u += float(acc[i, j]) * (1.0 - gamma)
+        assert abs(u - rec["utility"]) <= 1e-11 * max(1.0, abs(u))
         total += u
         clock, prev_model = end, g
     assert pos == len(sched)

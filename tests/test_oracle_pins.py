@@ -118,3 +118,29 @@ def test_ragged_models_per_app_pad_with_zero():
     s = oracle.score(w)
     np.testing.assert_allclose(s.acc, [[0.7, 0.0], [0.3, 0.8]], rtol=1e-6)
     assert s.v[0] == 1.0 and abs(s.v[1] - (1 + 0.0625)) < 1e-6
+
+
+# ------------------------------------------------------------------ penalties of Section 5.1 (reading: the design doc R12/R13)
+@pytest.mark.parametrize("kind", [1, 2])
+def test_soft_penalties_anchor_points_and_monotonicity(kind):
+    """gamma is 0 up to the deadline, 1/2 when late by half the relative deadline, 1 from a whole relative deadline
+    on, and never decreases with the completion time (the garbled print fixes no more than that)."""
+    from oracle import oracle
+    arrival, d = 1_000_000, 5_000_000                     # relative deadline 4 ms
+    delta = d - arrival
+    assert oracle.penalty(kind, d, arrival, d - 1) == 0.0 and oracle.penalty(kind, d, arrival, d) == 0.0
+    assert oracle.penalty(kind, d, arrival, d + delta // 2) == pytest.approx(0.5, abs=1e-15)
+    assert oracle.penalty(kind, d, arrival, d + delta) == 1.0 and oracle.penalty(kind, d, arrival, d + 10 * delta) == 1.0
+    g = [oracle.penalty(kind, d, arrival, d + k * delta // 1000) for k in range(0, 1001)]
+    assert all(b >= a for a, b in zip(g, g[1:])) and g[0] == 0.0 and g[-1] == 1.0
+    if kind == 1:
+        assert g[250] == pytest.approx(0.25, abs=1e-15)
+    else:                                                 # the sigmoid is symmetric about the half-way point
+        assert g[250] + g[750] == pytest.approx(1.0, abs=1e-15) and g[250] < 0.25
+
+
+def test_step_penalty_and_degenerate_relative_deadline():
+    from oracle import oracle
+    assert oracle.penalty(0, 10, 0, 10) == 0.0 and oracle.penalty(0, 10, 0, 11) == 1.0
+    for kind in (1, 2):                                   # deadline not after arrival: nothing to scale by
+        assert oracle.penalty(kind, 10, 10, 10) == 0.0 and oracle.penalty(kind, 10, 12, 11) == 1.0

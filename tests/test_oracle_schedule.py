@@ -286,3 +286,37 @@ def test_short_circuit_candidate_is_static_and_wins_when_nothing_else_is_in_time
     nr = int(d.n_rounds[0])
     assert np.all(d.rounds[0, :nr]["t_end_ns"] == w.t0_ns[0])           # zero latency: the clock does not move
     np.testing.assert_allclose(d.rounds[0, :nr]["utility"].sum(), s.acc[np.arange(60), 4].astype(np.float64).sum(), rtol=1e-12)
+
+
+@pytest.mark.parametrize("kind", [1, 2])
+def test_soft_penalty_late_member_keeps_part_of_its_accuracy(kind):
+    """One request, one variant, completion late by a quarter of the relative deadline: Eq. 2 leaves
+    acc * (1 - gamma), gamma = 1/4 (linear) or 1/28 (sigmoid: 1 / (1 + 3^3)); late by all of it: retired."""
+    from oracle import oracle
+    w = manual_workload([[0.5, 0.5]], [[0.8, 0.8]], app=[0], deadline_ms=[40], arrival_ms=[0], alpha_ms=[40], beta_ms=[10],
+                        swap_ms=[0], batch_sizes=[1], models_per_app=[1])
+    w.penalty_kind = np.asarray([kind], dtype=np.int32)
+    s = oracle.score(w)
+    d = oracle.drain(w, s.acc, s.v)                       # completes at 50 ms: 10 ms late, relative deadline 40 ms
+    assert d.reqs["status"][0] == 1
+    gamma = 0.25 if kind == 1 else 1.0 / 28.0
+    np.testing.assert_allclose(d.rounds[0, 0]["utility"], s.acc[0, 0] * (1.0 - gamma), rtol=1e-12)
+    assert abs(s.acc[0, 0] - 0.8) < 1e-7
+    w.lat_alpha_ns = np.asarray([[70 * 1_000_000]], dtype=np.int64)      # completes at 80 ms: late by the whole 40 ms
+    d = oracle.drain(w, s.acc, s.v)
+    assert d.reqs["status"][0] == 2 and d.n_rounds[0] == 0
+
+
+@pytest.mark.parametrize("kind", [1, 2])
+def test_soft_penalties_replay_and_never_below_the_step_schedule(kind):
+    from oracle import oracle
+    w = synth.make_workload("C1")
+    s = oracle.score(w)
+    step = oracle.drain(w, s.acc, s.v)
+    w.penalty_kind = np.full(3, kind, dtype=np.int32)
+    d = oracle.drain(w, s.acc, s.v)
+    nr = int(d.n_rounds[0])
+    total = replay_schedule(w, s.acc, d.reqs, d.rounds[0], nr)
+    np.testing.assert_allclose(total, d.rounds[0, :nr]["utility"].sum(), rtol=1e-12)
+    # a softer penalty retires fewer requests at the head of the queues
+    assert (d.reqs["status"] == 2).sum() <= (step.reqs["status"] == 2).sum()
