@@ -39,7 +39,10 @@ typedef enum {
 } sp_status;
 
 enum { SP_F32 = 0, SP_BF16 = 1 };                       /* feature / head-weight storage type */
-enum { SP_PEN_STEP = 0 };                               /* penalty of Eq. 2: step function of Section 5.1 */
+/* Penalty gamma of Eq. 2 (Section 5.1).  STEP: 1 once the deadline is missed.  LINEAR and SIGMOID degrade the utility
+ * after the deadline d over the request's relative deadline delta = d - arrival: with x = (completion - d) / delta,
+ * gamma = min(max(x, 0), 1) (LINEAR) or 0 for x <= 0, 1 for x >= 1, 1 / (1 + ((1 - x) / x)^3) in between (SIGMOID). */
+enum { SP_PEN_STEP = 0, SP_PEN_LINEAR = 1, SP_PEN_SIGMOID = 2 };
 enum { SP_PENDING = 0, SP_SCHEDULED = 1, SP_EXPIRED = 2 };
 
 /*
@@ -69,7 +72,7 @@ typedef struct {
     const int64_t *swap_ns;        /* [I][sumM]  time to load model m when another model is resident, >= 0 */
     const int32_t *batch_sizes;    /* [n_batch_sizes] strictly ascending, >= 1 (shared) */
     int32_t n_batch_sizes;         /* 1..16 */
-    const int32_t *penalty_kind;   /* [A] SP_PEN_STEP (shared), or NULL = all step */
+    const int32_t *penalty_kind;   /* [A] SP_PEN_* per application (shared by all instances), or NULL = all step */
     double prio_time_scale_s;      /* tau > 0 in exp(-(d - T)/tau) of Eq. 12, seconds */
 } sp_profiles;
 

@@ -318,7 +318,8 @@ sp_status sp_load_profiles(sp_ctx *c, const sp_profiles *p) {
     }
     if (p->penalty_kind)
         for (int a = 0; a < A; ++a)
-            if (p->penalty_kind[a] != SP_PEN_STEP) return fail(c, SP_EINVAL, "only the step penalty is implemented");
+            if (p->penalty_kind[a] < SP_PEN_STEP || p->penalty_kind[a] > SP_PEN_SIGMOID)
+                return fail(c, SP_EINVAL, "penalty_kind entries must be SP_PEN_STEP, SP_PEN_LINEAR or SP_PEN_SIGMOID");
     const int64_t n_models = (int64_t)I * sumM;
     const int64_t lat_limit = (int64_t)1 << 50;
     for (int64_t k = 0; k < n_models; ++k) {
@@ -386,6 +387,10 @@ sp_status sp_load_profiles(sp_ctx *c, const sp_profiles *p) {
     P.tau = p->prio_time_scale_s;
     for (int a = 0, g = 0; a <= A; ++a) { P.mfirst[a] = g; if (a < A) g += p->models_per_app[a]; }
     for (int b = 0; b < nB; ++b) P.batch[b] = p->batch_sizes[b];
+    for (int a = 0; a < A; ++a) {
+        P.pen[a] = p->penalty_kind ? p->penalty_kind[a] : SP_PEN_STEP;
+        if (P.pen[a] != SP_PEN_STEP) P.any_soft = 1;
+    }
 
     // kernel choices that depend on the shapes only
     c->sched_threads = I > 1 ? 128 : 1024;
@@ -676,7 +681,7 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
     SP_TRY(mark(c, c->ev_sched));
     // Batched mode, first call on a fresh table: one warp per instance takes every instance that fits its slice of
     // shared memory; k_sched follows for the rest (it returns at once when nothing is left).
-    if (P.I > 1 && !c->opt.trace_mode && !c->sched_started && c->tb.n > 0) {
+    if (P.I > 1 && !c->opt.trace_mode && !c->sched_started && c->tb.n > 0 && !P.any_soft) {
         int64_t wcap = 32;
         while (wcap < (c->tb.n + P.I - 1) / P.I) wcap <<= 1;
         const WarpSchedSmem W((int)wcap, P.Mmax, sp.bmax);

@@ -32,6 +32,8 @@ struct DevProfiles {
     double tau;
     int mfirst[kMaxApps + 1];  // first global model id of each application
     int batch[kMaxBatchSizes];
+    int pen[kMaxApps];         // penalty of Eq. 2 per application (SP_PEN_*)
+    int any_soft;              // some application has a penalty other than the step
 };
 
 // The request table: caller-owned inputs (borrowed) + context-owned results.

@@ -180,13 +180,14 @@ namespace sp {
 
 // Shared-memory carve-up of k_sched (bytes, 16-byte aligned pieces).
 struct SchedSmem {
-    size_t keys, pref, accs, mem_id, mem_dl, cand_u, cand_e, cand_bp, end;
+    size_t keys, pref, accs, mem_id, mem_dl, mem_delta, cand_u, cand_e, cand_bp, end;
     __host__ __device__ SchedSmem(int sort_cap, int Mmax, int bmax, int ncand) {
         size_t o = 0;
         keys = o;    o += (size_t)sort_cap * sizeof(SortKey);
         pref = o;    o += (size_t)Mmax * (bmax + 1) * sizeof(double);
         mem_id = o;  o += (size_t)bmax * sizeof(int64_t);
         mem_dl = o;  o += (size_t)bmax * sizeof(int64_t);
+        mem_delta = o; o += (size_t)bmax * sizeof(int64_t);
         cand_u = o;  o += (size_t)ncand * sizeof(double);
         cand_e = o;  o += (size_t)ncand * sizeof(int64_t);
         accs = o;    o += (size_t)bmax * Mmax * sizeof(float);
@@ -194,6 +195,25 @@ struct SchedSmem {
         end = (o + 15) & ~(size_t)15;
     }
 };
+
+// Penalty gamma of Eq. 2 (Section 5.1) for a member with deadline d and relative deadline delta = d - arrival that
+// would complete at e.  kind 0: step.  The linear and sigmoid forms are read as x = (e - d) / delta clamped to [0, 1]
+// (linear) and 1 / (1 + ((1 - x) / x)^3) in between (sigmoid): the utility degrades from the deadline on and is gone
+// once the request is late by its whole relative deadline.  A deadline that is not after the arrival: step.
+__device__ __forceinline__ double penalty_gamma(int kind, int64_t d, int64_t delta, int64_t e) {
+    if (kind == SP_PEN_STEP || delta <= 0) return d < e ? 1.0 : 0.0;
+    if (e <= d) return 0.0;
+    if (e - d >= delta) return 1.0;
+    const double x = __ddiv_rn((double)(e - d), (double)delta);
+    if (kind == SP_PEN_LINEAR) return x;
+    const double r = __ddiv_rn(__dsub_rn(1.0, x), x);
+    return __ddiv_rn(1.0, __dadd_rn(1.0, __dmul_rn(__dmul_rn(r, r), r)));
+}
+// No utility is left at completion time e: the request can be retired.
+__device__ __forceinline__ bool penalty_hopeless(int kind, int64_t d, int64_t delta, int64_t e) {
+    if (kind == SP_PEN_STEP || delta <= 0) return d < e;
+    return e > d && e - d >= delta;
+}
 
 __device__ __forceinline__ double prio_weight(double v, int64_t dl, int64_t tref, double tau) {
     return v * exp(-((double)(dl - tref) * 1e-9 / tau));
@@ -238,6 +258,7 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
     __shared__ int s_seg[kMaxApps + 2];
     __shared__ int s_newhead[kMaxApps];
     __shared__ int s_lstart[kMaxApps + 1];
+    __shared__ int s_again;
     __shared__ int64_t s_emin[kMaxApps];
     __shared__ unsigned s_ballot[32];
     __shared__ double s_part[32 * kMaxApps];
@@ -256,6 +277,7 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
     float *accs = reinterpret_cast<float *>(dyn + L.accs);
     int64_t *mem_id = reinterpret_cast<int64_t *>(dyn + L.mem_id);
     int64_t *mem_dl = reinterpret_cast<int64_t *>(dyn + L.mem_dl);
+    int64_t *mem_delta = reinterpret_cast<int64_t *>(dyn + L.mem_delta);   // relative deadlines (soft penalties only)
     double *cand_u = reinterpret_cast<double *>(dyn + L.cand_u);
     int64_t *cand_e = reinterpret_cast<int64_t *>(dyn + L.cand_e);
     int *cand_bp = reinterpret_cast<int *>(dyn + L.cand_bp);
@@ -413,49 +435,62 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
             s_emin[a] = emin;
         }
         __syncthreads();
-        {
-            // The queues are sorted by deadline, so the late requests of a queue are a prefix.  Every application
-            // gets NT / A threads that look at the head of its queue at once (one memory round trip); only a queue
-            // whose whole window is late continues with a binary search behind it.
+        for (int pass = 0; pass < max_iter; ++pass) {
+            // The hopeless requests at the head of a queue are retired.  Every application gets NT / A threads that
+            // look at the head of its queue at once (one memory round trip).  Step penalty: the queue is sorted by
+            // deadline, so the hopeless requests are a prefix and a queue whose whole window is hopeless continues with
+            // a binary search behind it.  Soft penalties: hopeless also depends on the relative deadline, so such a
+            // queue is looked at again, window by window, until its head has utility left.
             const int per = NT / A, a = tid / per, j = tid - a * per;
             bool late = false;
             if (a < A) {
                 const int k = st.head[a] + j;
-                late = k < st.tail[a] && (sp.q_dl[st.cur[a]] + tb.gstart[(int64_t)inst * A + a])[k] < s_emin[a];
+                if (k < st.tail[a]) {
+                    const int64_t gb = tb.gstart[(int64_t)inst * A + a];
+                    const int64_t dl = sp.q_dl[st.cur[a]][gb + k];
+                    const int kind = P.pen[a];
+                    const int64_t delta = kind == SP_PEN_STEP ? 0 : dl - tb.arrival[sp.q_id[st.cur[a]][gb + k]];
+                    late = penalty_hopeless(kind, dl, delta, s_emin[a]);
+                }
             }
             const unsigned bal = __ballot_sync(0xffffffffu, late);
             if (lane == 0) s_ballot[warp] = bal;
-        }
-        __syncthreads();
-        if (tid < A) {
-            const int a = tid, per = NT / A, head = st.head[a], tail = st.tail[a];
-            int cnt = 0;                      // leading late requests inside the window
-            for (int j = 0; j < per; ++j) {
-                const int t2 = a * per + j;
-                if (!((s_ballot[t2 >> 5] >> (t2 & 31)) & 1u)) break;
-                ++cnt;
+            if (tid == 0) s_again = 0;
+            __syncthreads();
+            if (tid < A) {
+                const int a2 = tid, head = st.head[a2], tail = st.tail[a2];
+                int cnt = 0;                      // leading hopeless requests inside the window
+                for (int j2 = 0; j2 < per; ++j2) {
+                    const int t2 = a2 * per + j2;
+                    if (!((s_ballot[t2 >> 5] >> (t2 & 31)) & 1u)) break;
+                    ++cnt;
+                }
+                int nh = head + cnt;
+                if (cnt == per && nh < tail) {
+                    if (P.pen[a2] == SP_PEN_STEP) {
+                        const int64_t *dl = sp.q_dl[st.cur[a2]] + tb.gstart[(int64_t)inst * A + a2];
+                        int lo = nh, hi = tail;
+                        while (lo < hi) { const int mid = (lo + hi) >> 1; if (dl[mid] < s_emin[a2]) lo = mid + 1; else hi = mid; }
+                        nh = lo;
+                    } else s_again = 1;
+                }
+                s_newhead[a2] = nh;
             }
-            int nh = head + cnt;
-            if (cnt == per && nh < tail) {
-                const int64_t *dl = sp.q_dl[st.cur[a]] + tb.gstart[(int64_t)inst * A + a];
-                int lo = nh, hi = tail;
-                while (lo < hi) { const int mid = (lo + hi) >> 1; if (dl[mid] < s_emin[a]) lo = mid + 1; else hi = mid; }
-                nh = lo;
+            __syncthreads();
+            for (int a2 = 0; a2 < A; ++a2) {
+                const int64_t *qid = sp.q_id[st.cur[a2]] + tb.gstart[(int64_t)inst * A + a2];
+                for (int k = st.head[a2] + tid; k < s_newhead[a2]; k += NT) {
+                    sp_req_rec r; r.status = SP_EXPIRED; r.round = st.round; r.model = -1; r.pad_ = 0; r.order = 0;
+                    tb.recs[qid[k]] = r;
+                }
             }
-            s_newhead[a] = nh;
+            __syncthreads();
+            const int again = s_again;
+            if (tid == 0)
+                for (int a2 = 0; a2 < A; ++a2) { st.exp_since += s_newhead[a2] - st.head[a2]; st.head[a2] = s_newhead[a2]; }
+            __syncthreads();
+            if (!again) break;
         }
-        __syncthreads();
-        for (int a = 0; a < A; ++a) {
-            const int64_t *qid = sp.q_id[st.cur[a]] + tb.gstart[(int64_t)inst * A + a];
-            for (int k = st.head[a] + tid; k < s_newhead[a]; k += NT) {
-                sp_req_rec r; r.status = SP_EXPIRED; r.round = st.round; r.model = -1; r.pad_ = 0; r.order = 0;
-                tb.recs[qid[k]] = r;
-            }
-        }
-        __syncthreads();
-        if (tid == 0)
-            for (int a = 0; a < A; ++a) { st.exp_since += s_newhead[a] - st.head[a]; st.head[a] = s_newhead[a]; }
-        __syncthreads();
         live = 0;
         for (int a = 0; a < A; ++a) live += st.tail[a] - st.head[a];
         if (live == 0) continue;
@@ -537,7 +572,9 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
         for (int k = tid; k < nb; k += NT) {
             mem_id[k] = sp.q_id[c][base + head + k];
             mem_dl[k] = sp.q_dl[c][base + head + k];
+            if (P.pen[a] != SP_PEN_STEP) mem_delta[k] = mem_dl[k] - tb.arrival[mem_id[k]];
         }
+        const int pen = P.pen[a];
         __syncthreads();
         for (int k = tid; k < nb * Mmax; k += NT) {
             const int r = k / Mmax, j = k - r * Mmax;
@@ -568,10 +605,19 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
             const bool valid = bi == 0 || P.batch[bi - 1] < na;   // a larger size with the same members never wins
             const int bp = b < na ? b : na;
             const int64_t e = st.T + (g != st.L ? sw[g] : 0) + al[g] + be[g] * (int64_t)bp;
-            int lo = 0, hi = bp;                                   // members with deadline < e are late
-            while (lo < hi) { const int mid = (lo + hi) >> 1; if (mem_dl[mid] < e) lo = mid + 1; else hi = mid; }
-            const double *pj = pref + (size_t)j * (bmax + 1);
-            cand_u[ci] = valid ? pj[bp] - pj[lo] : -INFINITY;
+            double u;
+            if (pen == SP_PEN_STEP) {
+                int lo = 0, hi = bp;                               // members with deadline < e are late
+                while (lo < hi) { const int mid = (lo + hi) >> 1; if (mem_dl[mid] < e) lo = mid + 1; else hi = mid; }
+                const double *pj = pref + (size_t)j * (bmax + 1);
+                u = pj[bp] - pj[lo];
+            } else {                                               // Eq. 2 member by member: acc * (1 - gamma)
+                u = 0.0;
+                if (valid)
+                    for (int k = 0; k < bp; ++k)
+                        u = __dadd_rn(u, __dmul_rn((double)accs[k * Mmax + j], __dsub_rn(1.0, penalty_gamma(pen, mem_dl[k], mem_delta[k], e))));
+            }
+            cand_u[ci] = valid ? u : -INFINITY;
             cand_e[ci] = e; cand_bp[ci] = bp;
         }
         __syncthreads();
@@ -591,8 +637,10 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
                     const int j = ci / nB, bp = cand_bp[ci];
                     const int64_t e = cand_e[ci];
                     u = 0.0;
-                    for (int k = 0; k < bp; ++k)
-                        if (!(mem_dl[k] < e)) u = __dadd_rn(u, tb.acc64[mem_id[k] * Mmax + j]);
+                    for (int k = 0; k < bp; ++k) {
+                        if (pen == SP_PEN_STEP) { if (!(mem_dl[k] < e)) u = __dadd_rn(u, tb.acc64[mem_id[k] * Mmax + j]); }
+                        else u = __dadd_rn(u, __dmul_rn(tb.acc64[mem_id[k] * Mmax + j], __dsub_rn(1.0, penalty_gamma(pen, mem_dl[k], mem_delta[k], e))));
+                    }
                 }
                 cand_u[ci] = u;
             }

@@ -267,3 +267,19 @@ def test_short_circuit_candidate(name, kw, tight):
     check_schedule(w, res, od)
     if tight:
         assert np.all(res.reqs["status"] == 1) and np.all(res.rounds[0, :int(res.n_rounds[0])]["t_end_ns"] == w.t0_ns[0])
+
+
+@pytest.mark.parametrize("name,kw,kinds,guards", [
+    ("C1", {}, [1, 1, 1], None), ("C1", {}, [2, 2, 2], None), ("C2", {}, [2, 0, 1], None),
+    ("C4", dict(n_instances=8), [0, 1, 2], None), ("C5", dict(n_requests=6000), [2, 2, 2], None),
+    ("C1", {}, [2, 1, 0], (1.0, 1.0)), ("C3", dict(n_requests=1500), [1, 2, 0], None)])
+def test_linear_and_sigmoid_penalties(name, kw, kinds, guards):
+    """Section 5.1's soft penalties (utility degrades after the deadline over the relative deadline), per application;
+    with guards of 1.0 every decision also goes through the fp64 re-evaluation."""
+    w = synth.make_workload(name, **kw)
+    w.penalty_kind = np.asarray(kinds, dtype=np.int32)
+    s, od, res = _both(w, guards=guards)
+    check_scores(res, s)
+    check_schedule(w, res, od)
+    late = od.reqs["status"] == 1
+    assert late.any()
