@@ -43,7 +43,7 @@ constexpr int kGBProducerWarp = 0, kGMmaWarp = 1, kGAWarp0 = 2, kGEpiWarp0 = 6;
 constexpr int kGThreads = 32 * 14;
 constexpr int kGAThreads = 128, kGEpiThreads = 256;
 constexpr int kMergeFloats = 2 + kMaxModelsPerApp;    // running max, running sum, running sums per model
-constexpr int kGMaxStages = 3;
+constexpr int kGMaxA = 5, kGMaxB = 3;      // largest A / B ring of the two flavours
 
 template <bool F32>
 struct GCfg {
@@ -51,34 +51,43 @@ struct GCfg {
     static constexpr int KSlab = F32 ? 32 : 64;                // features per slab row (128 bytes)
     static constexpr int KStep = F32 ? 8 : 16;                 // features per MMA
     static constexpr int BSlabBytes = NC * 128 * (F32 ? 2 : 1);   // fp32: W_hi rows, then W_lo rows
-    static constexpr int StageBytes = kASlabBytes + ((BSlabBytes + 1023) & ~1023);
-    static constexpr int Stages = F32 ? 2 : 3;
+    static constexpr int BSlot = (BSlabBytes + 1023) & ~1023;
+    // The A slabs are gathered by threads (cp.async) and need several slabs in flight to cover the L2 latency; the B
+    // slabs come by TMA.  Separate rings let the small A slabs (16 KB) run deeper than the large B slabs.
+    static constexpr int AStages = F32 ? 3 : 5;                // fp32: one x_lo slot of tensor memory per A stage (3 x 32 columns)
+    static constexpr int BStages = F32 ? 2 : 3;
+    // A slab is reported complete when ADepth newer slabs have been issued (cp.async completion is observed relative
+    // to newer groups); issuing needs free slots, so the ring is deeper than ADepth by the slabs the MMAs work on.
+    static constexpr int ADepth = F32 ? 1 : 2;
     static constexpr int RBytes = kMaxModelsPerApp * NC * 4;   // recall rows of a chunk
     static constexpr int BiasBytes = NC * 4;
     static constexpr int BiasSlot = (BiasBytes + 127) & ~127;     // TMA destinations are 128-byte aligned
     static_assert(RBytes % 128 == 0, "recall buffers must keep the 128-byte alignment of TMA destinations");
     static constexpr int TmemLo = 2 * NC;                      // fp32: x_lo slots (32 columns per stage) after the accumulators
     // byte offsets from the 1024-byte aligned base
-    static constexpr int stages = 0;                                          // [Stages][A slab | B slab]
-    static constexpr int rtab = stages + Stages * StageBytes;                 // [2][16][NC] floats
+    static constexpr int a_ring = 0;                                          // [AStages] slabs of 128 rows
+    static constexpr int b_ring = a_ring + AStages * kASlabBytes;             // [BStages] slabs of NC (x 2) rows
+    static constexpr int rtab = b_ring + BStages * BSlot;                     // [2][16][NC] floats
     static constexpr int bias = rtab + 2 * RBytes;                            // [2][NC] floats
     static constexpr int merge = bias + 2 * BiasSlot;                        // [128][kMergeFloats]
     static constexpr int bars = (merge + kGRows * kMergeFloats * 4 + 15) & ~15;
-    static constexpr int n_bars = 3 * kGMaxStages + 8 + 3;
+    static constexpr int n_bars = 2 * kGMaxA + 2 * kGMaxB + 8 + 3;
     static constexpr int misc = bars + n_bars * 8;
     static constexpr int end = misc + 16;
     static constexpr int bytes = end + 1024;
 };
 __device__ __forceinline__ constexpr int gbar_full_a(int s) { return s; }
-__device__ __forceinline__ constexpr int gbar_full_b(int s) { return kGMaxStages + s; }
-__device__ __forceinline__ constexpr int gbar_free(int s) { return 2 * kGMaxStages + s; }
-__device__ __forceinline__ constexpr int gbar_acc_full(int b) { return 3 * kGMaxStages + b; }
-__device__ __forceinline__ constexpr int gbar_acc_empty(int b) { return 3 * kGMaxStages + 2 + b; }
-__device__ __forceinline__ constexpr int gbar_r_full(int b) { return 3 * kGMaxStages + 4 + b; }
-__device__ __forceinline__ constexpr int gbar_r_free(int b) { return 3 * kGMaxStages + 6 + b; }
-constexpr int kGBarMergeReady = 3 * kGMaxStages + 8;
-constexpr int kGBarMergeDone = 3 * kGMaxStages + 9;
-constexpr int kGBarDrain = 3 * kGMaxStages + 10;
+__device__ __forceinline__ constexpr int gbar_free_a(int s) { return kGMaxA + s; }
+__device__ __forceinline__ constexpr int gbar_full_b(int s) { return 2 * kGMaxA + s; }
+__device__ __forceinline__ constexpr int gbar_free_b(int s) { return 2 * kGMaxA + kGMaxB + s; }
+constexpr int kGBar2 = 2 * kGMaxA + 2 * kGMaxB;
+__device__ __forceinline__ constexpr int gbar_acc_full(int b) { return kGBar2 + b; }
+__device__ __forceinline__ constexpr int gbar_acc_empty(int b) { return kGBar2 + 2 + b; }
+__device__ __forceinline__ constexpr int gbar_r_full(int b) { return kGBar2 + 4 + b; }
+__device__ __forceinline__ constexpr int gbar_r_free(int b) { return kGBar2 + 6 + b; }
+constexpr int kGBarMergeReady = kGBar2 + 8;
+constexpr int kGBarMergeDone = kGBar2 + 9;
+constexpr int kGBarDrain = kGBar2 + 10;
 
 struct GParams {
     DevProfiles P;
@@ -172,7 +181,7 @@ __global__ void __launch_bounds__(kGThreads, 1)
 k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__ CUtensorMap r_map,
              const __grid_constant__ CUtensorMap b_map, const GParams prm) {
     using G = GCfg<F32>;
-    constexpr int kNC = G::NC, kKSlab = G::KSlab, kGStages = G::Stages, kStageBytes = G::StageBytes;
+    constexpr int kNC = G::NC, kKSlab = G::KSlab, kAStages = G::AStages, kBStages = G::BStages;
     constexpr int kBSlabBytes = G::BSlabBytes, kRBytes = G::RBytes, kBiasBytes = G::BiasBytes;
     using GSmem = G;
     extern __shared__ unsigned char smem_raw[];
@@ -191,9 +200,8 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
     const int n_ch = (C + kNC - 1) / kNC;                  // label chunks
 
     if (tid == 0) {
-        for (int s = 0; s < kGStages; ++s) {
-            mbar_init(bar(gbar_full_a(s)), kGAThreads); mbar_init(bar(gbar_full_b(s)), 1); mbar_init(bar(gbar_free(s)), 1);
-        }
+        for (int s = 0; s < kAStages; ++s) { mbar_init(bar(gbar_full_a(s)), kGAThreads); mbar_init(bar(gbar_free_a(s)), 1); }
+        for (int s = 0; s < kBStages; ++s) { mbar_init(bar(gbar_full_b(s)), 1); mbar_init(bar(gbar_free_b(s)), 1); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar(gbar_acc_full(b)), 1); mbar_init(bar(gbar_acc_empty(b)), kGEpiThreads);
             mbar_init(bar(gbar_r_full(b)), 1); mbar_init(bar(gbar_r_free(b)), kGEpiThreads);
@@ -236,11 +244,11 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
                     tma_load_2d(base + GSmem::rtab + rb * kRBytes, &r_map, ch * kNC, inst * P.sumM + P.mfirst[a], bar(gbar_r_full(rb)));
                     tma_load_2d(base + GSmem::bias + rb * G::BiasSlot, &b_map, ch * kNC, d.x, bar(gbar_r_full(rb)));
                     for (int ks = 0; ks < n_ks; ++ks, ++slab_seq) {
-                        const int s = slab_seq % kGStages;
-                        const uint32_t use = slab_seq / kGStages;
-                        if (use > 0 && !mbar_wait(bar(gbar_free(s)), (use - 1) & 1, abort_flag)) { ok = false; break; }
+                        const int s = slab_seq % kBStages;
+                        const uint32_t use = slab_seq / kBStages;
+                        if (use > 0 && !mbar_wait(bar(gbar_free_b(s)), (use - 1) & 1, abort_flag)) { ok = false; break; }
                         mbar_arrive_expect_tx(bar(gbar_full_b(s)), kBSlabBytes);
-                        const uint32_t bdst = base + GSmem::stages + s * kStageBytes + kASlabBytes;
+                        const uint32_t bdst = base + GSmem::b_ring + s * G::BSlot;
                         tma_load_2d(bdst, &wt_map, ks * kKSlab, wrow0 + ch * kNC, bar(gbar_full_b(s)));
                         if (F32) tma_load_2d(bdst + kNC * 128, &wt_map, ks * kKSlab, prm.lo_row0 + wrow0 + ch * kNC, bar(gbar_full_b(s)));
                     }
@@ -263,13 +271,12 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
                     const uint32_t idesc = F32 ? instr_desc(ncols) : instr_desc_bf16(ncols);
                     const uint32_t d_tmem = b * kNC;
                     for (int ks = 0; ks < n_ks; ++ks, ++slab_seq) {
-                        const int s = slab_seq % kGStages;
-                        const uint32_t par = (slab_seq / kGStages) & 1;
-                        if (!mbar_wait(bar(gbar_full_a(s)), par, abort_flag)) { ok = false; break; }
-                        if (!mbar_wait(bar(gbar_full_b(s)), par, abort_flag)) { ok = false; break; }
+                        const int s = slab_seq % kAStages, sb = slab_seq % kBStages;
+                        if (!mbar_wait(bar(gbar_full_a(s)), (slab_seq / kAStages) & 1, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(bar(gbar_full_b(sb)), (slab_seq / kBStages) & 1, abort_flag)) { ok = false; break; }
                         tc_fence_after();
-                        const uint64_t a_desc = smem_desc(base + GSmem::stages + s * kStageBytes);
-                        const uint64_t b_desc = smem_desc(base + GSmem::stages + s * kStageBytes + kASlabBytes);
+                        const uint64_t a_desc = smem_desc(base + GSmem::a_ring + s * kASlabBytes);
+                        const uint64_t b_desc = smem_desc(base + GSmem::b_ring + sb * G::BSlot);
                         if (F32) {
                             const uint64_t bl_desc = b_desc + (uint64_t)((kNC * 128) >> 4);      // W_lo rows
                             const uint32_t a_lo = (uint32_t)(G::TmemLo + s * 32);                  // x_lo of this stage
@@ -284,7 +291,8 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
                             for (int k = 0; k < kKSlab / 16; ++k)
                                 umma_bf16(d_tmem, a_desc + (uint64_t)(k * 2), b_desc + (uint64_t)(k * 2), idesc, (ks | k) != 0);
                         }
-                        umma_commit(bar(gbar_free(s)));
+                        umma_commit(bar(gbar_free_a(s)));
+                        umma_commit(bar(gbar_free_b(sb)));
                     }
                     if (ok) umma_commit(bar(gbar_acc_full(b)));
                 }
@@ -301,12 +309,12 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
         constexpr int kEsz = F32 ? 4 : 2, kPiece = 16 / kEsz; // bytes per feature, features per 16-byte piece
         uint32_t slab_seq = 0;
         bool ok = true;
-        int pending = -1;                                      // stage whose copies are issued but not signalled
+        uint32_t issued = 0, signalled = 0;                    // slabs whose copies were issued / reported complete
         // The copies of stage ps have landed: (fp32) store this row's x_lo into the stage's tensor-memory slot, then
         // tell the MMA issuer that the A operand of the stage is complete.
         auto signal = [&](int ps) {
             if (F32) {
-                const unsigned char *xrow = sm + GSmem::stages + ps * kStageBytes + row * 128;
+                const unsigned char *xrow = sm + GSmem::a_ring + ps * kASlabBytes + row * 128;
                 uint32_t v[32];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
@@ -333,10 +341,10 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
             const unsigned char *src = (const unsigned char *)tb.feats + req * D * kEsz;
             for (int ch = 0; ch < n_ch && ok; ++ch) {
                 for (int ks = 0; ks < n_ks; ++ks, ++slab_seq) {
-                    const int s = slab_seq % kGStages;
-                    const uint32_t use = slab_seq / kGStages;
-                    if (use > 0 && !warp_wait(bar(gbar_free(s)), (use - 1) & 1, abort_flag)) { ok = false; break; }
-                    const uint32_t dst = base + GSmem::stages + s * kStageBytes + row * 128;
+                    const int s = slab_seq % kAStages;
+                    const uint32_t use = slab_seq / kAStages;
+                    if (use > 0 && !warp_wait(bar(gbar_free_a(s)), (use - 1) & 1, abort_flag)) { ok = false; break; }
+                    const uint32_t dst = base + GSmem::a_ring + s * kASlabBytes + row * 128;
                     const int k0 = ks * kKSlab;
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
@@ -346,16 +354,17 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
                                          left >= 16 ? 16u : left > 0 ? (uint32_t)left : 0u);
                     }
                     cp_async_commit();
-                    if (pending >= 0) {                        // the copies of the previous slab have landed by now
-                        cp_async_wait<1>();
-                        signal(pending);
+                    ++issued;
+                    if (issued - signalled > (uint32_t)G::ADepth) {    // keep ADepth slabs in flight: the oldest has landed
+                        cp_async_wait<G::ADepth>();
+                        signal((int)(signalled % kAStages));
+                        ++signalled;
                     }
-                    pending = s;
                 }
             }
         }
         cp_async_wait<0>();
-        if (pending >= 0 && ok) signal(pending);
+        while (ok && signalled < issued) { signal((int)(signalled % kAStages)); ++signalled; }
     } else {
         // ================================================================ epilogue warps (one row per thread, half the columns)
         const int eg = (warp - kGEpiWarp0) >> 2;               // column half of every chunk this group reads
