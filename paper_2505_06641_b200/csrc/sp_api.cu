@@ -14,6 +14,7 @@
 #include "sp_score_gemm.cuh"
 #include "sp_sched.cuh"
 #include "sp_sched_warp.cuh"
+#include "sp_presort.cuh"
 
 using namespace sp;
 
@@ -694,6 +695,30 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
             SP_TRY(launched(c, "k_sched_warp"));
             sp.only_unstarted = 1;
         }
+    }
+    // One large snapshot instance: its keys are sorted by the whole GPU first (k_sched would use one block for it).
+    if (P.I == 1 && !c->opt.trace_mode && !c->sched_started && c->tb.n > sort_cap && c->tb.n < ((int64_t)1 << 31)) {
+        const int64_t n = c->tb.n;
+        SortKey *keys = (SortKey *)c->sort_scratch.p;
+        k_presort_keys<<<(unsigned)((n + 255) / 256), 256, 0, c->stream>>>(c->tb, keys, n);
+        SP_TRY(launched(c, "k_presort_keys"));
+        const unsigned nblk = (unsigned)((n + kPresortChunk - 1) / kPresortChunk);
+        const size_t psm = (size_t)kPresortChunk * sizeof(SortKey);
+        SP_CUDA(c, cudaFuncSetAttribute(k_presort_local, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm));
+        k_presort_local<<<nblk, kPresortThreads, psm, c->stream>>>(keys, n, 2, kPresortChunk);
+        SP_TRY(launched(c, "k_presort_local"));
+        int64_t p2 = 1;
+        while (p2 < n) p2 <<= 1;
+        const int64_t n_pairs = p2 >> 1;
+        for (int64_t k = 2 * (int64_t)kPresortChunk; k <= p2; k <<= 1) {
+            for (int64_t j = k >> 1; j >= kPresortChunk; j >>= 1) {
+                k_presort_global<<<(unsigned)((n_pairs + 255) / 256), 256, 0, c->stream>>>(keys, n, k, j, n_pairs);
+                SP_TRY(launched(c, "k_presort_global"));
+            }
+            k_presort_local<<<nblk, kPresortThreads, psm, c->stream>>>(keys, n, k, k);
+            SP_TRY(launched(c, "k_presort_local"));
+        }
+        sp.presorted = 1;
     }
     c->sched_started = true;
     k_sched<<<P.I, c->sched_threads, L.end, c->stream>>>(sp);

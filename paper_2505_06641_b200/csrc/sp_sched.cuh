@@ -48,6 +48,7 @@ struct SchedParams {
     int bmax;                   // largest allowed batch size
     int zbuf_warps;             // zbuf rows per instance
     int only_unstarted;         // 1: k_sched runs after k_sched_warp and takes only what that kernel left (flags[2])
+    int presorted;              // 1: sort_scratch already holds the sorted keys of the whole (single) instance
 };
 
 __device__ __forceinline__ bool key_less(const SortKey &a, const SortKey &b) {
@@ -325,14 +326,17 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
         const int64_t nnew = arrived_upto - st.inserted;
         if (nnew > 0) {
             const int64_t ap = st.inserted;
+            const bool presorted = sp.presorted && ap == 0 && nnew == n_inst && nnew > sp.sort_cap;   // sorted by the whole GPU
             SortKey *keys = nnew <= sp.sort_cap ? smem_keys : sp.sort_scratch + r0 + ap;
-            for (int64_t t = tid; t < nnew; t += NT) {
-                const int64_t id = r0 + ap + t;
-                SortKey k; k.dl = tb.deadline[id]; k.id_rel = (int32_t)(ap + t); k.app = tb.app[id];
-                keys[t] = k;
+            if (!presorted) {
+                for (int64_t t = tid; t < nnew; t += NT) {
+                    const int64_t id = r0 + ap + t;
+                    SortKey k; k.dl = tb.deadline[id]; k.id_rel = (int32_t)(ap + t); k.app = tb.app[id];
+                    keys[t] = k;
+                }
+                __syncthreads();
+                block_sort(keys, (int)nnew);
             }
-            __syncthreads();
-            block_sort(keys, (int)nnew);
             if (tid <= A) {                   // first sorted position whose application is >= tid
                 int lo = 0, hi = (int)nnew;
                 while (lo < hi) { const int mid = (lo + hi) >> 1; if (keys[mid].app < tid) lo = mid + 1; else hi = mid; }

@@ -25,7 +25,8 @@ def _both(w, guards=None, **kw):
 CASES = [("C1", {}), ("C2", {}), ("C3", dict(n_requests=3000)), ("C4", dict(n_instances=40)),
          ("C5", dict(n_requests=20000)),
          ("C1", dict(n_requests=1)), ("C1", dict(n_requests=129)), ("C2", dict(n_requests=65)),
-         ("C4", dict(n_instances=3, n_requests=131)), ("C3", dict(n_requests=70, models=5))]
+         ("C4", dict(n_instances=3, n_requests=131)), ("C3", dict(n_requests=70, models=5)),
+         ("C2", dict(n_requests=20000)), ("C2", dict(n_requests=70001))]     # large snapshots: sorted by the whole GPU
 
 
 @pytest.mark.parametrize("name,kw", CASES)
