@@ -257,9 +257,8 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
     __shared__ double red[33];
     __shared__ double s_P[kMaxApps];
     __shared__ int s_seg[kMaxApps + 2];
-    __shared__ int s_newhead[kMaxApps];
     __shared__ int s_lstart[kMaxApps + 1];
-    __shared__ int s_again;
+    __shared__ int s_lo[kMaxApps], s_hi[kMaxApps], s_pdone[kMaxApps];
     __shared__ int64_t s_emin[kMaxApps];
     __shared__ unsigned s_ballot[32];
     __shared__ double s_part[32 * kMaxApps];
@@ -294,9 +293,12 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
     __syncthreads();
 
     const double tau = P.tau;
-    const int64_t *al = P.lat_alpha + (int64_t)inst * P.sumM;
-    const int64_t *be = P.lat_beta + (int64_t)inst * P.sumM;
-    const int64_t *sw = P.swap + (int64_t)inst * P.sumM;
+    __shared__ int64_t al[kMaxApps * kMaxModelsPerApp], be[kMaxApps * kMaxModelsPerApp], sw[kMaxApps * kMaxModelsPerApp];
+    for (int g = tid; g < P.sumM; g += NT) {  // this instance's latency and swap profile, read every round
+        al[g] = P.lat_alpha[(int64_t)inst * P.sumM + g];
+        be[g] = P.lat_beta[(int64_t)inst * P.sumM + g];
+        sw[g] = P.swap[(int64_t)inst * P.sumM + g];
+    }
     const int rounds_init = st.started == 2 ? st.handed : 0;   // rounds k_sched_warp ran in this call before handing over
     int rounds_done = rounds_init;
     __syncthreads();
@@ -437,63 +439,76 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
                 emin = e < emin ? e : emin;
             }
             s_emin[a] = emin;
+            s_lo[a] = st.head[a]; s_hi[a] = st.tail[a]; s_pdone[a] = st.tail[a] == st.head[a];
         }
         __syncthreads();
+        // The hopeless requests at the head of every queue are retired.  Each application gets per = NT / A threads
+        // that look at per queue positions at once (one memory round trip per pass):
+        //   - window: the next per positions behind lo; the leading hopeless ones are counted.  Soft penalties only
+        //     ever use windows (hopeless depends on the relative deadline too, so it is not a sorted prefix) and slide
+        //     the window while it is hopeless throughout.
+        //   - samples (step penalty, after a first window that was hopeless throughout, more than per positions left):
+        //     the queue is sorted by deadline, so the hopeless requests are a prefix; per evenly spaced samples narrow
+        //     [lo, hi) by a factor per + 1 per pass.
         for (int pass = 0; pass < max_iter; ++pass) {
-            // The hopeless requests at the head of a queue are retired.  Every application gets NT / A threads that
-            // look at the head of its queue at once (one memory round trip).  Step penalty: the queue is sorted by
-            // deadline, so the hopeless requests are a prefix and a queue whose whole window is hopeless continues with
-            // a binary search behind it.  Soft penalties: hopeless also depends on the relative deadline, so such a
-            // queue is looked at again, window by window, until its head has utility left.
             const int per = NT / A, a = tid / per, j = tid - a * per;
             bool late = false;
-            if (a < A) {
-                const int k = st.head[a] + j;
-                if (k < st.tail[a]) {
+            if (a < A && !s_pdone[a]) {
+                const int lo = s_lo[a], hi = s_hi[a], span = hi - lo, kind = P.pen[a];
+                const bool window = pass == 0 || kind != SP_PEN_STEP || span <= per;
+                const int k = window ? lo + j : lo + (int)(((int64_t)(j + 1) * span) / (per + 1));
+                if (k < hi) {
                     const int64_t gb = tb.gstart[(int64_t)inst * A + a];
                     const int64_t dl = sp.q_dl[st.cur[a]][gb + k];
-                    const int kind = P.pen[a];
                     const int64_t delta = kind == SP_PEN_STEP ? 0 : dl - tb.arrival[sp.q_id[st.cur[a]][gb + k]];
                     late = penalty_hopeless(kind, dl, delta, s_emin[a]);
                 }
             }
             const unsigned bal = __ballot_sync(0xffffffffu, late);
             if (lane == 0) s_ballot[warp] = bal;
-            if (tid == 0) s_again = 0;
             __syncthreads();
-            if (tid < A) {
-                const int a2 = tid, head = st.head[a2], tail = st.tail[a2];
-                int cnt = 0;                      // leading hopeless requests inside the window
-                for (int j2 = 0; j2 < per; ++j2) {
-                    const int t2 = a2 * per + j2;
-                    if (!((s_ballot[t2 >> 5] >> (t2 & 31)) & 1u)) break;
-                    ++cnt;
+            if (tid < A && !s_pdone[tid]) {
+                const int a2 = tid, lo = s_lo[a2], hi = s_hi[a2], span = hi - lo, kind = P.pen[a2];
+                const bool window = pass == 0 || kind != SP_PEN_STEP || span <= per;
+                int cnt = 0;                      // leading hopeless positions among the per looked at
+                for (int t2 = a2 * per, end = t2 + per; t2 < end;) {
+                    const unsigned clear = ~(s_ballot[t2 >> 5] >> (t2 & 31));
+                    const int avail = min(32 - (t2 & 31), end - t2), run = clear ? __ffs(clear) - 1 : 32;
+                    if (run < avail) { cnt += run; break; }
+                    cnt += avail; t2 += avail;
                 }
-                int nh = head + cnt;
-                if (cnt == per && nh < tail) {
-                    if (P.pen[a2] == SP_PEN_STEP) {
-                        const int64_t *dl = sp.q_dl[st.cur[a2]] + tb.gstart[(int64_t)inst * A + a2];
-                        int lo = nh, hi = tail;
-                        while (lo < hi) { const int mid = (lo + hi) >> 1; if (dl[mid] < s_emin[a2]) lo = mid + 1; else hi = mid; }
-                        nh = lo;
-                    } else s_again = 1;
+                if (window) {
+                    if (cnt == per && lo + per < hi) s_lo[a2] = lo + per;          // hopeless throughout: slide on
+                    else { s_lo[a2] = lo + cnt; s_pdone[a2] = 1; }
+                } else {                          // sample j2 sits at lo + (j2 + 1) span / (per + 1)
+                    const int below = cnt == 0 ? lo : lo + (int)(((int64_t)cnt * span) / (per + 1)) + 1;
+                    const int above = cnt == per ? hi : lo + (int)(((int64_t)(cnt + 1) * span) / (per + 1));
+                    s_lo[a2] = below; s_hi[a2] = above;
+                    if (below >= above) s_pdone[a2] = 1;
                 }
-                s_newhead[a2] = nh;
             }
             __syncthreads();
+            bool all_done = true;
+            for (int a2 = 0; a2 < A; ++a2) all_done = all_done && s_pdone[a2];
+            if (all_done) break;
+            __syncthreads();
+        }
+        int n_retired = 0;                    // s_lo is the new head of every queue
+        for (int a2 = 0; a2 < A; ++a2) n_retired += s_lo[a2] - st.head[a2];
+        if (n_retired > 0) {
             for (int a2 = 0; a2 < A; ++a2) {
                 const int64_t *qid = sp.q_id[st.cur[a2]] + tb.gstart[(int64_t)inst * A + a2];
-                for (int k = st.head[a2] + tid; k < s_newhead[a2]; k += NT) {
+                for (int k = st.head[a2] + tid; k < s_lo[a2]; k += NT) {
                     sp_req_rec r; r.status = SP_EXPIRED; r.round = st.round; r.model = -1; r.pad_ = 0; r.order = 0;
                     tb.recs[qid[k]] = r;
                 }
             }
             __syncthreads();
-            const int again = s_again;
-            if (tid == 0)
-                for (int a2 = 0; a2 < A; ++a2) { st.exp_since += s_newhead[a2] - st.head[a2]; st.head[a2] = s_newhead[a2]; }
+            if (tid == 0) {
+                for (int a2 = 0; a2 < A; ++a2) st.head[a2] = s_lo[a2];
+                st.exp_since += n_retired;
+            }
             __syncthreads();
-            if (!again) break;
         }
         live = 0;
         for (int a = 0; a < A; ++a) live += st.tail[a] - st.head[a];
