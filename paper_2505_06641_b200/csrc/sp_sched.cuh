@@ -73,8 +73,34 @@ __device__ void block_sort(SortKey *keys, int n) {
                     if (key_less(b, a)) { keys[i] = b; keys[partner] = a; }
                 }
             }
-            __syncthreads();
+            // A step with j <= 32 keeps every pair inside an aligned run of 64 keys, and pairs t .. t + 31 (one
+            // warp) cover exactly one such run: between two such steps the warp only has to wait for itself.
+            const int next_j = j > 1 ? (j >> 1) : k;              // first step of the next merge has j = k
+            if (j <= 32 && next_j <= 32 && (k < p2 || j > 1)) __syncwarp();
+            else __syncthreads();
         }
+    }
+}
+
+// Sort of a short key list by counting: the rank of a key is the number of keys that precede it (keys are
+// distinct).  G threads share the comparisons of one key, so every thread of the block works and the longest
+// dependent chain is n / G comparisons, where the sorting network above spends log^2 n steps on one or two warps.
+// keys and out hold n entries each and do not overlap; the caller synchronises before and after.
+__device__ void block_rank_sort(const SortKey *keys, SortKey *out, int n) {
+    const int NT = blockDim.x;
+    int G = 1;
+    while (G < 32 && G * 2 * n <= NT) G <<= 1;
+    const int r = threadIdx.x & (G - 1);
+    for (int q0 = 0; q0 < n; q0 += NT / G) {          // uniform trip count: the shuffles below need whole warps
+        const int q = q0 + threadIdx.x / G;
+        int cnt = 0;
+        SortKey mine; mine.dl = 0; mine.id_rel = 0; mine.app = 0;
+        if (q < n) {
+            mine = keys[q];
+            for (int m = r; m < n; m += G) cnt += key_less(keys[m], mine) ? 1 : 0;
+        }
+        for (int o = G >> 1; o >= 1; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+        if (q < n && r == 0) out[cnt] = mine;
     }
 }
 
@@ -337,7 +363,13 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
                     keys[t] = k;
                 }
                 __syncthreads();
-                block_sort(keys, (int)nnew);
+                // short lists: counting sort into the scratch of the candidate step, which is free here
+                SortKey *sorted = reinterpret_cast<SortKey *>(dyn + L.pref);
+                if (nnew <= sp.sort_cap && nnew * nnew <= 256 * (int64_t)NT && (size_t)nnew * (sizeof(SortKey) + sizeof(int)) <= L.end - L.pref) {
+                    block_rank_sort(keys, sorted, (int)nnew);
+                    keys = sorted;
+                    __syncthreads();
+                } else block_sort(keys, (int)nnew);
             }
             if (tid <= A) {                   // first sorted position whose application is >= tid
                 int lo = 0, hi = (int)nnew;
@@ -356,27 +388,11 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
                 s_lstart[A] = tot;
             }
             __syncthreads();
-            for (int t = tid; t < (int)nnew; t += NT) {      // new element: count live elements before it
-                const int a = keys[t].app, tl = t - s_seg[a];
-                const int64_t base = tb.gstart[(int64_t)inst * A + a];
-                const int head = st.head[a], tail = st.tail[a], nl = tail - head, c = st.cur[a];
-                const int64_t dl = keys[t].dl, idr = keys[t].id_rel, id = r0 + idr;
-                int lo = 0, buf = c;
-                if (nl > 0) {
-                    const int64_t *lid = sp.q_id[c] + base + head, *ldl = sp.q_dl[c] + base + head;
-                    int hi = nl;
-                    while (lo < hi) {
-                        const int mid = (lo + hi) >> 1;
-                        const int64_t md = ldl[mid];
-                        const bool less = md < dl || (md == dl && (lid[mid] - r0) < idr);
-                        if (less) lo = mid + 1; else hi = mid;
-                    }
-                    buf = 1 - c;
-                }
-                const int64_t pos = base + (nl > 0 ? head : tail) + tl + lo;
-                sp.q_id[buf][pos] = id; sp.q_dl[buf][pos] = dl;
-                sp.q_pw[buf][pos] = prio_weight((double)tb.v32[id], dl, st.Tref, tau);
-            }
+            // Few enough new keys: the live elements (which look their place up among the new keys in shared memory)
+            // also leave, for every new key, the number of live elements before it; the new keys then need no
+            // binary search of dependent loads through the live queue.  The scratch of the candidate step is free here.
+            int *live_before = reinterpret_cast<int *>(dyn + L.pref + (size_t)nnew * sizeof(SortKey));
+            const bool via_smem = nnew <= sp.sort_cap && (size_t)nnew * (sizeof(SortKey) + sizeof(int)) <= L.end - L.pref;
             for (int f = tid; f < s_lstart[A]; f += NT) {     // live element: count new elements before it
                 int a = 0;
                 while (f >= s_lstart[a + 1]) ++a;
@@ -385,6 +401,8 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
                 const int head = st.head[a], c = st.cur[a], d = 1 - c;
                 const SortKey *nk = keys + s_seg[a];
                 const int64_t lidk = sp.q_id[c][base + head + k], dl = sp.q_dl[c][base + head + k], idr = lidk - r0;
+                int64_t pdl = 0, pidr = 0;
+                if (via_smem && k > 0) { pdl = sp.q_dl[c][base + head + k - 1]; pidr = sp.q_id[c][base + head + k - 1] - r0; }
                 int lo = 0, hi = nn;
                 while (lo < hi) {
                     const int mid = (lo + hi) >> 1;
@@ -393,6 +411,45 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
                 }
                 const int64_t pos = base + head + k + lo;
                 sp.q_id[d][pos] = lidk; sp.q_dl[d][pos] = dl; sp.q_pw[d][pos] = sp.q_pw[c][base + head + k];
+                if (via_smem) {
+                    int plo = 0;                                  // new keys before the previous live element
+                    if (k > 0) {
+                        hi = lo;
+                        while (plo < hi) {
+                            const int mid = (plo + hi) >> 1;
+                            const bool less = nk[mid].dl < pdl || (nk[mid].dl == pdl && nk[mid].id_rel < pidr);
+                            if (less) plo = mid + 1; else hi = mid;
+                        }
+                    }
+                    for (int t = plo; t < lo; ++t) live_before[s_seg[a] + t] = k;
+                    if (k == st.tail[a] - head - 1)
+                        for (int t = lo; t < nn; ++t) live_before[s_seg[a] + t] = k + 1;
+                }
+            }
+            if (via_smem) __syncthreads();
+            for (int t = tid; t < (int)nnew; t += NT) {      // new element: count live elements before it
+                const int a = keys[t].app, tl = t - s_seg[a];
+                const int64_t base = tb.gstart[(int64_t)inst * A + a];
+                const int head = st.head[a], tail = st.tail[a], nl = tail - head, c = st.cur[a];
+                const int64_t dl = keys[t].dl, idr = keys[t].id_rel, id = r0 + idr;
+                int lo = 0, buf = c;
+                if (nl > 0) {
+                    if (via_smem) lo = live_before[t];
+                    else {
+                        const int64_t *lid = sp.q_id[c] + base + head, *ldl = sp.q_dl[c] + base + head;
+                        int hi = nl;
+                        while (lo < hi) {
+                            const int mid = (lo + hi) >> 1;
+                            const int64_t md = ldl[mid];
+                            const bool less = md < dl || (md == dl && (lid[mid] - r0) < idr);
+                            if (less) lo = mid + 1; else hi = mid;
+                        }
+                    }
+                    buf = 1 - c;
+                }
+                const int64_t pos = base + (nl > 0 ? head : tail) + tl + lo;
+                sp.q_id[buf][pos] = id; sp.q_dl[buf][pos] = dl;
+                sp.q_pw[buf][pos] = prio_weight((double)tb.v32[id], dl, st.Tref, tau);
             }
             __syncthreads();
             if (tid == 0) {
