@@ -266,6 +266,18 @@ def main():
                     "unit": "GB/s", "frac": achieved / peak if achieved else None, "traffic": traffic,
                     "algorithmic_bytes": bytes_per_launch, "kernel_ms": score_ms}
 
+    # ---- one scheduling round per call (launch, the round, synchronise): the latency a caller sees per decision
+    ses.score()
+    torch.cuda.synchronize()
+    single = []
+    for _ in range(min(21, max_rounds)):
+        t0 = time.perf_counter()
+        ses.schedule(1)
+        torch.cuda.synchronize()
+        single.append(time.perf_counter() - t0)
+    us_single_round_call = float(np.median(single[1:] or single)) * 1e6
+    api.sp_check(ses.ctx)
+
     # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
     e2e = None
     if not args.no_e2e:
@@ -307,6 +319,7 @@ def main():
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
             "extra": {"score_kernel_ms": score_ms, "sched_kernel_ms": sched_ms, "rounds_per_step": n_rounds_total,
                       "us_per_round_amortised": sched_ms * 1e3 / max(1, n_rounds_total),
+                      "us_single_round_call": us_single_round_call,
                       "exact_utility_rounds": st["exact_utility"], "exact_priority_rounds": st["exact_priority"],
                       "exact_rows": st["exact_rows"]},
         }

@@ -286,6 +286,7 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
     __shared__ int s_lstart[kMaxApps + 1];
     __shared__ int s_lo[kMaxApps], s_hi[kMaxApps], s_pdone[kMaxApps];
     __shared__ int64_t s_emin[kMaxApps];
+    __shared__ int64_t s_base[kMaxApps + 1];   // first table row of each application's queue of this instance
     __shared__ unsigned s_ballot[32];
     __shared__ double s_part[32 * kMaxApps];
     __shared__ int s_best_app, s_exactP, s_best_ci, s_nclose, s_maxbp;
@@ -316,9 +317,11 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
     const int64_t r0 = tb.gstart[(int64_t)inst * A], r1 = tb.gstart[(int64_t)(inst + 1) * A];
     const int64_t n_inst = r1 - r0;
     if (tid == 0) st = sp.state[inst];
+    if (tid <= A) s_base[tid] = tb.gstart[(int64_t)inst * A + tid];
     __syncthreads();
 
     const double tau = P.tau;
+    const int64_t reref_ns = tau > 1e8 ? INT64_MAX : (int64_t)(32.0 * tau * 1e9);   // exp((T - Tref)/tau) stays below e^32
     __shared__ int64_t al[kMaxApps * kMaxModelsPerApp], be[kMaxApps * kMaxModelsPerApp], sw[kMaxApps * kMaxModelsPerApp];
     for (int g = tid; g < P.sumM; g += NT) {  // this instance's latency and swap profile, read every round
         al[g] = P.lat_alpha[(int64_t)inst * P.sumM + g];
@@ -397,10 +400,11 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
                 int a = 0;
                 while (f >= s_lstart[a + 1]) ++a;
                 const int k = f - s_lstart[a], nn = s_seg[a + 1] - s_seg[a];
-                const int64_t base = tb.gstart[(int64_t)inst * A + a];
+                const int64_t base = s_base[a];
                 const int head = st.head[a], c = st.cur[a], d = 1 - c;
                 const SortKey *nk = keys + s_seg[a];
                 const int64_t lidk = sp.q_id[c][base + head + k], dl = sp.q_dl[c][base + head + k], idr = lidk - r0;
+                const double pwk = sp.q_pw[c][base + head + k];
                 int64_t pdl = 0, pidr = 0;
                 if (via_smem && k > 0) { pdl = sp.q_dl[c][base + head + k - 1]; pidr = sp.q_id[c][base + head + k - 1] - r0; }
                 int lo = 0, hi = nn;
@@ -410,7 +414,7 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
                     if (less) lo = mid + 1; else hi = mid;
                 }
                 const int64_t pos = base + head + k + lo;
-                sp.q_id[d][pos] = lidk; sp.q_dl[d][pos] = dl; sp.q_pw[d][pos] = sp.q_pw[c][base + head + k];
+                sp.q_id[d][pos] = lidk; sp.q_dl[d][pos] = dl; sp.q_pw[d][pos] = pwk;
                 if (via_smem) {
                     int plo = 0;                                  // new keys before the previous live element
                     if (k > 0) {
@@ -429,7 +433,7 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
             if (via_smem) __syncthreads();
             for (int t = tid; t < (int)nnew; t += NT) {      // new element: count live elements before it
                 const int a = keys[t].app, tl = t - s_seg[a];
-                const int64_t base = tb.gstart[(int64_t)inst * A + a];
+                const int64_t base = s_base[a];
                 const int head = st.head[a], tail = st.tail[a], nl = tail - head, c = st.cur[a];
                 const int64_t dl = keys[t].dl, idr = keys[t].id_rel, id = r0 + idr;
                 int lo = 0, buf = c;
@@ -476,9 +480,9 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
             break;
         }
         // keep exp((T - Tref)/tau) in range: re-reference the stored priority weights now and then
-        if ((double)(st.T - st.Tref) * 1e-9 / tau > 32.0) {
+        if (st.T - st.Tref > reref_ns) {
             for (int a = 0; a < A; ++a) {
-                const int64_t base = tb.gstart[(int64_t)inst * A + a];
+                const int64_t base = s_base[a];
                 const int c = st.cur[a];
                 for (int k = st.head[a] + tid; k < st.tail[a]; k += NT)
                     sp.q_pw[c][base + k] = prio_weight((double)tb.v32[sp.q_id[c][base + k]], sp.q_dl[c][base + k], st.T, tau);
@@ -515,7 +519,7 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
                 const bool window = pass == 0 || kind != SP_PEN_STEP || span <= per;
                 const int k = window ? lo + j : lo + (int)(((int64_t)(j + 1) * span) / (per + 1));
                 if (k < hi) {
-                    const int64_t gb = tb.gstart[(int64_t)inst * A + a];
+                    const int64_t gb = s_base[a];
                     const int64_t dl = sp.q_dl[st.cur[a]][gb + k];
                     const int64_t delta = kind == SP_PEN_STEP ? 0 : dl - tb.arrival[sp.q_id[st.cur[a]][gb + k]];
                     late = penalty_hopeless(kind, dl, delta, s_emin[a]);
@@ -554,7 +558,7 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
         for (int a2 = 0; a2 < A; ++a2) n_retired += s_lo[a2] - st.head[a2];
         if (n_retired > 0) {
             for (int a2 = 0; a2 < A; ++a2) {
-                const int64_t *qid = sp.q_id[st.cur[a2]] + tb.gstart[(int64_t)inst * A + a2];
+                const int64_t *qid = sp.q_id[st.cur[a2]] + s_base[a2];
                 for (int k = st.head[a2] + tid; k < s_lo[a2]; k += NT) {
                     sp_req_rec r; r.status = SP_EXPIRED; r.round = st.round; r.model = -1; r.pad_ = 0; r.order = 0;
                     tb.recs[qid[k]] = r;
@@ -578,7 +582,7 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
             for (int a = 0; a < kMaxApps; ++a) {
                 part[a] = 0.0;
                 if (a < A) {
-                    const double *pw = sp.q_pw[st.cur[a]] + tb.gstart[(int64_t)inst * A + a];
+                    const double *pw = sp.q_pw[st.cur[a]] + s_base[a];
                     for (int k = st.head[a] + tid; k < st.tail[a]; k += NT) part[a] += pw[k];
                 }
             }
@@ -618,7 +622,7 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
         if (s_exactP) {                        // near-tie between groups: decide on fp64 scores
             for (int a = 0; a < A; ++a) {
                 if (!s_contend[a]) continue;
-                const int64_t base = tb.gstart[(int64_t)inst * A + a];
+                const int64_t base = s_base[a];
                 const int c = st.cur[a];
                 exact_rows(sp, inst, sp.q_id[c] + base, st.head[a], st.tail[a]);
                 double part = 0.0;
@@ -641,7 +645,7 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
         }
         // ---------------------------------------------------------------- 4. candidates of the chosen group
         const int a = s_best_app;
-        const int64_t base = tb.gstart[(int64_t)inst * A + a];
+        const int64_t base = s_base[a];
         const int c = st.cur[a], head = st.head[a], na = st.tail[a] - head;
         const int nb = na < bmax ? na : bmax;
         const int m0 = P.mfirst[a], M = P.mfirst[a + 1] - m0, ncand = M * nB;
