@@ -72,7 +72,7 @@ struct Smem {                               // byte offsets from the 1024-byte a
 struct Params {
     DevProfiles P;
     DevTable tb;
-    const int4 *tiles;       // (instance, first request relative to the instance, rows, -)
+    const int4 *tiles;       // (instance, first request relative to the instance, rows, first request in the table)
     int n_tiles;             // entries in `tiles`; the valid ones come first, those past the end have instance -1
     float *acc_out;          // optional second destination of acc
     int *flags;
@@ -366,7 +366,7 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
                     bulk_load(base + Smem::wraw, (const float *)P.W + (int64_t)d.x * A * D * C, w_bytes, bar(kBarRawFull));
                     ++w_seq; cur_inst = d.x;
                 }
-                const int row0 = (int)(tb.gstart[(int64_t)d.x * A] + d.y);
+                const int row0 = d.w;
                 for (int s = 0; s < n_slabs; ++s, ++slab_seq) {
                     const int h = slab_seq % kXStages;
                     const uint32_t use = slab_seq / kXStages;
@@ -501,16 +501,17 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
                     const uint4 q = *reinterpret_cast<const uint4 *>(xrow + ((j ^ (crow & 7)) << 4));
                     v[4 * j] = q.x; v[4 * j + 1] = q.y; v[4 * j + 2] = q.z; v[4 * j + 3] = q.w;
                 }
+                uint32_t vlo[kSlabK];                          // remainders, computed while the slot may still be busy
+#pragma unroll
+                for (int k = 0; k < kSlabK; ++k) {
+                    const float x = __uint_as_float(v[k]);
+                    vlo[k] = __float_as_uint(x - tf32_part(x));
+                }
                 if (a_use > 0 && !warp_wait(bar(bar_a_free(l)), (a_use - 1) & 1, abort_flag)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t a_hi = ((uint32_t)(cquad * 32) << 16) + (uint32_t)(kTmemA + l * kSlotCols);
                 tmem_st32(a_hi, v);                            // read as x_hi: the unit drops the low mantissa bits
-#pragma unroll
-                for (int k = 0; k < kSlabK; ++k) {
-                    const float x = __uint_as_float(v[k]);
-                    v[k] = __float_as_uint(x - tf32_part(x));
-                }
-                tmem_st32(a_hi + kSlabK, v);
+                tmem_st32(a_hi + kSlabK, vlo);
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar(bar_a_ready(mg, l)));
@@ -530,6 +531,7 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
         int cur_inst = -1, pre_inst = -1;
         const int sumM = P.sumM, Mmax = P.Mmax;
         const int Cp = (C + 3) & ~3;                           // label stride of the tables in shared memory
+        const bool pair_st = (Mmax & 1) == 0 && ((uintptr_t)prm.acc_out & 7) == 0;
         // this instance's tables travel through registers so that the loads of the next instance are in flight
         // while the current one is processed
         float pre_rec[1024 / kEpiThreads], pre_bias = 0.f, pre_pdot[256 / kEpiThreads], pre_psum = 0.f;
@@ -550,20 +552,20 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
             }
             pre_inst = inst;
         };
-        // application of this thread's row in tile t (loaded one of the group's tiles ahead of its use)
-        auto load_app = [&](int t) -> int {
-            if (t >= t_end) return 0;
-            const int4 d = prm.tiles[t];
-            if (d.x < 0 || row >= d.z) return 0;
-            return tb.app[tb.gstart[(int64_t)d.x * A] + d.y + row];
-        };
-        int a_next = load_app(t_begin + eg);
-        for (int t = t_begin + eg; t < t_end; t += kEpiGroups) {
-            const int4 d = prm.tiles[t];
+        // Descriptors travel two of the group's tiles ahead and the application of this thread's row one tile ahead,
+        // so that no load of the loop waits for the result of another one issued in the same iteration.
+        const int t0 = t_begin + eg;
+        int4 d = t0 < t_end ? prm.tiles[t0] : make_int4(-1, 0, 0, 0);
+        int4 d_n = t0 + kEpiGroups < t_end ? prm.tiles[t0 + kEpiGroups] : make_int4(-1, 0, 0, 0);
+        int a_cur = (d.x >= 0 && row < d.z) ? tb.app[(int64_t)d.w + row] : 0;
+        for (int t = t0; t < t_end; t += kEpiGroups) {
             if (d.x < 0) break;                                // valid tiles form a prefix of the block's range
-            const int inst = d.x;
-            const int a = min(max(a_next, 0), A - 1);
-            a_next = load_app(t + kEpiGroups);
+            const int inst = d.x, rows = d.z;
+            const int64_t req = (int64_t)d.w + row;
+            const int a = min(max(a_cur, 0), A - 1);
+            a_cur = (d_n.x >= 0 && row < d_n.z) ? tb.app[(int64_t)d_n.w + row] : 0;
+            d = d_n;
+            d_n = t + 2 * kEpiGroups < t_end ? prm.tiles[t + 2 * kEpiGroups] : make_int4(-1, 0, 0, 0);
             if (inst != cur_inst) {
                 if (pre_inst != inst) fetch_tab(inst);
                 mbar_arrive(bar(bar_epi_a(eg)));
@@ -588,8 +590,7 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
                 cur_inst = inst;
                 if (inst + 1 < P.I) fetch_tab(inst + 1);
             }
-            const int64_t req = tb.gstart[(int64_t)inst * A] + d.y + row;
-            const bool valid = row < d.z;
+            const bool valid = row < rows;
             const uint32_t acc_use = (uint32_t)(t - t_begin) >> 1;      // earlier uses of accumulator eg
             if (!warp_wait(bar(bar_acc_full(eg)), acc_use & 1, abort_flag)) break;
             tc_fence_after();
@@ -632,28 +633,47 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
             float *dst = tb.acc32 + req * Mmax;
             float *dst2 = prm.acc_out ? prm.acc_out + req * Mmax : nullptr;
             float a0 = 0.f, s1 = 0.f, s2 = 0.f;
+            // two models per pass: their recall rows are loaded together and accumulate in four independent chains
 #pragma unroll 1
-            for (int j = 0; j < Mmax; ++j) {
-                float aj = 0.f;
-                if (j < M) {
-                    const float *rr = recall_s + (g0 + j) * Cp;
-                    float p0 = 0.f, p1 = 0.f;
+            for (int j = 0; j < Mmax; j += 2) {
+                float aj0 = 0.f, aj1 = 0.f;
+                const bool m0 = j < M, m1 = j + 1 < M;
+                if (m0) {
+                    const float *ra = recall_s + (g0 + j) * Cp, *rb = m1 ? ra + Cp : ra;
+                    float p0 = 0.f, p1 = 0.f, q0 = 0.f, q1 = 0.f;
 #pragma unroll
                     for (int c = 0; c < CT; c += 4)
                         if (c < C) {
-                            const float4 rv = *reinterpret_cast<const float4 *>(rr + c);
+                            const float4 rv = *reinterpret_cast<const float4 *>(ra + c);
+                            const float4 sv = *reinterpret_cast<const float4 *>(rb + c);
                             p0 = fmaf(z[c], rv.x, p0); p1 = fmaf(z[c + 1], rv.y, p1);
+                            q0 = fmaf(z[c], sv.x, q0); q1 = fmaf(z[c + 1], sv.y, q1);
                             p0 = fmaf(z[c + 2], rv.z, p0); p1 = fmaf(z[c + 3], rv.w, p1);
+                            q0 = fmaf(z[c + 2], sv.z, q0); q1 = fmaf(z[c + 3], sv.w, q1);
                         }
-                    aj = (p0 + p1) * inv;
-                    if (P.prior) aj = (pdot_s[g0 + j] + P.kappa * aj) / (psum_s[a] + P.kappa);
-                    if (j == 0) a0 = aj;
-                    const float dj = aj - a0;
-                    s1 += dj; s2 = fmaf(dj, dj, s2);
+                    aj0 = (p0 + p1) * inv;
+                    aj1 = (q0 + q1) * inv;
+                    if (P.prior) {
+                        aj0 = (pdot_s[g0 + j] + P.kappa * aj0) / (psum_s[a] + P.kappa);
+                        if (m1) aj1 = (pdot_s[g0 + j + 1] + P.kappa * aj1) / (psum_s[a] + P.kappa);
+                    }
+                    if (j == 0) a0 = aj0;
+                    const float d0 = aj0 - a0;
+                    s1 += d0; s2 = fmaf(d0, d0, s2);
+                    if (m1) {
+                        const float d1 = aj1 - a0;
+                        s1 += d1; s2 = fmaf(d1, d1, s2);
+                    } else aj1 = 0.f;
                 }
                 if (valid) {
-                    dst[j] = aj;
-                    if (dst2) dst2[j] = aj;
+                    if (pair_st) {                             // rows of an even number of floats: 8-byte stores
+                        *reinterpret_cast<float2 *>(dst + j) = make_float2(aj0, aj1);
+                        if (dst2) *reinterpret_cast<float2 *>(dst2 + j) = make_float2(aj0, aj1);
+                    } else {
+                        dst[j] = aj0;
+                        if (j + 1 < Mmax) dst[j + 1] = aj1;
+                        if (dst2) { dst2[j] = aj0; if (j + 1 < Mmax) dst2[j + 1] = aj1; }
+                    }
                 }
             }
             if (valid) {

@@ -51,7 +51,9 @@ __device__ __forceinline__ void load_half_row(float (&w)[CT], const float *p) {
     if (CT % 2) w[CT - 1] = p[CT - 1];
 }
 
-// Tile descriptors: tile t -> (instance, first request relative to the instance, rows), instance = -1 past the end.
+// Tile descriptors: tile t -> (instance, first request relative to the instance, rows, first request in the table),
+// instance = -1 past the end.  The last component is only meaningful below 2^31 requests (the tensor-core kernel,
+// whose TMA coordinates are 32-bit, is the one that reads it).
 __global__ void k_small_tiles(DevProfiles P, DevTable tb, const int32_t *__restrict__ small_start, int n_tiles,
                               int4 *__restrict__ desc, const int *__restrict__ flags) {
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
@@ -62,7 +64,7 @@ __global__ void k_small_tiles(DevProfiles P, DevTable tb, const int32_t *__restr
         while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (small_start[mid] <= t) lo = mid; else hi = mid; }
         const int64_t i0 = tb.gstart[(int64_t)lo * P.A], i1 = tb.gstart[(int64_t)(lo + 1) * P.A];
         const int64_t r0 = (int64_t)(t - small_start[lo]) * kSmallRows;
-        d = make_int4(lo, (int)r0, (int)((i1 - i0 - r0) < kSmallRows ? (i1 - i0 - r0) : kSmallRows), 0);
+        d = make_int4(lo, (int)r0, (int)((i1 - i0 - r0) < kSmallRows ? (i1 - i0 - r0) : kSmallRows), (int)(i0 + r0));
     }
     desc[t] = d;
 }
