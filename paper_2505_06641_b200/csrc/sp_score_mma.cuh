@@ -12,7 +12,7 @@
 //     each row later keeps the columns of its own application, so rows need no regrouping;
 //   * fp32 accuracy from the tf32 unit: x = x_hi + x_lo and W = W_hi + W_lo with x_hi, W_hi the values
 //     truncated to tf32 (what the unit reads from a 32-bit container) and the remainders exact in fp32;
-//     z = x_hi [W_hi | W_lo] + x_lo W_hi accumulates in fp32 in tensor memory, the dropped x_lo W_lo term
+//     z = x_hi W_hi + x_hi W_lo + x_lo W_hi accumulates in fp32 in tensor memory, the dropped x_lo W_lo term
 //     is below 2^-20 relative;
 //   * shared-memory bandwidth is the scarce resource (every MMA re-reads its operands), so the A operand
 //     comes from tensor memory: converter warps (one row per thread) read each slab once, store the row as
@@ -39,9 +39,9 @@ constexpr int kMaxD = 128;
 constexpr int kMaxSlabs = kMaxD / kSlabK;
 constexpr int kCols = 64;                  // logit columns (sum over applications of the label count)
 constexpr int kXStages = 6;                // ring of slabs in shared memory filled by TMA
-constexpr int kASlots = 4;                 // ring of A operands in tensor memory: 32 columns x_hi + 32 columns x_lo each
+constexpr int kASlots = 6;                 // ring of A operands in tensor memory: 32 columns x_hi + 32 columns x_lo each
 constexpr int kTmemCols = 512;             // whole tensor memory
-constexpr int kAccCols = 128;              // columns per accumulator: [x_hi W_hi + x_lo W_hi | x_hi W_lo]
+constexpr int kAccCols = 64;               // columns per accumulator: x_hi W_hi + x_hi W_lo + x_lo W_hi, all applications
 constexpr int kTmemA = 2 * kAccCols;       // accumulators first (epilogue reads may overhang into the A ring), then the ring
 constexpr int kSlotCols = 2 * kSlabK;
 constexpr int kProducerWarp = 0, kMmaWarp = 1, kConvWarp0 = 2, kEpiWarp0 = 6;
@@ -395,7 +395,8 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
         // All tensor-memory addresses below are compile-time offsets: the allocation covers the whole tensor
         // memory, so its base is column 0 (checked after the allocation).
         if (lane == 0) {
-            constexpr uint32_t idesc_hi = instr_desc(2 * kCols), idesc_lo = instr_desc(kCols);
+            constexpr uint32_t idesc = instr_desc(kCols);
+            constexpr uint64_t w_lo_rows = (uint64_t)((kCols * 128) >> 4);   // operand rows 64..127 hold W_lo
             const uint64_t w_desc = smem_desc(base + Smem::w);
             const int mg = warp == kMmaWarp ? 0 : 1;
             bool ok = true;
@@ -421,11 +422,11 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
                     const uint32_t a_hi = kTmemA + l * kSlotCols, a_lo = a_hi + kSlabK;
                     const uint64_t b_w = w_desc + (uint64_t)((s * kSlabBytes) >> 4);
 #pragma unroll
-                    for (int k = 0; k < kSlabK / 8; ++k)       // x_hi [W_hi | W_lo] -> all 128 columns
-                        umma_tf32_ts(d_tmem, a_hi + k * 8, b_w + (uint64_t)(k * 2), idesc_hi, (s | k) != 0);
-#pragma unroll
-                    for (int k = 0; k < kSlabK / 8; ++k)       // x_lo W_hi -> the first 64 columns
-                        umma_tf32_ts(d_tmem, a_lo + k * 8, b_w + (uint64_t)(k * 2), idesc_lo, 1u);
+                    for (int k = 0; k < kSlabK / 8; ++k) {     // the three products accumulate in the same 64 columns
+                        umma_tf32_ts(d_tmem, a_hi + k * 8, b_w + (uint64_t)(k * 2), idesc, (s | k) != 0);
+                        umma_tf32_ts(d_tmem, a_hi + k * 8, b_w + w_lo_rows + (uint64_t)(k * 2), idesc, 1u);
+                        umma_tf32_ts(d_tmem, a_lo + k * 8, b_w + (uint64_t)(k * 2), idesc, 1u);
+                    }
                     umma_commit(bar(bar_a_free(l)));
                 }
                 if (ok) umma_commit(bar(bar_acc_full(b)));
@@ -466,10 +467,12 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
                 const int h = slab_seq % kXStages, l = slab_seq % kASlots;
                 const uint32_t a_use = slab_seq / kASlots;
                 if (new_inst) {
-                    if (slab_seq >= (uint32_t)n_slabs) {       // MMAs of the previous tile's slab s read the old operand
-                        const uint32_t ps = slab_seq - (uint32_t)n_slabs;
-                        if (!warp_wait(bar(bar_a_free(ps % kASlots)), (ps / kASlots) & 1, abort_flag)) { ok = false; break; }
-                    }
+                    // MMAs of earlier tiles on slab s read the old operand.  Slabs more than kASlots back have
+                    // completed (their slots were taken again, which waited for them); the younger ones with the
+                    // same s are waited for here, each on a barrier phase that cannot have been passed yet.
+                    for (int64_t ps = (int64_t)slab_seq - n_slabs; ps >= 0 && ps + kASlots >= (int64_t)slab_seq && ok; ps -= n_slabs)
+                        if (!warp_wait(bar(bar_a_free((int)(ps % kASlots))), (uint32_t)(ps / kASlots) & 1, abort_flag)) ok = false;
+                    if (!ok) break;
                     if (w_row) {
 #pragma unroll
                         for (int q = 0; q < 4; ++q) {
@@ -600,13 +603,12 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
             for (int c = 0; c < CT; ++c) z[c] = 0.f;
             for (int ap = 0; ap < A; ++ap) {
                 if (__ballot_sync(0xffffffffu, a == ap) == 0) continue;
-                float r1[CT], r2[CT];
+                float r1[CT];
                 tmem_ld<CT>(taddr + (uint32_t)(ap * C), r1);
-                tmem_ld<CT>(taddr + (uint32_t)(kCols + ap * C), r2);
                 tmem_wait_ld();
                 if (a == ap) {
 #pragma unroll
-                    for (int c = 0; c < CT; ++c) z[c] = r1[c] + r2[c];
+                    for (int c = 0; c < CT; ++c) z[c] = r1[c];
                 }
             }
             tc_fence_before();

@@ -26,7 +26,10 @@ CASES = [("C1", {}), ("C2", {}), ("C3", dict(n_requests=3000)), ("C4", dict(n_in
          ("C5", dict(n_requests=20000)),
          ("C1", dict(n_requests=1)), ("C1", dict(n_requests=129)), ("C2", dict(n_requests=65)),
          ("C4", dict(n_instances=3, n_requests=131)), ("C3", dict(n_requests=70, models=5)),
-         ("C2", dict(n_requests=20000)), ("C2", dict(n_requests=70001))]     # large snapshots: sorted by the whole GPU
+         ("C2", dict(n_requests=20000)), ("C2", dict(n_requests=70001)),     # large snapshots: sorted by the whole GPU
+         # many instances per block with 2 and 1 feature slabs per tile: the head operand is rebuilt at every instance
+         # change while tiles of the previous instance may still be in the tensor pipe
+         ("C4", dict(n_instances=700, feat_dim=64)), ("C4", dict(n_instances=700, n_requests=300, feat_dim=32))]
 
 
 @pytest.mark.parametrize("name,kw", CASES)
