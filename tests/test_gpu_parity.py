@@ -287,3 +287,28 @@ def test_linear_and_sigmoid_penalties(name, kw, kinds, guards):
     check_schedule(w, res, od)
     late = od.reqs["status"] == 1
     assert late.any()
+
+
+def _shape_cases():
+    """Seeded draws of small shapes around the limits of the scoring kernels (labels, feature slabs, model counts)."""
+    rng = np.random.default_rng(2024)
+    cases = []
+    for k in range(14):
+        base = ["C4", "C1", "C2"][k % 3]
+        kw = dict(n_apps=int(rng.integers(1, 5)), models=int(rng.integers(1, 7)),
+                  n_classes=int(rng.choice([3, 5, 8, 10, 12, 16, 20, 21, 32, 40])),
+                  feat_dim=int(rng.choice([32, 64, 96, 128, 160, 256])), n_requests=int(rng.integers(1, 700)))
+        if base == "C4":
+            kw["n_instances"] = int(rng.choice([2, 37, 400]))
+            kw["n_requests"] = int(rng.integers(1, 300))
+        cases.append((base, kw))
+    return cases
+
+
+@pytest.mark.parametrize("name,kw", _shape_cases())
+def test_random_shapes_match_oracle(name, kw):
+    w = synth.make_workload(name, **kw)
+    s, od, res = _both(w)
+    worst = check_scores(res, s)
+    check_schedule(w, res, od)
+    assert worst < ACC_RTOL
