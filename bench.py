@@ -328,7 +328,7 @@ def main():
         dist.destroy_process_group()
 
 
-KERNEL_VERSION = 4     # bump when the scoring kernel changes: stale ncu traffic figures are then ignored
+KERNEL_VERSION = 5     # bump when the scoring kernel changes: stale ncu traffic figures are then ignored
 
 
 if __name__ == "__main__":
