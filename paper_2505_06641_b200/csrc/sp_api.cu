@@ -338,7 +338,7 @@ sp_status sp_load_profiles(sp_ctx *c, const sp_profiles *p) {
     }
     // shared memory the scheduler kernel needs for its candidate tables (sort buffer is sized at launch)
     const int bmax = p->batch_sizes[nB - 1];
-    const SchedSmem ss(0, Mmax, bmax, kMaxModelsPerApp * kMaxBatchSizes);
+    const SchedSmem ss(0, Mmax, bmax, kMaxModelsPerApp * kMaxBatchSizes, sumM, 32);
     if (ss.end > 96 * 1024) return fail(c, SP_EINVAL, "models_per_app x largest batch size is too large for one block");
 
     c->have_profiles = false;
@@ -677,7 +677,7 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
     while (sort_cap > 64 && sort_cap / 2 >= per_inst) sort_cap /= 2;
     sp.sort_cap = sort_cap;
     sp.zbuf_warps = c->sched_threads / 32;
-    const SchedSmem L(sort_cap, P.Mmax, sp.bmax, kMaxModelsPerApp * kMaxBatchSizes);
+    const SchedSmem L(sort_cap, P.Mmax, sp.bmax, kMaxModelsPerApp * kMaxBatchSizes, P.sumM, c->sched_threads / 32);
     SP_CUDA(c, cudaFuncSetAttribute(k_sched, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.end));
     SP_TRY(mark(c, c->ev_sched));
     // Batched mode, first call on a fresh table: one warp per instance takes every instance that fits its slice of
@@ -686,14 +686,16 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
         int64_t wcap = 32;
         while (wcap < (c->tb.n + P.I - 1) / P.I) wcap <<= 1;
         const WarpSchedSmem W((int)wcap, P.Mmax, sp.bmax);
-        if (wcap <= 2048 && P.sumM <= 32 && W.end * kWarpSchedWarps <= 200 * 1024) {
+        if (wcap <= 2048 && P.sumM <= 32 && W.end * kWarpSchedWarps <= 200 * 1024 && c->sched_threads == kWarpSchedWarps * 32) {
             const int wgrid = (P.I + kWarpSchedWarps - 1) / kWarpSchedWarps;
-            const size_t wsmem = W.end * kWarpSchedWarps;
-            SP_CUDA(c, cudaMemsetAsync((int *)c->flags.p + 2, 0, sizeof(int), c->stream));
+            // the block-wide scheduler runs inside the same kernel for the instances a warp hands over: its shared
+            // memory is laid over the warps' slices
+            const size_t wsmem = W.end * kWarpSchedWarps > L.end ? W.end * kWarpSchedWarps : L.end;
             SP_CUDA(c, cudaFuncSetAttribute(k_sched_warp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)wsmem));
             k_sched_warp<<<wgrid, kWarpSchedWarps * 32, wsmem, c->stream>>>(sp, (int)wcap);
             SP_TRY(launched(c, "k_sched_warp"));
-            sp.only_unstarted = 1;
+            c->sched_started = true;
+            return mark(c, c->ev_sched);
         }
     }
     // One large snapshot instance: its keys are sorted by the whole GPU first (k_sched would use one block for it).

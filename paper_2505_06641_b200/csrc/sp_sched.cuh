@@ -47,7 +47,6 @@ struct SchedParams {
     int sort_cap;               // SortKey entries available in shared memory
     int bmax;                   // largest allowed batch size
     int zbuf_warps;             // zbuf rows per instance
-    int only_unstarted;         // 1: k_sched runs after k_sched_warp and takes only what that kernel left (flags[2])
     int presorted;              // 1: sort_scratch already holds the sorted keys of the whole (single) instance
 };
 
@@ -207,9 +206,12 @@ namespace sp {
 
 // Shared-memory carve-up of k_sched (bytes, 16-byte aligned pieces).
 struct SchedSmem {
-    size_t keys, pref, accs, mem_id, mem_dl, mem_delta, cand_u, cand_e, cand_bp, end;
-    __host__ __device__ SchedSmem(int sort_cap, int Mmax, int bmax, int ncand) {
+    size_t lat, part, keys, pref, accs, mem_id, mem_dl, mem_delta, cand_u, cand_e, cand_bp, end;
+    __host__ __device__ SchedSmem(int sort_cap, int Mmax, int bmax, int ncand, int sumM, int nwarps) {
         size_t o = 0;
+        lat = o;     o += (size_t)3 * sumM * sizeof(int64_t);                 // latency alpha, beta and swap of the instance
+        part = o;    o += (size_t)nwarps * kMaxApps * sizeof(double);          // per-warp partial priority sums
+        o = (o + 15) & ~(size_t)15;
         keys = o;    o += (size_t)sort_cap * sizeof(SortKey);
         pref = o;    o += (size_t)Mmax * (bmax + 1) * sizeof(double);
         mem_id = o;  o += (size_t)bmax * sizeof(int64_t);
@@ -277,7 +279,8 @@ __device__ __forceinline__ void warp_argmax(const double *cand_u, const int *can
     best = bi; best_u = bu; n_close = cnt; max_bp = mb;
 }
 
-__global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
+// All rounds of one instance by one thread block (every thread of the block calls it).
+__device__ void sched_instance(const SchedParams &sp, const int inst) {
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ InstState st;
     __shared__ double red[33];
@@ -288,7 +291,6 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
     __shared__ int64_t s_emin[kMaxApps];
     __shared__ int64_t s_base[kMaxApps + 1];   // first table row of each application's queue of this instance
     __shared__ unsigned s_ballot[32];
-    __shared__ double s_part[32 * kMaxApps];
     __shared__ int s_best_app, s_exactP, s_best_ci, s_nclose, s_maxbp;
     __shared__ double s_best_u, s_best_p;
     __shared__ unsigned char s_contend[kMaxApps];
@@ -296,9 +298,9 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
     const DevProfiles &P = sp.P;
     const DevTable &tb = sp.tb;
     const int tid = threadIdx.x, NT = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarps = NT >> 5;
-    const int inst = blockIdx.x, A = P.A, nB = P.nB, Mmax = P.Mmax, bmax = sp.bmax;
+    const int A = P.A, nB = P.nB, Mmax = P.Mmax, bmax = sp.bmax;
     const int ncand_max = kMaxModelsPerApp * kMaxBatchSizes;
-    const SchedSmem L(sp.sort_cap, Mmax, bmax, ncand_max);
+    const SchedSmem L(sp.sort_cap, Mmax, bmax, ncand_max, P.sumM, nwarps);
     SortKey *smem_keys = reinterpret_cast<SortKey *>(dyn + L.keys);
     double *pref = reinterpret_cast<double *>(dyn + L.pref);
     float *accs = reinterpret_cast<float *>(dyn + L.accs);
@@ -313,7 +315,6 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
         if (tid == 0 && sp.n_done) sp.n_done[inst] = 0;
         return;
     }
-    if (sp.only_unstarted && (!sp.flags[2] || sp.state[inst].started == 1)) return;   // the warp kernel has done it
     const int64_t r0 = tb.gstart[(int64_t)inst * A], r1 = tb.gstart[(int64_t)(inst + 1) * A];
     const int64_t n_inst = r1 - r0;
     if (tid == 0) st = sp.state[inst];
@@ -322,7 +323,8 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
 
     const double tau = P.tau;
     const int64_t reref_ns = tau > 1e8 ? INT64_MAX : (int64_t)(32.0 * tau * 1e9);   // exp((T - Tref)/tau) stays below e^32
-    __shared__ int64_t al[kMaxApps * kMaxModelsPerApp], be[kMaxApps * kMaxModelsPerApp], sw[kMaxApps * kMaxModelsPerApp];
+    int64_t *al = reinterpret_cast<int64_t *>(dyn + L.lat), *be = al + P.sumM, *sw = be + P.sumM;
+    double *s_part = reinterpret_cast<double *>(dyn + L.part);
     for (int g = tid; g < P.sumM; g += NT) {  // this instance's latency and swap profile, read every round
         al[g] = P.lat_alpha[(int64_t)inst * P.sumM + g];
         be[g] = P.lat_beta[(int64_t)inst * P.sumM + g];
@@ -765,5 +767,7 @@ __global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) {
         if (n_exact_p) atomicAdd(&sp.stats[2], n_exact_p);
     }
 }
+
+__global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) { sched_instance(sp, blockIdx.x); }
 
 }  // namespace sp

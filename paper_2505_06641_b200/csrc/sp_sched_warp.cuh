@@ -12,7 +12,7 @@
 // not contain the fp64 re-evaluation of near-ties (which keeps it small): when the two best group priorities or
 // candidate utilities of a round are closer than the guard band, the warp writes its queues and state out and
 // hands the instance to k_sched, which runs after this kernel in the same call and also takes the instances that
-// do not fit a warp (flags[2] tells it that there is work left).
+// do not fit a warp.
 #pragma once
 
 #include "sp_common.cuh"
@@ -80,17 +80,14 @@ __device__ __forceinline__ void warp_sort(int64_t *dl, uint32_t *ida, int n) {
     }
 }
 
-__global__ void __launch_bounds__(kWarpSchedWarps * 32)
-k_sched_warp(SchedParams sp, int cap) {
-    extern __shared__ __align__(16) unsigned char dyn[];
+// One instance by one warp.  Returns true when the block-wide scheduler has to take the instance over: a near-tie
+// to decide in fp64, more requests than the warp's slice holds, or an instance that had already started.
+__device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const int inst, unsigned char *mine) {
     const DevProfiles &P = sp.P;
     const DevTable &tb = sp.tb;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int inst = blockIdx.x * kWarpSchedWarps + warp;
-    if (inst >= P.I || sp.flags[1]) return;
+    const int lane = threadIdx.x & 31;
     const int A = P.A, nB = P.nB, Mmax = P.Mmax, bmax = sp.bmax, sumM = P.sumM;
     const WarpSchedSmem L(cap, Mmax, bmax);
-    unsigned char *mine = dyn + (size_t)warp * L.end;
     int64_t *s_dl = reinterpret_cast<int64_t *>(mine + L.dl);
     double *s_pw = reinterpret_cast<double *>(mine + L.pw);
     uint32_t *s_ida = reinterpret_cast<uint32_t *>(mine + L.ida);
@@ -99,11 +96,8 @@ k_sched_warp(SchedParams sp, int cap) {
     const int64_t r0 = tb.gstart[(int64_t)inst * A], r1 = tb.gstart[(int64_t)(inst + 1) * A];
     const int n_inst = (int)(r1 - r0);
     InstState *stp = &sp.state[inst];
-    if (stp->started) return;                                         // not a fresh instance: k_sched resumes it
-    if (r1 - r0 > cap || r1 - r0 >= (1 << 24)) {                      // does not fit a warp: leave it to k_sched
-        if (lane == 0) sp.flags[2] = 1;
-        return;
-    }
+    if (stp->started) return true;                                    // not a fresh instance: the block resumes it
+    if (r1 - r0 > cap || r1 - r0 >= (1 << 24)) return true;           // does not fit a warp
     int64_t T = stp->T, next_order = stp->next_order;
     int64_t Tref = T;
     int Lm = stp->L, round = stp->round, exp_since = stp->exp_since;
@@ -360,9 +354,36 @@ k_sched_warp(SchedParams sp, int cap) {
         stp->T = T; stp->next_order = next_order; stp->Tref = Tref; stp->inserted = n_inst;
         stp->L = Lm; stp->round = round; stp->exp_since = exp_since; stp->started = handover ? 2 : 1;
         stp->handed = rounds_done;
-        if (handover) sp.flags[2] = 1;
         if (sp.n_done) sp.n_done[inst] = rounds_done;
         if (rounds_done) atomicAdd(&sp.stats[0], (unsigned long long)rounds_done);
+    }
+    return handover;
+}
+
+// Four instances per block, one per warp; the instances a warp cannot finish are then run by the whole block with
+// the block-wide scheduler (the same code as k_sched), while the other blocks of the grid go on with theirs.
+__global__ void __launch_bounds__(kWarpSchedWarps * 32)
+k_sched_warp(SchedParams sp, int cap) {
+    extern __shared__ __align__(16) unsigned char dyn[];
+    __shared__ int s_takeover[kWarpSchedWarps];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int inst = blockIdx.x * kWarpSchedWarps + warp;
+    int take = -1;
+    if (inst < sp.P.I) {
+        if (sp.flags[1]) {                   // request table failed validation: do nothing
+            if (lane == 0 && sp.n_done) sp.n_done[inst] = 0;
+        } else {
+            const WarpSchedSmem L(cap, sp.P.Mmax, sp.bmax);
+            if (sched_warp_instance(sp, cap, inst, dyn + (size_t)warp * L.end)) take = inst;
+        }
+    }
+    if (lane == 0) s_takeover[warp] = take;
+    __syncthreads();                         // queues and state of a handed-over instance are in global memory
+    for (int w = 0; w < kWarpSchedWarps; ++w) {
+        if (s_takeover[w] >= 0) {
+            sched_instance(sp, s_takeover[w]);
+            __syncthreads();
+        }
     }
 }
 
