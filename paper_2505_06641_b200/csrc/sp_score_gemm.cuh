@@ -45,6 +45,22 @@ constexpr int kGAThreads = 128, kGEpiThreads = 256;
 constexpr int kMergeFloats = 2 + kMaxModelsPerApp;    // running max, running sum, running sums per model
 constexpr int kGMaxA = 5, kGMaxB = 3;      // largest A / B ring of the two flavours
 
+// Two fp32 values in one 64-bit register for the two-wide FP32 instructions.
+__device__ __forceinline__ unsigned long long pack_f32x2(float lo, float hi) {
+    unsigned long long v;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(lo), "f"(hi));
+    return v;
+}
+// acc = a * b + acc on both halves (round to nearest, one instruction).
+__device__ __forceinline__ void fma_f32x2(unsigned long long &acc, unsigned long long a, unsigned long long b) {
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
+}
+__device__ __forceinline__ float sum_f32x2(unsigned long long v) {
+    float lo, hi;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+    return lo + hi;
+}
+
 template <bool F32>
 struct GCfg {
     static constexpr int NC = F32 ? 208 : 256;                 // logit columns per chunk = MMA N (2 accumulators <= 512 columns)
@@ -428,20 +444,25 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
 #pragma unroll
                     for (int c = 0; c < 32; ++c) { z[c] = exp2_unit(z[c] - run_m); ps += z[c]; }
                     run_s += ps;
+                    // recall contraction with two-wide FMAs: label pairs (c, c + 1) of a model's row against the pair of
+                    // numerators; the two halves of the accumulator are added once per block of 32 labels
+                    unsigned long long zz[16];
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) zz[c] = pack_f32x2(z[2 * c], z[2 * c + 1]);
 #pragma unroll
                     for (int j = 0; j < kMaxModelsPerApp; ++j) {
                         if (j < M) {
                             const float *rr = rt + j * kNC + col0;
-                            float p0 = 0.f, p1 = 0.f;
+                            unsigned long long pp = 0ull;
 #pragma unroll
                             for (int c = 0; c < 32; c += 4) {
                                 if (col0 + c < kNC) {                      // a recall row has NC entries; z is 0 past the group's end
-                                    const float4 rv = *reinterpret_cast<const float4 *>(rr + c);
-                                    p0 = fmaf(z[c], rv.x, p0); p1 = fmaf(z[c + 1], rv.y, p1);
-                                    p0 = fmaf(z[c + 2], rv.z, p0); p1 = fmaf(z[c + 3], rv.w, p1);
+                                    const ulonglong2 rv = *reinterpret_cast<const ulonglong2 *>(rr + c);
+                                    fma_f32x2(pp, zz[c >> 1], rv.x);
+                                    fma_f32x2(pp, zz[(c >> 1) + 1], rv.y);
                                 }
                             }
-                            racc[j] += p0 + p1;
+                            racc[j] += sum_f32x2(pp);
                         }
                     }
                 }
