@@ -450,19 +450,23 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
 #pragma unroll
                     for (int c = 0; c < 16; ++c) zz[c] = pack_f32x2(z[2 * c], z[2 * c + 1]);
 #pragma unroll
-                    for (int j = 0; j < kMaxModelsPerApp; ++j) {
+                    for (int j = 0; j < kMaxModelsPerApp; j += 2) {        // two models at a time: four independent chains
                         if (j < M) {
-                            const float *rr = rt + j * kNC + col0;
-                            unsigned long long pp = 0ull;
+                            const float *r0 = rt + j * kNC + col0, *r1 = j + 1 < M ? r0 + kNC : r0;
+                            unsigned long long p0a = 0ull, p0b = 0ull, p1a = 0ull, p1b = 0ull;
 #pragma unroll
                             for (int c = 0; c < 32; c += 4) {
                                 if (col0 + c < kNC) {                      // a recall row has NC entries; z is 0 past the group's end
-                                    const ulonglong2 rv = *reinterpret_cast<const ulonglong2 *>(rr + c);
-                                    fma_f32x2(pp, zz[c >> 1], rv.x);
-                                    fma_f32x2(pp, zz[(c >> 1) + 1], rv.y);
+                                    const ulonglong2 rv0 = *reinterpret_cast<const ulonglong2 *>(r0 + c);
+                                    const ulonglong2 rv1 = *reinterpret_cast<const ulonglong2 *>(r1 + c);
+                                    fma_f32x2(p0a, zz[c >> 1], rv0.x);
+                                    fma_f32x2(p1a, zz[c >> 1], rv1.x);
+                                    fma_f32x2(p0b, zz[(c >> 1) + 1], rv0.y);
+                                    fma_f32x2(p1b, zz[(c >> 1) + 1], rv1.y);
                                 }
                             }
-                            racc[j] += sum_f32x2(pp);
+                            racc[j] += sum_f32x2(p0a) + sum_f32x2(p0b);
+                            if (j + 1 < M) racc[j + 1] += sum_f32x2(p1a) + sum_f32x2(p1b);
                         }
                     }
                 }
