@@ -470,8 +470,10 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
                     // MMAs of earlier tiles on slab s read the old operand.  Slabs more than kASlots back have
                     // completed (their slots were taken again, which waited for them); the younger ones with the
                     // same s are waited for here, each on a barrier phase that cannot have been passed yet.
-                    for (int64_t ps = (int64_t)slab_seq - n_slabs; ps >= 0 && ps + kASlots >= (int64_t)slab_seq && ok; ps -= n_slabs)
-                        if (!warp_wait(bar(bar_a_free((int)(ps % kASlots))), (uint32_t)(ps / kASlots) & 1, abort_flag)) ok = false;
+                    for (uint32_t back = (uint32_t)n_slabs; back <= slab_seq && back <= (uint32_t)kASlots && ok; back += (uint32_t)n_slabs) {
+                        const uint32_t ps = slab_seq - back;
+                        if (!warp_wait(bar(bar_a_free(ps % kASlots)), (ps / kASlots) & 1, abort_flag)) ok = false;
+                    }
                     if (!ok) break;
                     if (w_row) {
 #pragma unroll
