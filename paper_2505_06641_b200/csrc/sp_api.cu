@@ -56,7 +56,7 @@ struct sp_ctx {
     // profile buffers
     Buf W, bias, recall, prior, prior_dot, prior_sum, lat_alpha, lat_beta, swap;
     // per-instance state and scratch
-    Buf state, zbuf, flags, stats, cnt, gstart, cursor, small_start, tiled_start, small_tiles, scan_partial, wt_image, gemm_tiles, gemm_counter, mma_image;
+    Buf state, zbuf, flags, stats, cnt, gstart, cursor, small_start, tiled_start, small_tiles, scan_partial, wt_image, gemm_tiles, gemm_counter;
     // per-request buffers
     Buf acc32, v32, acc64, v64, exact, recs, perm, q_id0, q_id1, q_dl0, q_dl1, q_pw0, q_pw1, sort_scratch;
     // staging of sp_run_host
@@ -281,7 +281,7 @@ void sp_destroy(sp_ctx *c) {
     drain_events(c->ev_sched, &dummy);
     Buf *all[] = {&c->W, &c->bias, &c->recall, &c->prior, &c->prior_dot, &c->prior_sum, &c->lat_alpha, &c->lat_beta,
                   &c->swap, &c->state, &c->zbuf, &c->flags, &c->stats, &c->cnt, &c->gstart, &c->cursor,
-                  &c->small_start, &c->tiled_start, &c->small_tiles, &c->scan_partial, &c->wt_image, &c->gemm_tiles, &c->gemm_counter, &c->mma_image, &c->acc32, &c->v32, &c->acc64, &c->v64, &c->exact, &c->recs,
+                  &c->small_start, &c->tiled_start, &c->small_tiles, &c->scan_partial, &c->wt_image, &c->gemm_tiles, &c->gemm_counter, &c->acc32, &c->v32, &c->acc64, &c->v64, &c->exact, &c->recs,
                   &c->perm, &c->q_id0, &c->q_id1, &c->q_dl0, &c->q_dl1, &c->q_pw0, &c->q_pw1, &c->sort_scratch,
                   &c->h_feats, &c->h_app, &c->h_arrival, &c->h_deadline, &c->h_instance, &c->h_t0, &c->h_loaded,
                   &c->h_rounds, &c->h_ndone};
@@ -432,10 +432,6 @@ sp_status sp_load_profiles(sp_ctx *c, const sp_profiles *p) {
     if (c->gemm_on) {
     } else if (p->feat_dtype == SP_F32 && D % 4 == 0 && D <= mma::kMaxD && A * C <= mma::kCols && sumM * ((C + 3) & ~3) <= 1024) {
         c->mma_ct = C <= 8 ? 8 : C <= 16 ? 16 : C <= 24 ? 24 : C <= 32 ? 32 : C <= 48 ? 48 : 64;
-        const int n_slabs = (D + mma::kSlabK - 1) / mma::kSlabK;
-        SP_TRY(ensure(c, c->mma_image, (size_t)I * n_slabs * mma::kSlabBytes));
-        mma::k_head_image<<<(unsigned)(I * n_slabs), 256, 0, c->stream>>>((const float *)c->W.p, (unsigned char *)c->mma_image.p, A, D, C, n_slabs);
-        SP_TRY(launched(c, "k_head_image"));
     } else if (p->feat_dtype == SP_F32 && D % 4 == 0 && C <= 64) {
         const int ct = small_ct_for(C);
         const SmallSmem L(A, D, sumM, (ct + 3) & ~3);
@@ -593,7 +589,7 @@ sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, 
         if (c->mma_ct) SP_TRY(feature_map(c, &x_map, feats, n, P.D));
         SP_TRY(mark(c, c->ev_score));
         if (c->mma_ct) {
-            mma::Params prm{P, tb, (const int4 *)c->small_tiles.p, (const unsigned char *)c->mma_image.p, grid, acc_out, (int *)c->flags.p};
+            mma::Params prm{P, tb, (const int4 *)c->small_tiles.p, grid, acc_out, (int *)c->flags.p};
             switch (c->mma_ct) {
                 case 8: SP_TRY(launch_mma<8>(c, x_map, prm)); break;
                 case 16: SP_TRY(launch_mma<16>(c, x_map, prm)); break;

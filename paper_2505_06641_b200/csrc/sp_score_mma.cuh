@@ -17,9 +17,8 @@
 //   * shared-memory bandwidth is the scarce resource (every MMA re-reads its operands), so the A operand
 //     comes from tensor memory: converter warps (one row per thread) read each slab once, store the row as
 //     loaded (read as x_hi) and its remainder x_lo into a ring of tensor-memory columns, and the MMAs read
-//     only the small W operand from shared memory.  The W operand of every instance ([W_hi | W_lo] of
-//     W log2(e), already in the swizzled K-major layout) is built once when the profiles are loaded
-//     (k_head_image); the producer copies it in slab by slab when the instance changes;
+//     only the small W operand from shared memory.  The converters also rebuild the W operand when the
+//     instance changes;
 //   * epilogue warps read the accumulator from tensor memory (one row per thread), add the bias, and do
 //     softmax, the recall contraction, the Dirichlet step and the variance in registers.
 // Every wait on an mbarrier is bounded; when a wait runs out the block raises kDevLimit and leaves.
@@ -39,7 +38,7 @@ constexpr int kSlabBytes = kRows * 128;    // 16 KB: 128 rows x 128 bytes
 constexpr int kMaxD = 128;
 constexpr int kMaxSlabs = kMaxD / kSlabK;
 constexpr int kCols = 64;                  // logit columns (sum over applications of the label count)
-constexpr int kXStages = 8;                // ring of slabs in shared memory filled by TMA (two tiles)
+constexpr int kXStages = 6;                // ring of slabs in shared memory filled by TMA
 constexpr int kASlots = 6;                 // ring of A operands in tensor memory: 32 columns x_hi + 32 columns x_lo each
 constexpr int kTmemCols = 512;             // whole tensor memory
 constexpr int kAccCols = 64;               // columns per accumulator: x_hi W_hi + x_hi W_lo + x_lo W_hi, all applications
@@ -56,14 +55,15 @@ constexpr unsigned long long kWaitLimitNs = 1000ull * 1000ull * 1000ull;
 
 struct Smem {                               // byte offsets from the 1024-byte aligned base
     static constexpr int w = 0;                                        // kMaxSlabs slabs: rows 0..63 W_hi, 64..127 W_lo
-    static constexpr int x = w + kMaxSlabs * kSlabBytes;
+    static constexpr int wraw = w + kMaxSlabs * kSlabBytes;            // the next instance's heads as stored: W[a][d][c] fp32
+    static constexpr int x = wraw + kCols * kMaxD * 4;
     // per-instance tables, one copy per epilogue group, label rows padded with zeros to a multiple of 4 floats (Cp):
     // recall [sumM][Cp] (<= 1024 floats), bias * log2(e) [A][Cp] (<= 128), prior_dot [sumM] (<= 256), prior_sum [A] (<= 16)
     static constexpr int tab_recall = 0, tab_bias = 1024, tab_pdot = tab_bias + 2 * kCols, tab_psum = tab_pdot + 256;
     static constexpr int tab_floats = tab_psum + 16;
     static constexpr int tabs = x + kXStages * kSlabBytes;
     static constexpr int bars = tabs + kEpiGroups * tab_floats * 4;
-    static constexpr int n_bars = 2 * kXStages + 3 * kASlots + 9 + 2 * kEpiGroups + 2 * kMaxSlabs;
+    static constexpr int n_bars = 2 * kXStages + 3 * kASlots + 9 + 2 * kEpiGroups;
     static constexpr int misc = bars + n_bars * 8;                     // tmem base, abort flag
     static constexpr int end = misc + 16;
     static constexpr int bytes = end + 1024;                           // slack for the manual alignment
@@ -73,7 +73,6 @@ struct Params {
     DevProfiles P;
     DevTable tb;
     const int4 *tiles;       // (instance, first request relative to the instance, rows, first request in the table)
-    const unsigned char *head_image;   // [I][n_slabs][kSlabBytes] operand slabs written by k_head_image
     int n_tiles;             // entries in `tiles`; the valid ones come first, those past the end have instance -1
     float *acc_out;          // optional second destination of acc
     int *flags;
@@ -269,32 +268,6 @@ __device__ __forceinline__ float exp2_unit(float x) {
     return p;
 }
 
-// Head operand of every instance, built once when the profiles are loaded: per instance and feature slab one
-// 16 KB block in the layout the MMA reads (K-major rows of 32 features, 128-byte swizzle): rows 0..63 hold W_hi and
-// rows 64..127 W_lo of W log2(e) for logit column (application, label) = row & 63; rows and features without a
-// weight are zero.  One thread block per (instance, slab).
-__global__ void k_head_image(const float *__restrict__ W, unsigned char *__restrict__ image, int A, int D, int C, int n_slabs) {
-    const int inst = blockIdx.x / n_slabs, s = blockIdx.x - inst * n_slabs;
-    unsigned char *slab = image + (size_t)blockIdx.x * kSlabBytes;
-    for (int q = threadIdx.x; q < kRows * 8; q += blockDim.x) {
-        const int r = q >> 3, j = q & 7, col = r & (kCols - 1);
-        float v[4] = {0.f, 0.f, 0.f, 0.f};
-        if (col < A * C) {
-            const int a = col / C, c = col - a * C;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int dd = s * kSlabK + j * 4 + e;
-                if (dd < D) {
-                    const float w = W[(((int64_t)inst * A + a) * D + dd) * C + c] * kLog2e;
-                    const float hi = tf32_part(w);
-                    v[e] = r < kCols ? hi : w - hi;
-                }
-            }
-        }
-        *reinterpret_cast<float4 *>(slab + r * 128 + ((j ^ (r & 7)) << 4)) = make_float4(v[0], v[1], v[2], v[3]);
-    }
-}
-
 // Barrier indices
 constexpr int kBarBase2 = 2 * kXStages + 3 * kASlots;
 __device__ __forceinline__ constexpr int bar_full(int h) { return h; }                       // slab landed in shared memory
@@ -306,16 +279,12 @@ __device__ __forceinline__ constexpr int bar_a_free(int l) { return 2 * kXStages
 __device__ __forceinline__ constexpr int bar_acc_full(int b) { return kBarBase2 + b; }
 __device__ __forceinline__ constexpr int bar_acc_empty(int b) { return kBarBase2 + 2 + b; }
 constexpr int kBarDrain = kBarBase2 + 5;
+constexpr int kBarRawFull = kBarBase2 + 6;    // raw heads of an instance landed in shared memory
+constexpr int kBarRawFree = kBarBase2 + 7;    // converters have turned them into the operand
 constexpr int kBarDrain2 = kBarBase2 + 8;     // drain barrier of the second MMA issuer
 // per epilogue group: A = every thread is done reading the old tables, B = the new tables are written
 __device__ __forceinline__ constexpr int bar_epi_a(int g) { return kBarBase2 + 9 + g; }
 __device__ __forceinline__ constexpr int bar_epi_b(int g) { return kBarBase2 + 9 + kEpiGroups + g; }
-
-// Head operand, slab s: the instance's slab has landed in shared memory (both MMA issuers wait on it, each once per
-// instance and in order, so neither can be a phase behind) / both issuers have completed their MMAs of the instance on it
-constexpr int kBarBase3 = kBarBase2 + 9 + 2 * kEpiGroups;
-__device__ __forceinline__ constexpr int bar_w_ready(int s) { return kBarBase3 + s; }
-__device__ __forceinline__ constexpr int bar_w_free(int s) { return kBarBase3 + kMaxSlabs + s; }
 
 // Warp-uniform outcome of a bounded wait done by every lane.
 __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
@@ -354,11 +323,14 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
         for (int b = 0; b < 2; ++b) { mbar_init(bar(bar_acc_full(b)), 1); mbar_init(bar(bar_acc_empty(b)), kEpiThreads); }
         mbar_init(bar(kBarDrain), 1);
         mbar_init(bar(kBarDrain2), 1);
-        for (int q = 0; q < kMaxSlabs; ++q) { mbar_init(bar(bar_w_ready(q)), 1); mbar_init(bar(bar_w_free(q)), 2); }
+        mbar_init(bar(kBarRawFull), 1);
+        mbar_init(bar(kBarRawFree), kConvThreads);
         for (int g = 0; g < kEpiGroups; ++g) { mbar_init(bar(bar_epi_a(g)), kEpiThreads); mbar_init(bar(bar_epi_b(g)), kEpiThreads); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    for (int k = tid; k < kMaxSlabs * kSlabBytes / 16; k += kThreads)
+        reinterpret_cast<float4 *>(sm + Smem::w)[k] = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int k = tid; k < kEpiGroups * Smem::tab_floats; k += kThreads)      // the padding of the label rows stays zero
         reinterpret_cast<float *>(sm + Smem::tabs)[k] = 0.f;
     if (warp == kMmaWarp) {
@@ -379,72 +351,35 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
     } else if (warp == kProducerWarp) {
         // ================================================================ TMA producer (one thread)
         if (lane == 0) {
-            uint32_t slab_seq = 0;
+            uint32_t slab_seq = 0, w_seq = 0;
+            int cur_inst = -1;
+            const uint32_t w_bytes = (uint32_t)(A * D * C) * 4u;
             bool ok = true;
-            // Head operands: instance number w_seq of this block (first tile w_tile) is copied in slab by slab; slab s
-            // may be overwritten once both MMA issuers are through with it for the previous instance (bar_w_free).
-            // The copies are pumped from inside the producer's waits, so they start as soon as a slab is free: the
-            // remaining slabs of the previous instance's last tile cover their latency.
-            const size_t image_bytes = (size_t)n_slabs * kSlabBytes;
-            uint32_t w_seq = 0;
-            int w_slab = 0, w_tile = t_begin;
-            int4 w_d = t_begin < t_end ? prm.tiles[t_begin] : make_int4(-1, 0, 0, 0);
-            auto pump_w = [&]() {
-                while (w_d.x >= 0) {
-                    if (w_seq > 0 && !mbar_try_wait(bar(bar_w_free(w_slab)), (w_seq - 1) & 1)) return;
-                    mbar_arrive_expect_tx(bar(bar_w_ready(w_slab)), kSlabBytes);
-                    bulk_load(base + Smem::w + w_slab * kSlabBytes,
-                              prm.head_image + (size_t)w_d.x * image_bytes + (size_t)w_slab * kSlabBytes, kSlabBytes,
-                              bar(bar_w_ready(w_slab)));
-                    if (++w_slab == n_slabs) {                 // on to the next instance of this block's tiles
-                        w_slab = 0; ++w_seq;
-                        const int cur = w_d.x;
-                        do { ++w_tile; w_d = w_tile < t_end ? prm.tiles[w_tile] : make_int4(-1, 0, 0, 0); } while (w_d.x == cur);
-                    }
-                }
-            };
-            // bounded wait that keeps the head copies going
-            auto wait_pumping = [&](uint32_t b, uint32_t parity) -> bool {
-                if (mbar_try_wait(b, parity)) return true;
-                const unsigned long long t0 = global_ns();
-                for (uint32_t it = 1;; ++it) {
-                    pump_w();
-                    if (mbar_try_wait(b, parity)) return true;
-                    if ((it & 63) == 0) {
-                        if (*abort_flag) return false;
-                        if (global_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
-                    }
-                }
-            };
-            pump_w();
             int4 d_next = t_begin < t_end ? prm.tiles[t_begin] : make_int4(-1, 0, 0, 0);
             for (int t = t_begin; t < t_end && ok; ++t) {
                 const int4 d = d_next;
                 if (d.x < 0) break;                            // valid tiles form a prefix of the block's range
                 if (t + 1 < t_end) d_next = prm.tiles[t + 1];
+                if (d.x != cur_inst) {                         // stage the heads of the instance this tile starts
+                    if (w_seq > 0 && !mbar_wait(bar(kBarRawFree), (w_seq - 1) & 1, abort_flag)) break;
+                    mbar_arrive_expect_tx(bar(kBarRawFull), w_bytes);
+                    bulk_load(base + Smem::wraw, (const float *)P.W + (int64_t)d.x * A * D * C, w_bytes, bar(kBarRawFull));
+                    ++w_seq; cur_inst = d.x;
+                }
                 const int row0 = d.w;
                 for (int s = 0; s < n_slabs; ++s, ++slab_seq) {
                     const int h = slab_seq % kXStages;
                     const uint32_t use = slab_seq / kXStages;
-                    if (use > 0 && !wait_pumping(bar(bar_x_free(h)), (use - 1) & 1)) { ok = false; break; }
+                    if (use > 0 && !mbar_wait(bar(bar_x_free(h)), (use - 1) & 1, abort_flag)) { ok = false; break; }
                     mbar_arrive_expect_tx(bar(bar_full(h)), kSlabBytes);
                     tma_load_2d(base + Smem::x + h * kSlabBytes, &x_map, s * kSlabK, row0, bar(bar_full(h)));
-                    pump_w();
                 }
-            }
-            // every feature slab is on its way; the head operands of the last instances may still be waiting for
-            // their slabs to become free
-            while (ok && w_d.x >= 0) {
-                if (w_seq > 0 && !wait_pumping(bar(bar_w_free(w_slab)), (w_seq - 1) & 1)) { ok = false; break; }
-                pump_w();
             }
             if (!ok || *abort_flag) {
                 // copies already issued still land in shared memory: give them a bounded time to finish
-                for (int q = 0; q < n_slabs; ++q) {
-                    const uint32_t issued = w_seq + (q < w_slab ? 1u : 0u);     // copies into slab q so far
-                    if (issued == 0) continue;
+                if (w_seq > 0) {
                     const unsigned long long t0 = global_ns();
-                    while (!mbar_try_wait(bar(bar_w_ready(q)), (issued - 1) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+                    while (!mbar_try_wait(bar(kBarRawFull), (w_seq - 1) & 1) && global_ns() - t0 < kWaitLimitNs) {}
                 }
                 const uint32_t first = slab_seq > (uint32_t)kXStages ? slab_seq - kXStages : 0;
                 for (uint32_t q = first; q < slab_seq; ++q) {
@@ -466,56 +401,35 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
             const int mg = warp == kMmaWarp ? 0 : 1;
             bool ok = true;
             uint32_t rdy_par = 0;                              // bit l: parity of this issuer's next wait on slot l
-            // The issuer walks over every tile of the block (descriptors three tiles ahead) to follow the instance
-            // sequence: per instance and slab it waits once for the head operand (bar_w_ready) and arrives once when
-            // its MMAs of the instance on that slab are done (bar_w_free), also for instances it has no tile in, so
-            // that every phase of those barriers is consumed in order by both issuers.
-            auto desc = [&](int t) { return t < t_end ? prm.tiles[t] : make_int4(-1, 0, 0, 0); };
-            int4 d0 = desc(t_begin), d1 = desc(t_begin + 1), d2 = desc(t_begin + 2);
-            uint32_t inst_seq = 0;
-            int cur = d0.x;
-            bool own_in_inst = false, w_seen = false;          // w_seen: operand of the current instance already waited for
-            for (int t = t_begin; t < t_end && ok; ++t) {
-                const int4 d = d0;
+            int4 d_next = t_begin + mg < t_end ? prm.tiles[t_begin + mg] : make_int4(-1, 0, 0, 0);
+            for (int t = t_begin + mg; t < t_end && ok; t += 2) {
+                const int4 d = d_next;
                 if (d.x < 0) break;                            // valid tiles form a prefix of the block's range
-                d0 = d1; d1 = d2; d2 = desc(t + 3);            // d0, d1 = tiles t + 1, t + 2
-                if (d.x != cur) { cur = d.x; ++inst_seq; own_in_inst = false; w_seen = false; }
+                if (t + 2 < t_end) d_next = prm.tiles[t + 2];
                 const uint32_t tile_seq = (uint32_t)(t - t_begin);
-                const bool last_of_inst = d0.x != d.x;
-                if ((tile_seq & 1) == (uint32_t)mg) {
-                    own_in_inst = true;
-                    const bool last_own = last_of_inst || d1.x != d.x;   // tile t + 2 belongs to another instance
-                    uint32_t slab_seq = tile_seq * (uint32_t)n_slabs;
-                    const uint32_t b = tile_seq & 1, acc_use = tile_seq >> 1;
-                    if (acc_use > 0 && !mbar_wait(bar(bar_acc_empty(b)), (acc_use - 1) & 1, abort_flag)) break;
+                uint32_t slab_seq = tile_seq * (uint32_t)n_slabs;
+                const uint32_t b = tile_seq & 1, acc_use = tile_seq >> 1;
+                if (acc_use > 0 && !mbar_wait(bar(bar_acc_empty(b)), (acc_use - 1) & 1, abort_flag)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = b * kAccCols;
+                for (int s = 0; s < n_slabs; ++s, ++slab_seq) {
+                    const uint32_t l = slab_seq % kASlots;
+                    // the slot holds the rows of this slab; the same arrival says that the head operand of the
+                    // slab's features is in place (the converters rebuild it before they arrive)
+                    if (!mbar_wait(bar(bar_a_ready(mg, l)), (rdy_par >> l) & 1, abort_flag)) { ok = false; break; }
+                    rdy_par ^= 1u << l;
                     tc_fence_after();
-                    const uint32_t d_tmem = b * kAccCols;
-                    for (int s = 0; s < n_slabs; ++s, ++slab_seq) {
-                        const uint32_t l = slab_seq % kASlots;
-                        if (!w_seen && !mbar_wait(bar(bar_w_ready(s)), inst_seq & 1, abort_flag)) { ok = false; break; }
-                        if (!mbar_wait(bar(bar_a_ready(mg, l)), (rdy_par >> l) & 1, abort_flag)) { ok = false; break; }
-                        rdy_par ^= 1u << l;
-                        tc_fence_after();
-                        const uint32_t a_hi = kTmemA + l * kSlotCols, a_lo = a_hi + kSlabK;
-                        const uint64_t b_w = w_desc + (uint64_t)((s * kSlabBytes) >> 4);
+                    const uint32_t a_hi = kTmemA + l * kSlotCols, a_lo = a_hi + kSlabK;
+                    const uint64_t b_w = w_desc + (uint64_t)((s * kSlabBytes) >> 4);
 #pragma unroll
-                        for (int k = 0; k < kSlabK / 8; ++k) {     // the three products accumulate in the same 64 columns
-                            umma_tf32_ts(d_tmem, a_hi + k * 8, b_w + (uint64_t)(k * 2), idesc, (s | k) != 0);
-                            umma_tf32_ts(d_tmem, a_hi + k * 8, b_w + w_lo_rows + (uint64_t)(k * 2), idesc, 1u);
-                            umma_tf32_ts(d_tmem, a_lo + k * 8, b_w + (uint64_t)(k * 2), idesc, 1u);
-                        }
-                        umma_commit(bar(bar_a_free(l)));
-                        if (last_own) umma_commit(bar(bar_w_free(s)));
+                    for (int k = 0; k < kSlabK / 8; ++k) {     // the three products accumulate in the same 64 columns
+                        umma_tf32_ts(d_tmem, a_hi + k * 8, b_w + (uint64_t)(k * 2), idesc, (s | k) != 0);
+                        umma_tf32_ts(d_tmem, a_hi + k * 8, b_w + w_lo_rows + (uint64_t)(k * 2), idesc, 1u);
+                        umma_tf32_ts(d_tmem, a_lo + k * 8, b_w + (uint64_t)(k * 2), idesc, 1u);
                     }
-                    w_seen = true;
-                    if (ok) umma_commit(bar(bar_acc_full(b)));
+                    umma_commit(bar(bar_a_free(l)));
                 }
-                if (ok && last_of_inst && !own_in_inst) {      // an instance without a tile of this issuer
-                    for (int s = 0; s < n_slabs && ok; ++s) {
-                        if (!mbar_wait(bar(bar_w_ready(s)), inst_seq & 1, abort_flag)) { ok = false; break; }
-                        mbar_arrive(bar(bar_w_free(s)));
-                    }
-                }
+                if (ok) umma_commit(bar(bar_acc_full(b)));
             }
             if (*abort_flag) {                                 // leaving early: let the issued MMAs finish first
                 const uint32_t drain = bar(mg ? kBarDrain2 : kBarDrain);
@@ -526,8 +440,19 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
         }
     } else if (warp < kEpiWarp0) {
         // ================================================================ converter warps
+        const int ct = tid - kConvWarp0 * 32;                  // 0..127
         const int cquad = warp & 3, crow = cquad * 32 + lane;  // tensor-memory lanes this warp may write = its rows
-        uint32_t slab_seq = 0;
+        uint32_t slab_seq = 0, w_seq = 0;
+        int cur_inst = -1;
+        // Head operand: this thread owns logit column wn (= operand row) and, per slab, 4 of its 8 chunks of 4
+        // features.  The raw heads W[a][d][c] of the instance were staged in shared memory by the producer;
+        // consecutive threads read consecutive labels (distinct banks) and write 16-byte pieces of the swizzled
+        // operand rows.  The operand is rebuilt slab by slab during the first tile of an instance: slab s as soon
+        // as the MMAs of the previous tile's slab s have completed, so the pipeline never drains.
+        const int wn = ct & (kCols - 1), wq0 = (ct >> 6) * 4;
+        const int wa = wn / C, wc = wn - wa * C;
+        const bool w_row = wn < A * C;
+        const float *wraw = reinterpret_cast<const float *>(sm + Smem::wraw) + wa * D * C + wc;
         bool ok = true;
         int4 d_next = t_begin < t_end ? prm.tiles[t_begin] : make_int4(-1, 0, 0, 0);
         for (int t = t_begin; t < t_end && ok; ++t) {
@@ -535,9 +460,43 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
             if (d.x < 0) break;                                // valid tiles form a prefix of the block's range
             if (t + 1 < t_end) d_next = prm.tiles[t + 1];
             const int mg = (t - t_begin) & 1;                  // MMA issuer of this tile
+            const bool new_inst = d.x != cur_inst;
+            cur_inst = d.x;
+            if (new_inst && !warp_wait(bar(kBarRawFull), w_seq & 1, abort_flag)) break;
             for (int s = 0; s < n_slabs; ++s, ++slab_seq) {
                 const int h = slab_seq % kXStages, l = slab_seq % kASlots;
                 const uint32_t a_use = slab_seq / kASlots;
+                if (new_inst) {
+                    // MMAs of earlier tiles on slab s read the old operand.  Slabs more than kASlots back have
+                    // completed (their slots were taken again, which waited for them); the younger ones with the
+                    // same s are waited for here, each on a barrier phase that cannot have been passed yet.
+                    for (uint32_t back = (uint32_t)n_slabs; back <= slab_seq && back <= (uint32_t)kASlots && ok; back += (uint32_t)n_slabs) {
+                        const uint32_t ps = slab_seq - back;
+                        if (!warp_wait(bar(bar_a_free(ps % kASlots)), (ps / kASlots) & 1, abort_flag)) ok = false;
+                    }
+                    if (!ok) break;
+                    if (w_row) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            const int j = wq0 + q, dd = s * kSlabK + j * 4;   // 16-byte piece j of the operand row
+                            if (dd < D) {
+                                const uint32_t off = (uint32_t)(s * kSlabBytes + wn * 128 + ((j ^ (wn & 7)) << 4));
+                                const float *src = wraw + dd * C;
+                                const float w0 = src[0] * kLog2e, w1 = src[C] * kLog2e;
+                                const float w2 = src[2 * C] * kLog2e, w3 = src[3 * C] * kLog2e;
+                                float4 hi, lo;
+                                hi.x = tf32_part(w0); lo.x = w0 - hi.x;
+                                hi.y = tf32_part(w1); lo.y = w1 - hi.y;
+                                hi.z = tf32_part(w2); lo.z = w2 - hi.z;
+                                hi.w = tf32_part(w3); lo.w = w3 - hi.w;
+                                *reinterpret_cast<float4 *>(sm + Smem::w + off) = hi;
+                                *reinterpret_cast<float4 *>(sm + Smem::w + off + kCols * 128) = lo;
+                            }
+                        }
+                    }
+                    fence_proxy_async();
+                    if (s == n_slabs - 1) { mbar_arrive(bar(kBarRawFree)); ++w_seq; }
+                }
                 if (!warp_wait(bar(bar_full(h)), (slab_seq / kXStages) & 1, abort_flag)) { ok = false; break; }
                 // this thread's row of the slab: 8 pieces of 16 bytes, un-swizzled into feature order
                 const unsigned char *xrow = sm + Smem::x + h * kSlabBytes + crow * 128;
