@@ -279,7 +279,10 @@ __device__ __forceinline__ void warp_argmax(const double *cand_u, const int *can
     best = bi; best_u = bu; n_close = cnt; max_bp = mb;
 }
 
-// All rounds of one instance by one thread block (every thread of the block calls it).
+// All rounds of one instance by one thread block (every thread of the block calls it).  SOFT = false leaves the
+// linear and sigmoid penalties out of the code (every application has the step penalty): the round loop is a long
+// stretch of code that every warp walks through once per round, and what is not there is not fetched.
+template <bool SOFT>
 __device__ void sched_instance(const SchedParams &sp, const int inst) {
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ InstState st;
@@ -517,7 +520,7 @@ __device__ void sched_instance(const SchedParams &sp, const int inst) {
             const int per = NT / A, a = tid / per, j = tid - a * per;
             bool late = false;
             if (a < A && !s_pdone[a]) {
-                const int lo = s_lo[a], hi = s_hi[a], span = hi - lo, kind = P.pen[a];
+                const int lo = s_lo[a], hi = s_hi[a], span = hi - lo, kind = SOFT ? P.pen[a] : SP_PEN_STEP;
                 const bool window = pass == 0 || kind != SP_PEN_STEP || span <= per;
                 const int k = window ? lo + j : lo + (int)(((int64_t)(j + 1) * span) / (per + 1));
                 if (k < hi) {
@@ -531,7 +534,7 @@ __device__ void sched_instance(const SchedParams &sp, const int inst) {
             if (lane == 0) s_ballot[warp] = bal;
             __syncthreads();
             if (tid < A && !s_pdone[tid]) {
-                const int a2 = tid, lo = s_lo[a2], hi = s_hi[a2], span = hi - lo, kind = P.pen[a2];
+                const int a2 = tid, lo = s_lo[a2], hi = s_hi[a2], span = hi - lo, kind = SOFT ? P.pen[a2] : SP_PEN_STEP;
                 const bool window = pass == 0 || kind != SP_PEN_STEP || span <= per;
                 int cnt = 0;                      // leading hopeless positions among the per looked at
                 for (int t2 = a2 * per, end = t2 + per; t2 < end;) {
@@ -654,9 +657,9 @@ __device__ void sched_instance(const SchedParams &sp, const int inst) {
         for (int k = tid; k < nb; k += NT) {
             mem_id[k] = sp.q_id[c][base + head + k];
             mem_dl[k] = sp.q_dl[c][base + head + k];
-            if (P.pen[a] != SP_PEN_STEP) mem_delta[k] = mem_dl[k] - tb.arrival[mem_id[k]];
+            if (SOFT && P.pen[a] != SP_PEN_STEP) mem_delta[k] = mem_dl[k] - tb.arrival[mem_id[k]];
         }
-        const int pen = P.pen[a];
+        const int pen = SOFT ? P.pen[a] : SP_PEN_STEP;
         __syncthreads();
         for (int k = tid; k < nb * Mmax; k += NT) {
             const int r = k / Mmax, j = k - r * Mmax;
@@ -768,6 +771,7 @@ __device__ void sched_instance(const SchedParams &sp, const int inst) {
     }
 }
 
-__global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) { sched_instance(sp, blockIdx.x); }
+template <bool SOFT>
+__global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) { sched_instance<SOFT>(sp, blockIdx.x); }
 
 }  // namespace sp
