@@ -237,13 +237,17 @@ sp_status matrix_map(sp_ctx *c, CUtensorMap *map, const void *ptr, CUtensorMapDa
     return SP_OK;
 }
 
-template <int CT>
-sp_status launch_mma(sp_ctx *c, const CUtensorMap &map, const mma::Params &prm) {
-    auto kern = mma::k_score_mma<CT>;
+template <int CT, bool PRIOR>
+sp_status launch_mma_p(sp_ctx *c, const CUtensorMap &map, const mma::Params &prm) {
+    auto kern = mma::k_score_mma<CT, PRIOR>;
     SP_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, mma::Smem::bytes));
     const int grid = prm.n_tiles < c->n_sms ? prm.n_tiles : c->n_sms;
     kern<<<grid, mma::kThreads, mma::Smem::bytes, c->stream>>>(map, prm);
     return launched(c, "k_score_mma");
+}
+template <int CT>
+sp_status launch_mma(sp_ctx *c, const CUtensorMap &map, const mma::Params &prm) {
+    return prm.P.prior ? launch_mma_p<CT, true>(c, map, prm) : launch_mma_p<CT, false>(c, map, prm);
 }
 
 }  // namespace

@@ -292,8 +292,9 @@ __device__ __forceinline__ bool warp_wait(uint32_t bar, uint32_t parity, volatil
     return __all_sync(0xffffffffu, ok);
 }
 
-// CT = power of two >= C: logit columns one epilogue thread keeps in registers.
-template <int CT>
+// CT = logit columns one epilogue thread keeps in registers (>= C); PRIOR = a Dirichlet prior is set (without it the
+// code of that step is left out).
+template <int CT, bool PRIOR>
 __global__ void __launch_bounds__(kThreads, 1)
 k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
     extern __shared__ unsigned char smem_raw[];
@@ -547,7 +548,7 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
                 pre_rec[q] = k < sumM * C ? P.recall[(int64_t)inst * sumM * C + k] : 0.f;
             }
             pre_bias = et < A * C ? P.bias[(int64_t)inst * A * C + et] : 0.f;
-            if (P.prior) {
+            if (PRIOR) {
 #pragma unroll
                 for (int q = 0; q < 256 / kEpiThreads; ++q) {
                     const int k = q * kEpiThreads + et;
@@ -581,7 +582,7 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
                     if (k < sumM * C) { const int g = k / C; tab[Smem::tab_recall + g * Cp + (k - g * C)] = pre_rec[q]; }
                 }
                 if (et < A * C) { const int g = et / C; tab[Smem::tab_bias + g * Cp + (et - g * C)] = pre_bias * kLog2e; }
-                if (P.prior) {
+                if (PRIOR) {
 #pragma unroll
                     for (int q = 0; q < 256 / kEpiThreads; ++q) {
                         const int k = q * kEpiThreads + et;
@@ -657,7 +658,7 @@ k_score_mma(const __grid_constant__ CUtensorMap x_map, const Params prm) {
                         }
                     aj0 = (p0 + p1) * inv;
                     aj1 = (q0 + q1) * inv;
-                    if (P.prior) {
+                    if (PRIOR) {
                         aj0 = (pdot_s[g0 + j] + P.kappa * aj0) / (psum_s[a] + P.kappa);
                         if (m1) aj1 = (pdot_s[g0 + j + 1] + P.kappa * aj1) / (psum_s[a] + P.kappa);
                     }
