@@ -167,9 +167,12 @@ __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const 
 #pragma unroll
         for (int u = 0; u < kWarpLoadChunk * 2; ++u) {
             const int k = (q0 + u) * 32 + lane;
-            if (k < m) s_pw[k] = prio_weight((double)vreg[u], s_dl[k], Tref, tau);
+            if (k < m) s_pw[k] = (double)vreg[u];
         }
     }
+    // the weights in a rolled loop: one copy of the fp64 exponential in the code instead of sixteen
+#pragma unroll 1
+    for (int k = lane; k < m; k += 32) s_pw[k] = prio_weight(s_pw[k], s_dl[k], Tref, tau);
     int seg = 0;                                          // lane a <= A: first position whose application is >= a
     if (lane <= A) {
         int lo = 0, hi = m;
