@@ -147,14 +147,6 @@ __global__ void k_get_clock(const InstState *st, int n_inst, int64_t *t, int32_t
     if (l) l[i] = st[i].L;
 }
 
-__global__ void k_init_requests(sp_req_rec *recs, unsigned char *exact, int64_t n) {
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n) return;
-    sp_req_rec r; r.status = SP_PENDING; r.round = -1; r.model = -1; r.pad_ = 0; r.order = 0;
-    recs[i] = r;
-    exact[i] = 0;
-}
-
 constexpr size_t kMaxTimedCalls = 512;
 
 // Records an event on the context's stream and keeps it in `list` (timing option only).
@@ -547,8 +539,6 @@ sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, 
     SP_CUDA(c, cudaMemsetAsync(tb.cursor, 0, nkeys * 4, c->stream));
     const unsigned gb = (unsigned)((n + 255) / 256);
     if (n > 0) {
-        k_init_requests<<<gb, 256, 0, c->stream>>>(tb.recs, tb.exact, n);
-        SP_TRY(launched(c, "k_init_requests"));
         k_group_count<<<gb, 256, 0, c->stream>>>(P, tb, c->opt.trace_mode, (int *)c->flags.p);
         SP_TRY(launched(c, "k_group_count"));
     }

@@ -10,10 +10,16 @@ namespace sp {
 constexpr int kTiledRows = 64;    // requests per tile of the tiled scoring kernel
 constexpr int kSmallRows = 128;   // requests per tile of the small-head scoring kernel
 
+// Validation of the request table, initial request records, requests per (instance, application).
 // flags[0]: device status (DevErr), flags[1]: 1 when the request table failed validation.
 __global__ void k_group_count(DevProfiles P, DevTable tb, int trace_mode, int *flags) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= tb.n) return;
+    if (tb.recs) {                           // the request starts pending, without an fp64 re-scoring (a table
+        sp_req_rec r; r.status = SP_PENDING; r.round = -1; r.model = -1; r.pad_ = 0; r.order = 0;   // that is only scored has no records)
+        tb.recs[i] = r;
+        tb.exact[i] = 0;
+    }
     const int a = tb.app[i];
     const int inst = tb.instance ? tb.instance[i] : 0;
     bool bad = a < 0 || a >= P.A || inst < 0 || inst >= P.I;
