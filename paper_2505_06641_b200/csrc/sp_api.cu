@@ -686,8 +686,14 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
             // the block-wide scheduler runs inside the same kernel for the instances a warp hands over: its shared
             // memory is laid over the warps' slices
             const size_t wsmem = W.end * kWarpSchedWarps > L.end ? W.end * kWarpSchedWarps : L.end;
-            SP_CUDA(c, cudaFuncSetAttribute(k_sched_warp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)wsmem));
-            k_sched_warp<<<wgrid, kWarpSchedWarps * 32, wsmem, c->stream>>>(sp, (int)wcap);
+            if (P.Mmax <= 8 && P.Mmax * P.nB <= 64) {          // short unrolled loops for small model and batch-size sets
+                SP_CUDA(c, cudaFuncSetAttribute(k_sched_warp<8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)wsmem));
+                k_sched_warp<8, 2><<<wgrid, kWarpSchedWarps * 32, wsmem, c->stream>>>(sp, (int)wcap);
+            } else {
+                SP_CUDA(c, cudaFuncSetAttribute(k_sched_warp<kMaxModelsPerApp, kMaxModelsPerApp * kMaxBatchSizes / 32>,
+                                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)wsmem));
+                k_sched_warp<kMaxModelsPerApp, kMaxModelsPerApp * kMaxBatchSizes / 32><<<wgrid, kWarpSchedWarps * 32, wsmem, c->stream>>>(sp, (int)wcap);
+            }
             SP_TRY(launched(c, "k_sched_warp"));
             c->sched_started = true;
             return mark(c, c->ev_sched);

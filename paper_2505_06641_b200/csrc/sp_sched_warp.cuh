@@ -22,7 +22,6 @@ namespace sp {
 
 constexpr int kWarpSchedWarps = 4;          // instances per block
 constexpr int kWarpLoadChunk = 8;           // requests per lane loaded together at the start
-constexpr int kWarpCandPerLane = kMaxModelsPerApp * kMaxBatchSizes / 32;
 
 struct WarpSchedSmem {                      // per-warp byte offsets (8-byte aligned pieces)
     size_t dl, pw, ida, pref, end;
@@ -82,6 +81,9 @@ __device__ __forceinline__ void warp_sort(int64_t *dl, uint32_t *ida, int n) {
 
 // One instance by one warp.  Returns true when the block-wide scheduler has to take the instance over: a near-tie
 // to decide in fp64, more requests than the warp's slice holds, or an instance that had already started.
+// MM bounds the models per application and CPL the candidates per lane (models x batch sizes / 32): the loops over
+// them are unrolled, and the small instantiation keeps the code of a round short.
+template <int MM, int CPL>
 __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const int inst, unsigned char *mine) {
     const DevProfiles &P = sp.P;
     const DevTable &tb = sp.tb;
@@ -248,17 +250,17 @@ __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const 
         const uint32_t *mida = s_ida + qh;
         for (int j = lane; j < M; j += 32) pref[(size_t)j * (bmax + 1)] = 0.0;
         {
-            double carry[kMaxModelsPerApp];
+            double carry[MM];
 #pragma unroll
-            for (int j = 0; j < kMaxModelsPerApp; ++j) carry[j] = 0.0;
+            for (int j = 0; j < MM; ++j) carry[j] = 0.0;
             for (int k0 = 0; k0 < nb; k0 += 32) {             // fp64 prefix sums of the members' accuracies, per model
                 const int k = k0 + lane;
                 const float *row = tb.acc32 + (r0 + (k < nb ? (int64_t)(mida[k] & 0xFFFFFFu) : 0)) * Mmax;
-                float rv[kMaxModelsPerApp];
+                float rv[MM];
 #pragma unroll
-                for (int j = 0; j < kMaxModelsPerApp; ++j) rv[j] = (j < M && k < nb) ? row[j] : 0.f;
+                for (int j = 0; j < MM; ++j) rv[j] = (j < M && k < nb) ? row[j] : 0.f;
 #pragma unroll
-                for (int j = 0; j < kMaxModelsPerApp; ++j) {
+                for (int j = 0; j < MM; ++j) {
                     if (j < M) {
                         double v = (double)rv[j];
 #pragma unroll
@@ -276,11 +278,11 @@ __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const 
         __syncwarp();
         // completion time base and slope of every model, for the candidates: lane g holds model g
         const int64_t base_e = T + (lane != Lm ? my_sw : 0) + my_al;
-        double cu[kWarpCandPerLane];                          // utilities of this lane's candidates
+        double cu[CPL];                          // utilities of this lane's candidates
         double bu = -INFINITY;
         int bi_ = 0x7fffffff;
 #pragma unroll
-        for (int q = 0; q < kWarpCandPerLane; ++q) {
+        for (int q = 0; q < CPL; ++q) {
             const int ci = q * 32 + lane;
             cu[q] = -INFINITY;
             if (q * 32 < ncand) {                                  // uniform: shuffles below are warp-wide
@@ -312,7 +314,7 @@ __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const 
         const double thr = wu - fabs(wu) * sp.guard_u;
         int ncl = 0;
 #pragma unroll
-        for (int q = 0; q < kWarpCandPerLane; ++q) ncl += (cu[q] >= thr && cu[q] != -INFINITY) ? 1 : 0;
+        for (int q = 0; q < CPL; ++q) ncl += (cu[q] >= thr && cu[q] != -INFINITY) ? 1 : 0;
         if (warp_sum_i32(ncl) > 1) { handover = true; break; }     // near-tie between candidates
         // ---------------------------------------------------------------- emit, remove, advance the clock
         const int bj = wi / nB, bbi = wi - bj * nB, g = m0 + bj;
@@ -365,6 +367,7 @@ __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const 
 
 // Four instances per block, one per warp; the instances a warp cannot finish are then run by the whole block with
 // the block-wide scheduler (the same code as k_sched), while the other blocks of the grid go on with theirs.
+template <int MM, int CPL>
 __global__ void __launch_bounds__(kWarpSchedWarps * 32)
 k_sched_warp(SchedParams sp, int cap) {
     extern __shared__ __align__(16) unsigned char dyn[];
@@ -377,7 +380,7 @@ k_sched_warp(SchedParams sp, int cap) {
             if (lane == 0 && sp.n_done) sp.n_done[inst] = 0;
         } else {
             const WarpSchedSmem L(cap, sp.P.Mmax, sp.bmax);
-            if (sched_warp_instance(sp, cap, inst, dyn + (size_t)warp * L.end)) take = inst;
+            if (sched_warp_instance<MM, CPL>(sp, cap, inst, dyn + (size_t)warp * L.end)) take = inst;
         }
     }
     if (lane == 0) s_takeover[warp] = take;
