@@ -672,8 +672,10 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
     sp.sort_cap = sort_cap;
     sp.zbuf_warps = c->sched_threads / 32;
     const SchedSmem L(sort_cap, P.Mmax, sp.bmax, kMaxModelsPerApp * kMaxBatchSizes, P.sumM, c->sched_threads / 32);
-    SP_CUDA(c, cudaFuncSetAttribute(k_sched<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.end));
-    SP_CUDA(c, cudaFuncSetAttribute(k_sched<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.end));
+    // instantiations: soft penalties or not, at most 4 applications or up to kMaxApps
+    void (*sched_kernel)(SchedParams) = P.any_soft ? (P.A <= 4 ? k_sched<true, 4> : k_sched<true, kMaxApps>)
+                                                   : (P.A <= 4 ? k_sched<false, 4> : k_sched<false, kMaxApps>);
+    SP_CUDA(c, cudaFuncSetAttribute(sched_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.end));
     SP_TRY(mark(c, c->ev_sched));
     // Batched mode, first call on a fresh table: one warp per instance takes every instance that fits its slice of
     // shared memory; k_sched follows for the rest (it returns at once when nothing is left).
@@ -724,8 +726,7 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
         sp.presorted = 1;
     }
     c->sched_started = true;
-    if (P.any_soft) k_sched<true><<<P.I, c->sched_threads, L.end, c->stream>>>(sp);
-    else k_sched<false><<<P.I, c->sched_threads, L.end, c->stream>>>(sp);
+    sched_kernel<<<P.I, c->sched_threads, L.end, c->stream>>>(sp);
     SP_TRY(launched(c, "k_sched"));
     return mark(c, c->ev_sched);
 }

@@ -282,7 +282,8 @@ __device__ __forceinline__ void warp_argmax(const double *cand_u, const int *can
 // All rounds of one instance by one thread block (every thread of the block calls it).  SOFT = false leaves the
 // linear and sigmoid penalties out of the code (every application has the step penalty): the round loop is a long
 // stretch of code that every warp walks through once per round, and what is not there is not fetched.
-template <bool SOFT>
+// MA bounds the applications of the instance: the priority sums are unrolled over it.
+template <bool SOFT, int MA>
 __device__ void sched_instance(const SchedParams &sp, const int inst) {
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ InstState st;
@@ -582,9 +583,9 @@ __device__ void sched_instance(const SchedParams &sp, const int inst) {
         // ---------------------------------------------------------------- 3. group priorities (Eq. 14)
         {
             // partial sums of every application first (their loads are in flight together), then one reduction
-            double part[kMaxApps];
+            double part[MA];
 #pragma unroll
-            for (int a = 0; a < kMaxApps; ++a) {
+            for (int a = 0; a < MA; ++a) {
                 part[a] = 0.0;
                 if (a < A) {
                     const double *pw = sp.q_pw[st.cur[a]] + s_base[a];
@@ -592,7 +593,7 @@ __device__ void sched_instance(const SchedParams &sp, const int inst) {
                 }
             }
 #pragma unroll
-            for (int a = 0; a < kMaxApps; ++a) {
+            for (int a = 0; a < MA; ++a) {
                 if (a < A) {
                     double v = part[a];
 #pragma unroll
@@ -771,7 +772,7 @@ __device__ void sched_instance(const SchedParams &sp, const int inst) {
     }
 }
 
-template <bool SOFT>
-__global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) { sched_instance<SOFT>(sp, blockIdx.x); }
+template <bool SOFT, int MA>
+__global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) { sched_instance<SOFT, MA>(sp, blockIdx.x); }
 
 }  // namespace sp
