@@ -688,7 +688,7 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
             // the block-wide scheduler runs inside the same kernel for the instances a warp hands over: its shared
             // memory is laid over the warps' slices
             const size_t wsmem = W.end * kWarpSchedWarps > L.end ? W.end * kWarpSchedWarps : L.end;
-            if (P.Mmax <= 8 && P.Mmax * P.nB <= 64) {          // short unrolled loops for small model and batch-size sets
+            if (P.Mmax <= 8 && P.Mmax * P.nB <= 64 && P.A <= 4) {   // short unrolled loops for small model, batch-size and application sets
                 SP_CUDA(c, cudaFuncSetAttribute(k_sched_warp<8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)wsmem));
                 k_sched_warp<8, 2><<<wgrid, kWarpSchedWarps * 32, wsmem, c->stream>>>(sp, (int)wcap);
             } else {

@@ -82,7 +82,8 @@ __device__ __forceinline__ void warp_sort(int64_t *dl, uint32_t *ida, int n) {
 // One instance by one warp.  Returns true when the block-wide scheduler has to take the instance over: a near-tie
 // to decide in fp64, more requests than the warp's slice holds, or an instance that had already started.
 // MM bounds the models per application and CPL the candidates per lane (models x batch sizes / 32): the loops over
-// them are unrolled, and the small instantiation keeps the code of a round short.
+// them are unrolled, and the small instantiation (which also stands for at most 4 applications) keeps the code of a
+// round short.
 template <int MM, int CPL>
 __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const int inst, unsigned char *mine) {
     const DevProfiles &P = sp.P;
@@ -387,7 +388,7 @@ k_sched_warp(SchedParams sp, int cap) {
     __syncthreads();                         // queues and state of a handed-over instance are in global memory
     for (int w = 0; w < kWarpSchedWarps; ++w) {
         if (s_takeover[w] >= 0) {
-            sched_instance<false, kMaxApps>(sp, s_takeover[w]);   // the warp path runs for step penalties only
+            sched_instance<false, (MM <= 8 ? 4 : kMaxApps)>(sp, s_takeover[w]);   // the warp path runs for step penalties only
             __syncthreads();
         }
     }
