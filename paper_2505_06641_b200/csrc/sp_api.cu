@@ -678,7 +678,7 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
     SP_CUDA(c, cudaFuncSetAttribute(sched_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.end));
     SP_TRY(mark(c, c->ev_sched));
     // Batched mode, first call on a fresh table: one warp per instance takes every instance that fits its slice of
-    // shared memory; k_sched follows for the rest (it returns at once when nothing is left).
+    // shared memory and, block-wide, the few it has to hand over; no k_sched launch is needed then.
     if (P.I > 1 && !c->opt.trace_mode && !c->sched_started && c->tb.n > 0 && !P.any_soft) {
         int64_t wcap = 32;
         while (wcap < (c->tb.n + P.I - 1) / P.I) wcap <<= 1;

@@ -8,11 +8,11 @@
 // latency and swap profiles in lane registers, one global round trip per round (the accuracy rows of the
 // candidate members).  Requests that are already hopeless at the starting clock are retired before the sort, so
 // only the survivors are sorted.
-// The kernel takes instances that have not started, are not in trace mode and fit the per-warp capacity.  It does
-// not contain the fp64 re-evaluation of near-ties (which keeps it small): when the two best group priorities or
-// candidate utilities of a round are closer than the guard band, the warp writes its queues and state out and
-// hands the instance to k_sched, which runs after this kernel in the same call and also takes the instances that
-// do not fit a warp.
+// A warp takes an instance that has not started, is not in trace mode and fits the per-warp capacity.  The warp
+// path does not contain the fp64 re-evaluation of near-ties (which keeps it small): when the two best group
+// priorities or candidate utilities of a round are closer than the guard band, the warp writes its queues and
+// state out in k_sched's format; after a block barrier the four warps of the block run the block-wide scheduler
+// (sched_instance, the body of k_sched) for those instances and for the ones that do not fit a warp.
 #pragma once
 
 #include "sp_common.cuh"
