@@ -670,8 +670,11 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
     int sort_cap = P.I > 1 ? 1024 : 8192;
     while (sort_cap > 64 && sort_cap / 2 >= per_inst) sort_cap /= 2;
     sp.sort_cap = sort_cap;
-    sp.zbuf_warps = c->sched_threads / 32;
-    const SchedSmem L(sort_cap, P.Mmax, sp.bmax, kMaxModelsPerApp * kMaxBatchSizes, P.sumM, c->sched_threads / 32);
+    // a single instance with a short table is faster with half the threads (cheaper block barriers); the scratch
+    // buffers are sized for the full block
+    const int nt = P.I == 1 && !c->opt.trace_mode && c->tb.n <= 8192 ? 512 : c->sched_threads;
+    sp.zbuf_warps = nt / 32;
+    const SchedSmem L(sort_cap, P.Mmax, sp.bmax, kMaxModelsPerApp * kMaxBatchSizes, P.sumM, nt / 32);
     // instantiations: soft penalties or not, at most 4 applications or up to kMaxApps
     void (*sched_kernel)(SchedParams) = P.any_soft ? (P.A <= 4 ? k_sched<true, 4> : k_sched<true, kMaxApps>)
                                                    : (P.A <= 4 ? k_sched<false, 4> : k_sched<false, kMaxApps>);
@@ -726,7 +729,7 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
         sp.presorted = 1;
     }
     c->sched_started = true;
-    sched_kernel<<<P.I, c->sched_threads, L.end, c->stream>>>(sp);
+    sched_kernel<<<P.I, nt, L.end, c->stream>>>(sp);
     SP_TRY(launched(c, "k_sched"));
     return mark(c, c->ev_sched);
 }
