@@ -675,9 +675,12 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
     const int nt = P.I == 1 && !c->opt.trace_mode && c->tb.n <= 8192 ? 512 : c->sched_threads;
     sp.zbuf_warps = nt / 32;
     const SchedSmem L(sort_cap, P.Mmax, sp.bmax, kMaxModelsPerApp * kMaxBatchSizes, P.sumM, nt / 32);
-    // instantiations: soft penalties or not, at most 4 applications or up to kMaxApps
-    void (*sched_kernel)(SchedParams) = P.any_soft ? (P.A <= 4 ? k_sched<true, 4> : k_sched<true, kMaxApps>)
-                                                   : (P.A <= 4 ? k_sched<false, 4> : k_sched<false, kMaxApps>);
+    // instantiations: soft penalties or not, at most 4 applications or up to kMaxApps, long queues (one large snapshot)
+    const bool longq = P.I == 1 && !c->opt.trace_mode && c->tb.n > 16384;
+    void (*sched_kernel)(SchedParams) =
+        P.any_soft ? (P.A <= 4 ? k_sched<true, 4, false> : k_sched<true, kMaxApps, false>)
+                   : (P.A <= 4 ? (longq ? k_sched<false, 4, true> : k_sched<false, 4, false>)
+                               : (longq ? k_sched<false, kMaxApps, true> : k_sched<false, kMaxApps, false>));
     SP_CUDA(c, cudaFuncSetAttribute(sched_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.end));
     SP_TRY(mark(c, c->ev_sched));
     // Batched mode, first call on a fresh table: one warp per instance takes every instance that fits its slice of

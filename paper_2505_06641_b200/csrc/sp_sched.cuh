@@ -282,8 +282,10 @@ __device__ __forceinline__ void warp_argmax(const double *cand_u, const int *can
 // All rounds of one instance by one thread block (every thread of the block calls it).  SOFT = false leaves the
 // linear and sigmoid penalties out of the code (every application has the step penalty): the round loop is a long
 // stretch of code that every warp walks through once per round, and what is not there is not fetched.
-// MA bounds the applications of the instance: the priority sums are unrolled over it.
-template <bool SOFT, int MA>
+// MA bounds the applications of the instance: the priority sums are unrolled over it.  LONGQ: the queues are long
+// (a large snapshot), so the priority sums keep four loads in flight per thread; short-queue workloads do without
+// that code.
+template <bool SOFT, int MA, bool LONGQ>
 __device__ void sched_instance(const SchedParams &sp, const int inst) {
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ InstState st;
@@ -589,7 +591,16 @@ __device__ void sched_instance(const SchedParams &sp, const int inst) {
                 part[a] = 0.0;
                 if (a < A) {
                     const double *pw = sp.q_pw[st.cur[a]] + s_base[a];
-                    for (int k = st.head[a] + tid; k < st.tail[a]; k += NT) part[a] += pw[k];
+                    int k = st.head[a] + tid;
+                    if (LONGQ) {                      // read at the SM's bandwidth, not at one round trip per element
+                        const int tail = st.tail[a];
+                        double p1 = 0.0, p2 = 0.0, p3 = 0.0;
+                        for (; k + 3 * NT < tail; k += 4 * NT) {
+                            part[a] += pw[k]; p1 += pw[k + NT]; p2 += pw[k + 2 * NT]; p3 += pw[k + 3 * NT];
+                        }
+                        part[a] += (p1 + p2) + p3;
+                    }
+                    for (; k < st.tail[a]; k += NT) part[a] += pw[k];
                 }
             }
 #pragma unroll
@@ -772,7 +783,7 @@ __device__ void sched_instance(const SchedParams &sp, const int inst) {
     }
 }
 
-template <bool SOFT, int MA>
-__global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) { sched_instance<SOFT, MA>(sp, blockIdx.x); }
+template <bool SOFT, int MA, bool LONGQ>
+__global__ void __launch_bounds__(1024, 1) k_sched(SchedParams sp) { sched_instance<SOFT, MA, LONGQ>(sp, blockIdx.x); }
 
 }  // namespace sp

@@ -388,7 +388,7 @@ k_sched_warp(SchedParams sp, int cap) {
     __syncthreads();                         // queues and state of a handed-over instance are in global memory
     for (int w = 0; w < kWarpSchedWarps; ++w) {
         if (s_takeover[w] >= 0) {
-            sched_instance<false, (MM <= 8 ? 4 : kMaxApps)>(sp, s_takeover[w]);   // the warp path runs for step penalties only
+            sched_instance<false, (MM <= 8 ? 4 : kMaxApps), false>(sp, s_takeover[w]);   // the warp path runs for step penalties only
             __syncthreads();
         }
     }
