@@ -238,10 +238,12 @@ __device__ __forceinline__ double penalty_gamma(int kind, int64_t d, int64_t del
     const double r = __ddiv_rn(__dsub_rn(1.0, x), x);
     return __ddiv_rn(1.0, __dadd_rn(1.0, __dmul_rn(__dmul_rn(r, r), r)));
 }
-// No utility is left at completion time e: the request can be retired.
+// No utility is left at completion time e: the request can be retired.  For the soft penalties that is gamma >= 1
+// evaluated as the utility evaluates it (fp64): the sigmoid rounds to 1 a little before the request is late by its
+// whole relative deadline, and a request with gamma = 1 earns nothing whether it is retired or served.
 __device__ __forceinline__ bool penalty_hopeless(int kind, int64_t d, int64_t delta, int64_t e) {
     if (kind == SP_PEN_STEP || delta <= 0) return d < e;
-    return e > d && e - d >= delta;
+    return penalty_gamma(kind, d, delta, e) >= 1.0;
 }
 
 __device__ __forceinline__ double prio_weight(double v, int64_t dl, int64_t tref, double tau) {
@@ -500,13 +502,14 @@ __device__ void sched_instance(const SchedParams &sp, const int inst) {
             __syncthreads();
         }
         // ---------------------------------------------------------------- 2. retire hopeless requests
-        if (tid < A) {                        // earliest completion any candidate of the application can reach
+        // earliest completion any candidate of the application can reach: every model by its own thread, then the
+        // minimum per application (the candidate table is free at this point of the round)
+        if (tid < P.sumM) cand_e[tid] = st.T + (tid != st.L ? sw[tid] : 0) + al[tid] + be[tid] * (int64_t)P.batch[0];
+        __syncthreads();
+        if (tid < A) {
             const int a = tid;
             int64_t emin = INT64_MAX;
-            for (int g = P.mfirst[a]; g < P.mfirst[a + 1]; ++g) {
-                const int64_t e = st.T + (g != st.L ? sw[g] : 0) + al[g] + be[g] * (int64_t)P.batch[0];
-                emin = e < emin ? e : emin;
-            }
+            for (int g = P.mfirst[a]; g < P.mfirst[a + 1]; ++g) emin = cand_e[g] < emin ? cand_e[g] : emin;
             s_emin[a] = emin;
             s_lo[a] = st.head[a]; s_hi[a] = st.tail[a]; s_pdone[a] = st.tail[a] == st.head[a];
         }

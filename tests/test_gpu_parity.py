@@ -312,3 +312,13 @@ def test_random_shapes_match_oracle(name, kw):
     worst = check_scores(res, s)
     check_schedule(w, res, od)
     assert worst < ACC_RTOL
+
+
+def test_sigmoid_penalty_that_rounds_to_one_retires_the_request():
+    """A request late by all but a few millionths of its relative deadline has a sigmoid penalty that is 1.0 in
+    fp64: it is retired like the oracle retires it (found by a random sweep: one of these 1,500 instances has two)."""
+    w = synth.make_workload("C4", n_apps=4, models=1, n_classes=24, feat_dim=128, n_requests=329, n_instances=1500)
+    w.penalty_kind = np.array([0, 2, 1, 2], dtype=np.int32)
+    s, od, res = _both(w)
+    check_scores(res, s)
+    check_schedule(w, res, od)
