@@ -139,6 +139,18 @@ def test_soft_penalties_anchor_points_and_monotonicity(kind):
         assert g[250] + g[750] == pytest.approx(1.0, abs=1e-15) and g[250] < 0.25
 
 
+def test_sigmoid_penalty_reaches_one_in_fp64_just_before_the_whole_relative_deadline():
+    """1 / (1 + ((1 - x) / x)^3) rounds to 1.0 once ((1 - x) / x)^3 drops below half an ulp of 1, i.e. from
+    x = 1 - 4.8e-6 on; the linear penalty stays below 1 until x = 1.  The purge rule (gamma >= 1) therefore retires a
+    sigmoid request that is late by all but a few millionths of its relative deadline."""
+    from oracle import oracle
+    arrival, d = 0, 1_000_000_000                         # relative deadline 1 s
+    for late_ns, expect_one in ((999_990_000, False), (999_996_000, True), (999_999_999, True)):
+        g = oracle.penalty(2, d, arrival, d + late_ns)
+        assert (g == 1.0) == expect_one and g <= 1.0
+        assert oracle.penalty(1, d, arrival, d + late_ns) < 1.0
+
+
 def test_step_penalty_and_degenerate_relative_deadline():
     from oracle import oracle
     assert oracle.penalty(0, 10, 0, 10) == 0.0 and oracle.penalty(0, 10, 0, 11) == 1.0
