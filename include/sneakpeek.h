@@ -41,7 +41,10 @@ typedef enum {
 enum { SP_F32 = 0, SP_BF16 = 1 };                       /* feature / head-weight storage type */
 /* Penalty gamma of Eq. 2 (Section 5.1).  STEP: 1 once the deadline is missed.  LINEAR and SIGMOID degrade the utility
  * after the deadline d over the request's relative deadline delta = d - arrival: with x = (completion - d) / delta,
- * gamma = min(max(x, 0), 1) (LINEAR) or 0 for x <= 0, 1 for x >= 1, 1 / (1 + ((1 - x) / x)^3) in between (SIGMOID). */
+ * gamma = min(max(x, 0), 1) (LINEAR) or 0 for x <= 0, 1 for x >= 1, 1 / (1 + ((1 - x) / x)^3) in between (SIGMOID).
+ * gamma is evaluated in fp64; a pending request whose gamma is 1 for the earliest completion any candidate of its
+ * application can still reach is retired as SP_EXPIRED (for SIGMOID that is from x = 1 - 4.8e-6 on, where the
+ * expression rounds to 1). */
 enum { SP_PEN_STEP = 0, SP_PEN_LINEAR = 1, SP_PEN_SIGMOID = 2 };
 enum { SP_PENDING = 0, SP_SCHEDULED = 1, SP_EXPIRED = 2 };
 
