@@ -44,6 +44,7 @@ def parse_args():
     ap.add_argument("--cpu-sample-instances", type=int, default=4096)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-side-workloads", action="store_true", help="skip the short C3 and C5 passes of the default run")
     return ap.parse_args()
 
 
@@ -98,6 +99,70 @@ def cpu_oracle_sample(args):
     cpu_oracle_time(w)                                          # load the library, touch the pages
     dt, _ = cpu_oracle_time(w)
     return w.n_requests / dt, oracle.num_threads(), what + ", score+drain %.2f s" % dt
+
+
+KERNEL_NAMES = ("k_score_tiled", "k_score_small", "k_score_mma", "k_score_gemm<bf16>", "k_score_gemm<f32>")
+
+
+def roofline_entry(w, n, kernel, score_ms, peaks, traffic):
+    """Roofline object of the scoring kernel of workload ``w`` (n requests per launch, score_ms per launch)."""
+    if kernel.startswith("k_score_gemm"):
+        # the head is a dense contraction far above the HBM ridge: bound by the tensor pipe.  The kernel is short and
+        # timed by its own events, so the burst figure of the measured bf16 peak applies; the fp32 flavour runs on the
+        # tf32 unit (nominal ratio to bf16: 0.5) and needs three MMA passes for fp32 accuracy, but the algorithmic
+        # flops (2 n D C) are what is counted.
+        f32 = kernel.endswith("<f32>")
+        flops = 2.0 * n * int(w.feat_dim) * int(w.n_classes)
+        peak, peak_src = (float(peaks["bf16_tflops"]), "measured") if peaks else (1590.0, "fallback")
+        if f32:
+            peak, peak_src = peak * 0.5, peak_src + " bf16 x 0.5 (tf32)"
+        achieved = flops / (score_ms * 1e-3) / 1e12 if score_ms > 0 else None
+        return {"bound": "tensor", "kernel": kernel, "achieved": achieved, "peak": peak, "peak_source": peak_src,
+                "unit": "TFLOP/s", "frac": achieved / peak if achieved else None, "traffic": traffic,
+                "algorithmic_flops": flops, "mma_passes": 3 if f32 else 1,
+                "algorithmic_bytes": algorithmic_bytes_per_request(w) * n, "kernel_ms": score_ms}
+    bytes_per_launch = algorithmic_bytes_per_request(w) * n
+    peak, peak_src = (float(peaks["hbm_gbs"]), "measured") if peaks else (6650.0, "fallback")
+    achieved = bytes_per_launch / (score_ms * 1e-3) / 1e9 if score_ms > 0 else None
+    return {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "peak_source": peak_src,
+            "unit": "GB/s", "frac": achieved / peak if achieved else None, "traffic": traffic,
+            "algorithmic_bytes": bytes_per_launch, "kernel_ms": score_ms}
+
+
+def side_workload(name, steps, peaks, device):
+    """A short pass over another full-size configuration (score + drain, inputs resident), for the record beside the
+    headline workload: step time, scoring-kernel roofline, scheduling time per round."""
+    import torch
+    from paper_2505_06641_b200 import api, runner, synth
+    w = synth.make_workload(name)
+    n = w.n_requests
+    ses = runner.Session(w, device=device)
+    api.sp_set_options(ses.ctx, trace_mode=bool(w.trace_mode), timing=True)
+    ses.upload()
+    ses.alloc_outputs(max(1, min(n, 1 << 16)))
+    for _ in range(3):
+        ses.score(); ses.schedule(n + 1)
+    api.sp_check(ses.ctx)
+    api.sp_get_stats(ses.ctx)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        ses.score(); ses.schedule(n + 1)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    api.sp_check(ses.ctx)
+    st = api.sp_get_stats(ses.ctx)
+    rounds = int(ses.n_done.sum().item())
+    score_ms = st["score_kernel_ms"] / max(1, st["score_calls"])
+    sched_ms = st["sched_kernel_ms"] / max(1, st["sched_calls"])
+    kernel = KERNEL_NAMES[int(st["score_kernel"])]
+    ses.close()
+    return {"workload": name, "requests": n, "steps": steps, "ms_per_step": ms, "requests_per_s": n / (ms * 1e-3),
+            "roofline": roofline_entry(w, n, kernel, score_ms, peaks, None), "sched_kernel_ms": sched_ms,
+            "rounds_per_step": rounds, "us_per_round": sched_ms * 1e3 / max(1, rounds),
+            "l2": "features %.2f GB per step" % (w.feats.nbytes / 1e9)}
 
 
 class ClockSampler:
@@ -234,7 +299,7 @@ def main():
     # ---- roofline of the dominant kernel (the scoring kernel), from CUDA events recorded around it
     score_ms = st["score_kernel_ms"] / max(1, st["score_calls"])
     sched_ms = st["sched_kernel_ms"] / max(1, st["sched_calls"])
-    kernel = ("k_score_tiled", "k_score_small", "k_score_mma", "k_score_gemm<bf16>", "k_score_gemm<f32>")[int(st.get("score_kernel", 0))]
+    kernel = KERNEL_NAMES[int(st.get("score_kernel", 0))]
     peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     peaks = json.load(open(peaks_path)) if os.path.exists(peaks_path) else None
     traffic = None
@@ -243,28 +308,7 @@ def main():
         tj = json.load(open(tpath)).get(args.workload)
         if tj and tj.get("kernel_version") == KERNEL_VERSION:
             traffic = tj["dram_bytes_per_request"] * n
-    if kernel.startswith("k_score_gemm"):
-        # the head is a dense contraction far above the HBM ridge: bound by the tensor pipe.  The kernel is short and
-        # timed by its own events, so the burst figure of the measured bf16 peak applies; the fp32 flavour runs on the
-        # tf32 unit (nominal ratio to bf16: 0.5) and needs three MMA passes for fp32 accuracy, but the algorithmic
-        # flops (2 n D C) are what is counted.
-        f32 = kernel.endswith("<f32>")
-        flops = 2.0 * n * int(w.feat_dim) * int(w.n_classes)
-        peak, peak_src = (float(peaks["bf16_tflops"]), "measured") if peaks else (1590.0, "fallback")
-        if f32:
-            peak, peak_src = peak * 0.5, peak_src + " bf16 x 0.5 (tf32)"
-        achieved = flops / (score_ms * 1e-3) / 1e12 if score_ms > 0 else None
-        roofline = {"bound": "tensor", "kernel": kernel, "achieved": achieved, "peak": peak, "peak_source": peak_src,
-                    "unit": "TFLOP/s", "frac": achieved / peak if achieved else None, "traffic": traffic,
-                    "algorithmic_flops": flops, "mma_passes": 3 if f32 else 1,
-                    "algorithmic_bytes": algorithmic_bytes_per_request(w) * n, "kernel_ms": score_ms}
-    else:
-        bytes_per_launch = algorithmic_bytes_per_request(w) * n
-        peak, peak_src = (float(peaks["hbm_gbs"]), "measured") if peaks else (6650.0, "fallback")
-        achieved = bytes_per_launch / (score_ms * 1e-3) / 1e9 if score_ms > 0 else None
-        roofline = {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "peak_source": peak_src,
-                    "unit": "GB/s", "frac": achieved / peak if achieved else None, "traffic": traffic,
-                    "algorithmic_bytes": bytes_per_launch, "kernel_ms": score_ms}
+    roofline = roofline_entry(w, n, kernel, score_ms, peaks, traffic)
 
     # ---- one scheduling round per call (launch, the round, synchronise): the latency a caller sees per decision
     ses.score()
@@ -306,6 +350,13 @@ def main():
         e2e = {"value": n_total / (dt / e2e_steps), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                "d2h_bytes_per_step": int(d2h), "ms_per_step": dt / e2e_steps * 1e3, "steps": e2e_steps}
     ses.close()
+    del ses
+    torch.cuda.empty_cache()
+
+    # ---- the other two large configurations, a few steps each, for the record (single-GPU run of the default only)
+    others = None
+    if rank == 0 and world == 1 and args.workload == "C4" and args.instances is None and not args.no_side_workloads:
+        others = [side_workload("C3", 3, peaks, local), side_workload("C5", 2, peaks, local)]
 
     if rank == 0:
         out = {
@@ -321,7 +372,7 @@ def main():
                       "us_per_round_amortised": sched_ms * 1e3 / max(1, n_rounds_total),
                       "us_single_round_call": us_single_round_call,
                       "exact_utility_rounds": st["exact_utility"], "exact_priority_rounds": st["exact_priority"],
-                      "exact_rows": st["exact_rows"]},
+                      "exact_rows": st["exact_rows"], "other_workloads": others},
         }
         print(json.dumps(out))
     if world > 1:

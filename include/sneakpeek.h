@@ -42,9 +42,9 @@ enum { SP_F32 = 0, SP_BF16 = 1 };                       /* feature / head-weight
 /* Penalty gamma of Eq. 2 (Section 5.1).  STEP: 1 once the deadline is missed.  LINEAR and SIGMOID degrade the utility
  * after the deadline d over the request's relative deadline delta = d - arrival: with x = (completion - d) / delta,
  * gamma = min(max(x, 0), 1) (LINEAR) or 0 for x <= 0, 1 for x >= 1, 1 / (1 + ((1 - x) / x)^3) in between (SIGMOID).
- * gamma is evaluated in fp64; a pending request whose gamma is 1 for the earliest completion any candidate of its
- * application can still reach is retired as SP_EXPIRED (for SIGMOID that is from x = 1 - 4.8e-6 on, where the
- * expression rounds to 1). */
+ * gamma is evaluated in fp64.  A pending request at the head of its queue that is hopeless -- the earliest completion
+ * any candidate of its application can still reach misses the deadline (STEP) or lies a whole relative deadline or
+ * more after it (x >= 1, tested on the integer times) -- is retired as SP_EXPIRED. */
 enum { SP_PEN_STEP = 0, SP_PEN_LINEAR = 1, SP_PEN_SIGMOID = 2 };
 enum { SP_PENDING = 0, SP_SCHEDULED = 1, SP_EXPIRED = 2 };
 
@@ -101,7 +101,8 @@ typedef struct {
 typedef struct {
     int32_t trace_mode;   /* 0: every scored request is pending at once; 1: a request joins when arrival <= clock */
     int32_t timing;       /* 1: bracket the scoring and the scheduling kernel with CUDA events (see sp_stats) */
-    double guard_utility; /* relative margin under which candidate utilities are re-evaluated in fp64 (default 2e-5) */
+    double guard_utility; /* relative margin under which candidate utilities are re-evaluated in fp64; 0 = the
+                             default (2e-5), so a zero-initialised struct is safe; (0, 1]: that margin */
     double guard_priority;/* same for group priorities (default 2e-6) */
 } sp_options;
 
@@ -130,6 +131,9 @@ const char *sp_last_error(const sp_ctx *ctx);
  * model resident.  SP_EINVAL on a bad shape/value, naming it in sp_last_error(). */
 sp_status sp_load_profiles(sp_ctx *ctx, const sp_profiles *profiles);
 
+/* Fills *out (HOST) with the defaults: snapshot mode, no timing, the default guards.  Needs no GPU. */
+void sp_default_options(sp_options *out);
+/* Replaces the context's options.  Guards must lie in [0, 1]; 0 selects the default. */
 sp_status sp_set_options(sp_ctx *ctx, const sp_options *opt);
 
 /* Sets the clock T and the resident model L (global id, -1 = none) of one instance, or of all (instance = -1). */
@@ -201,9 +205,14 @@ sp_status sp_run_host(sp_ctx *ctx, int64_t n, const void *feats, const int32_t *
  * at start-up -- a serving process that has given all remaining memory to its own pool, or a real-time loop
  * in which a driver allocation (which may block or fail) is not acceptable -- so the context-based calls
  * above, which grow their buffers with cudaMalloc, are closed to them.  This call does steps a1-a4 of
- * sp_score() for ONE instance (no Dirichlet prior) and allocates nothing, neither through CUDA nor through any
- * library: its scratch (per-application counters, prefix sums, the request permutation; about 0.5 MB) is a
- * fixed array inside the library image, which every GPU that loads the library holds until the process ends.
+ * sp_score() for ONE instance (no Dirichlet prior) and requests no device memory, neither through CUDA nor
+ * through any library: its scratch (per-application counters, prefix sums, the request permutation; about
+ * 0.5 MB) is a fixed array inside the library image, which every GPU that loads the library holds until the
+ * process ends.  That claim is about the second and later calls on a device.  The FIRST call on a device makes
+ * the device current, which creates its primary context and loads the library's module (the 0.5 MB array
+ * included) if nothing has done so yet: those are driver allocations, so make that first call at start-up,
+ * before the memory budget is handed out.  Like the context-based calls, every call leaves `device` the calling
+ * thread's current device.  Error texts are formatted on the host heap.
  *
  *   head      HOST struct; models_per_app is a HOST array, head_w [A][D][C], head_b [A][C], recall [sumM][C]
  *             are DEVICE arrays (inputs, the caller's).

@@ -184,10 +184,16 @@ double orc_penalty(int kind, int64_t d, int64_t arrival, int64_t e)
     return 1.0 / (1.0 + r * r * r);
 }
 
-/* A request is hopeless when even the earliest completion `emin` its group can reach leaves it no utility. */
+/* A request is hopeless when even the earliest completion `emin` its group can reach leaves it no utility:
+ * gamma = 1 there.  Stated on the integer times, not on the rounded value of gamma: under the step penalty the
+ * deadline precedes emin; under the soft penalties x >= 1, i.e. emin is at least the whole relative deadline
+ * after the deadline (the sigmoid expression rounds to 1.0 in fp64 slightly before x reaches 1; such a request
+ * is not hopeless yet, it merely earns nothing if served then). */
 static int hopeless(int kind, int64_t d, int64_t arrival, int64_t emin)
 {
-    return orc_penalty(kind, d, arrival, emin) >= 1.0;
+    const int64_t delta = d - arrival;
+    if (kind == ORC_PEN_STEP || delta <= 0) return d < emin;
+    return emin - d >= delta;
 }
 
 /* ---------------------------------------------------------------------------------------------

@@ -28,7 +28,7 @@ REQ_DTYPE = np.dtype([("status", "<i4"), ("round", "<i4"), ("model", "<i4"), ("p
                      align=True)
 assert ROUND_DTYPE.itemsize == 64 and REQ_DTYPE.itemsize == 24
 
-EXPORTS = ["sp_create", "sp_destroy", "sp_last_error", "sp_load_profiles", "sp_set_options", "sp_set_clock",
+EXPORTS = ["sp_create", "sp_destroy", "sp_last_error", "sp_load_profiles", "sp_default_options", "sp_set_options", "sp_set_clock",
            "sp_set_clocks", "sp_score", "sp_get_scores", "sp_schedule_round", "sp_get_requests", "sp_get_clocks",
            "sp_reset", "sp_check", "sp_get_stats", "sp_run_host", "sp_score_static"]
 
@@ -86,6 +86,8 @@ def load_library():
     lib.sp_last_error.restype = C.c_char_p
     lib.sp_load_profiles.argtypes = [vp, C.POINTER(_Profiles)]
     lib.sp_set_options.argtypes = [vp, C.POINTER(_Options)]
+    lib.sp_default_options.argtypes = [C.POINTER(_Options)]
+    lib.sp_default_options.restype = None
     lib.sp_set_clock.argtypes = [vp, i32, i64, i32]
     lib.sp_set_clocks.argtypes = [vp, vp, vp]
     lib.sp_score.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp]
@@ -99,7 +101,7 @@ def load_library():
     lib.sp_run_host.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, i64, vp]
     lib.sp_score_static.argtypes = [C.c_int, vp, C.POINTER(_StaticHead), i64, vp, vp, vp, vp, C.c_char_p, i32]
     for name in EXPORTS:
-        if name not in ("sp_destroy", "sp_last_error"):
+        if name not in ("sp_destroy", "sp_last_error", "sp_default_options"):
             getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
@@ -159,6 +161,12 @@ def sp_load_profiles(ctx: int, w) -> None:
                   float(w.evidence_k), _host(keep["recall"]), _host(keep["al"]), _host(keep["be"]), _host(keep["sw"]),
                   _host(keep["bs"]), int(keep["bs"].shape[0]), _host(keep["pen"]), float(w.prio_time_scale_s))
     _ok(ctx, load_library().sp_load_profiles(ctx, C.byref(p)))
+
+
+def sp_default_options() -> dict:
+    o = _Options()
+    load_library().sp_default_options(C.byref(o))
+    return {k: getattr(o, k) for k, _ in _Options._fields_}
 
 
 def sp_set_options(ctx: int, trace_mode: bool = False, guard_utility: float = 2e-5,

@@ -20,6 +20,8 @@ using namespace sp;
 
 namespace {
 
+constexpr double kDefaultGuardUtility = 2e-5, kDefaultGuardPriority = 2e-6;
+
 struct Buf {                     // a device allocation that only grows
     void *p = nullptr;
     size_t bytes = 0;
@@ -41,7 +43,7 @@ struct sp_ctx {
     HostProfiles hp;
     DevProfiles P{};
     DevTable tb{};
-    sp_options opt{0, 0, 2e-5, 2e-6};
+    sp_options opt{0, 0, kDefaultGuardUtility, kDefaultGuardPriority};
     std::vector<cudaEvent_t> ev_score, ev_sched;   // start/stop pairs recorded since the last sp_get_stats
     int64_t launches = 0;
     int sched_threads = 1024;
@@ -451,6 +453,12 @@ sp_status sp_load_profiles(sp_ctx *c, const sp_profiles *p) {
     return SP_OK;
 }
 
+void sp_default_options(sp_options *out) {
+    if (!out) return;
+    out->trace_mode = 0; out->timing = 0;
+    out->guard_utility = kDefaultGuardUtility; out->guard_priority = kDefaultGuardPriority;
+}
+
 sp_status sp_set_options(sp_ctx *c, const sp_options *o) {
     if (!c) return SP_EINVAL;
     if (!o || !(o->guard_utility >= 0.0) || !(o->guard_priority >= 0.0) || o->guard_utility > 1.0 || o->guard_priority > 1.0)
@@ -458,6 +466,9 @@ sp_status sp_set_options(sp_ctx *c, const sp_options *o) {
     if (c->have_table && (o->trace_mode != 0) != (c->opt.trace_mode != 0))
         return fail(c, SP_ESTATE, "trace_mode cannot change while requests are scored; call sp_reset first");
     c->opt = *o;
+    // a zero-initialised struct asks for the defaults, not for decisions on fp32 sums without a guard band
+    if (c->opt.guard_utility == 0.0) c->opt.guard_utility = kDefaultGuardUtility;
+    if (c->opt.guard_priority == 0.0) c->opt.guard_priority = kDefaultGuardPriority;
     return SP_OK;
 }
 
@@ -685,7 +696,8 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
     SP_TRY(mark(c, c->ev_sched));
     // Batched mode, first call on a fresh table: one warp per instance takes every instance that fits its slice of
     // shared memory and, block-wide, the few it has to hand over; no k_sched launch is needed then.
-    if (P.I > 1 && !c->opt.trace_mode && !c->sched_started && c->tb.n > 0 && !P.any_soft) {
+    // (A call for zero rounds changes nothing: it goes to k_sched, which returns before touching any queue.)
+    if (P.I > 1 && !c->opt.trace_mode && !c->sched_started && c->tb.n > 0 && !P.any_soft && max_rounds > 0) {
         int64_t wcap = 32;
         while (wcap < (c->tb.n + P.I - 1) / P.I) wcap <<= 1;
         const WarpSchedSmem W((int)wcap, P.Mmax, sp.bmax);
@@ -708,7 +720,7 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
         }
     }
     // One large snapshot instance: its keys are sorted by the whole GPU first (k_sched would use one block for it).
-    if (P.I == 1 && !c->opt.trace_mode && !c->sched_started && c->tb.n > sort_cap && c->tb.n < ((int64_t)1 << 31)) {
+    if (P.I == 1 && !c->opt.trace_mode && !c->sched_started && max_rounds > 0 && c->tb.n > sort_cap && c->tb.n < ((int64_t)1 << 31)) {
         const int64_t n = c->tb.n;
         SortKey *keys = (SortKey *)c->sort_scratch.p;
         k_presort_keys<<<(unsigned)((n + 255) / 256), 256, 0, c->stream>>>(c->tb, keys, n);
@@ -731,7 +743,7 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
         }
         sp.presorted = 1;
     }
-    c->sched_started = true;
+    if (max_rounds > 0) c->sched_started = true;
     sched_kernel<<<P.I, nt, L.end, c->stream>>>(sp);
     SP_TRY(launched(c, "k_sched"));
     return mark(c, c->ev_sched);

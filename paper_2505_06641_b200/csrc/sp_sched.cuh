@@ -238,12 +238,11 @@ __device__ __forceinline__ double penalty_gamma(int kind, int64_t d, int64_t del
     const double r = __ddiv_rn(__dsub_rn(1.0, x), x);
     return __ddiv_rn(1.0, __dadd_rn(1.0, __dmul_rn(__dmul_rn(r, r), r)));
 }
-// No utility is left at completion time e: the request can be retired.  For the soft penalties that is gamma >= 1
-// evaluated as the utility evaluates it (fp64): the sigmoid rounds to 1 a little before the request is late by its
-// whole relative deadline, and a request with gamma = 1 earns nothing whether it is retired or served.
+// No utility is left at completion time e: the request can be retired.  An exact test on the integer times: the
+// deadline is missed (step), or e is a whole relative deadline or more after the deadline (soft penalties, x >= 1).
 __device__ __forceinline__ bool penalty_hopeless(int kind, int64_t d, int64_t delta, int64_t e) {
     if (kind == SP_PEN_STEP || delta <= 0) return d < e;
-    return penalty_gamma(kind, d, delta, e) >= 1.0;
+    return e - d >= delta;
 }
 
 __device__ __forceinline__ double prio_weight(double v, int64_t dl, int64_t tref, double tau) {

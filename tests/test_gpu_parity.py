@@ -314,11 +314,52 @@ def test_random_shapes_match_oracle(name, kw):
     assert worst < ACC_RTOL
 
 
-def test_sigmoid_penalty_that_rounds_to_one_retires_the_request():
+def test_sigmoid_penalty_that_rounds_to_one_before_the_request_is_hopeless():
     """A request late by all but a few millionths of its relative deadline has a sigmoid penalty that is 1.0 in
-    fp64: it is retired like the oracle retires it (found by a random sweep: one of these 1,500 instances has two)."""
+    fp64 although x < 1: it is not hopeless yet (the test is on the integer times) and, if served then, earns exactly
+    nothing, on both sides (one of these 1,500 instances has two such requests)."""
     w = synth.make_workload("C4", n_apps=4, models=1, n_classes=24, feat_dim=128, n_requests=329, n_instances=1500)
     w.penalty_kind = np.array([0, 2, 1, 2], dtype=np.int32)
     s, od, res = _both(w)
     check_scores(res, s)
     check_schedule(w, res, od)
+
+
+@pytest.mark.parametrize("name,kw", [("C4", dict(n_instances=9)), ("C1", {})])
+def test_a_call_for_zero_rounds_changes_nothing(name, kw):
+    """sp_schedule_round(max_rounds = 0) retires nothing and starts nothing, in batched mode as for one instance: the
+    clock can still be set afterwards, and the rounds that follow are the oracle's."""
+    from oracle import oracle
+    from paper_2505_06641_b200 import api, runner
+    w = synth.make_workload(name, **kw)
+    s = oracle.score(w)
+    od = oracle.drain(w, s.acc, s.v)
+    ses = runner.Session(w)
+    ses.upload(); ses.alloc_outputs(600); ses.score()
+    ses.schedule(0)
+    api.sp_check(ses.ctx)
+    api.sp_get_requests(ses.ctx, 0, ses.n, ses.recs)
+    reqs = ses.recs.cpu().numpy().reshape(-1).view(api.REQ_DTYPE)[:ses.n]
+    assert np.all(reqs["status"] == api.SP_PENDING) and int(ses.n_done.sum()) == 0
+    api.sp_set_clocks(ses.ctx, ses.dev["t0"], ses.dev["l0"])
+    ses.schedule(10_000)
+    api.sp_check(ses.ctx)
+    api.sp_get_requests(ses.ctx, 0, ses.n, ses.recs)
+    reqs = ses.recs.cpu().numpy().reshape(-1).view(api.REQ_DTYPE)[:ses.n]
+    for f in ("status", "round", "model", "order"):
+        assert np.array_equal(reqs[f], od.reqs[f]), f
+    assert np.array_equal(ses.n_done.cpu().numpy(), od.n_rounds)
+    ses.close()
+
+
+def test_zero_guards_select_the_defaults():
+    """A zero-initialised options struct must not switch the fp64 re-evaluation of near-ties off."""
+    from paper_2505_06641_b200 import api, runner
+    w = synth.make_workload("C4", n_instances=300)
+    ses = runner.Session(w)
+    ref = ses.run()
+    api.sp_set_options(ses.ctx, trace_mode=False, guard_utility=0.0, guard_priority=0.0)
+    got = ses.run()
+    ses.close()
+    assert np.array_equal(ref.reqs, got.reqs)
+    assert got.stats["exact_utility"] + got.stats["exact_priority"] == ref.stats["exact_utility"] + ref.stats["exact_priority"]

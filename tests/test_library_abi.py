@@ -48,6 +48,13 @@ def test_no_silent_fallback_without_a_gpu(lib):
         runner.Session(synth.make_workload("C1"))
 
 
+def test_default_options_need_no_gpu(lib):
+    from paper_2505_06641_b200 import api
+    o = api.sp_default_options()
+    assert o == dict(trace_mode=0, timing=0, guard_utility=2e-5, guard_priority=2e-6)
+    lib.sp_default_options(None)
+
+
 def test_null_context_is_rejected(lib):
     assert lib.sp_reset(None) == 1 and lib.sp_check(None) == 1
     assert lib.sp_last_error(None) == b"null context"

@@ -120,7 +120,7 @@ def test_ragged_models_per_app_pad_with_zero():
     assert s.v[0] == 1.0 and abs(s.v[1] - (1 + 0.0625)) < 1e-6
 
 
-# ------------------------------------------------------------------ penalties of Section 5.1 (reading: the design doc R12/R13)
+# ------------------------------------------------------------------ penalties of Section 5.1 (read as a penalty that grows over the relative deadline)
 @pytest.mark.parametrize("kind", [1, 2])
 def test_soft_penalties_anchor_points_and_monotonicity(kind):
     """gamma is 0 up to the deadline, 1/2 when late by half the relative deadline, 1 from a whole relative deadline
@@ -139,16 +139,26 @@ def test_soft_penalties_anchor_points_and_monotonicity(kind):
         assert g[250] + g[750] == pytest.approx(1.0, abs=1e-15) and g[250] < 0.25
 
 
-def test_sigmoid_penalty_reaches_one_in_fp64_just_before_the_whole_relative_deadline():
+def test_sigmoid_penalty_rounds_to_one_in_fp64_just_before_the_whole_relative_deadline():
     """1 / (1 + ((1 - x) / x)^3) rounds to 1.0 once ((1 - x) / x)^3 drops below half an ulp of 1, i.e. from
-    x = 1 - 4.8e-6 on; the linear penalty stays below 1 until x = 1.  The purge rule (gamma >= 1) therefore retires a
-    sigmoid request that is late by all but a few millionths of its relative deadline."""
+    x = 1 - 4.8e-6 on; the linear penalty stays below 1 until x = 1.  Hopeless is x >= 1 on the integer times, so a
+    sigmoid request that is late by all but a few millionths of its relative deadline stays in its queue and, served
+    then, earns exactly nothing; one that is late by the whole relative deadline is retired."""
     from oracle import oracle
+    from helpers import manual_workload
     arrival, d = 0, 1_000_000_000                         # relative deadline 1 s
     for late_ns, expect_one in ((999_990_000, False), (999_996_000, True), (999_999_999, True)):
         g = oracle.penalty(2, d, arrival, d + late_ns)
         assert (g == 1.0) == expect_one and g <= 1.0
         assert oracle.penalty(1, d, arrival, d + late_ns) < 1.0
+    # request 0: deadline 0.9 s, request 1: deadline 1 s; the only candidate completes 1.999996 s after the arrivals
+    w = manual_workload([[0.5, 0.5]] * 2, [[0.8, 0.8]], app=[0, 0], deadline_ms=[900, 1000], alpha_ms=[1], beta_ms=[1],
+                        swap_ms=[0], batch_sizes=[1], models_per_app=[1], t0_ms=1997.996)
+    w.penalty_kind[:] = 2
+    s = oracle.score(w)
+    dr = oracle.drain(w, s.acc, s.v)
+    assert list(dr.reqs["status"]) == [oracle.EXPIRED, oracle.SCHEDULED]
+    assert dr.n_rounds[0] == 1 and dr.rounds[0, 0]["utility"] == 0.0 and dr.rounds[0, 0]["n_expired"] == 1
 
 
 def test_step_penalty_and_degenerate_relative_deadline():

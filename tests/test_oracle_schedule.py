@@ -124,35 +124,15 @@ def test_expired_requests_were_hopeless():
         assert w.deadline_ns[i] < best
 
 
-# ------------------------------------------------------------------ Algorithm 1, literal
-
-def _algorithm1_literal(w, acc, v):
-    """Group-level scheduling as printed: groups sorted once by mean priority, one model per group chosen by
-    summed member utility at the time the group starts, members ordered inside the group."""
-    t, loaded, order = int(w.t0_ns[0]), -1, 1
-    groups = {}
-    for i in range(w.n_requests):
-        groups.setdefault(int(w.app[i]), []).append(i)
-    prio = {a: np.mean([v[i] * math.exp(-(int(w.deadline_ns[i]) - t) * 1e-9 / w.prio_time_scale_s) for i in g])
-            for a, g in groups.items()}
-    out = {}
-    for a in sorted(groups, key=lambda a: (-prio[a], a)):
-        members = sorted(groups[a], key=lambda i: (int(w.deadline_ns[i]), i))
-        best = None
-        for j in range(int(w.models_per_app[a])):
-            g = first_model(w, a) + j
-            e = t + (int(w.swap_ns[0, g]) if g != loaded else 0) + int(w.lat_alpha_ns[0, g]) + int(w.lat_beta_ns[0, g]) * len(members)
-            u = sum(acc[i, j] for i in members if not (w.deadline_ns[i] < e))
-            if best is None or u > best[0]:
-                best = (u, g, e)
-        for i in members:
-            out[i] = (best[1], order); order += 1
-        t, loaded = best[2], best[1]
-    return out
-
+# ------------------------------------------------------------------ Algorithm 1 when every group fits one batch
 
 @pytest.mark.parametrize("seed", range(6))
-def test_reduces_to_algorithm1_when_groups_fit_one_batch(seed):
+def test_one_batch_groups_are_served_by_eq14_order_with_eq13_models(seed):
+    """With one allowed batch size that holds any group and nothing to retire, every application is served whole in
+    one round.  The emitted schedule must then have the properties Algorithm 1's greedy branch is defined by: groups
+    go in descending Eq. 14 priority (a common clock shift rescales all priorities alike, so the order at the
+    starting clock is the order throughout), and each group runs on the model that maximises its members' summed
+    Eq. 2 utility at the moment the group starts (Eq. 13 on the group; ties to the lowest model)."""
     rng = np.random.default_rng(100 + seed)
     n, a, m, c = 18, 3, 3, 4
     probs = rng.dirichlet(np.ones(c), size=n)
@@ -162,9 +142,31 @@ def test_reduces_to_algorithm1_when_groups_fit_one_batch(seed):
                         batch_sizes=[64], models_per_app=[m] * a)
     s, d = _run(w)
     assert np.all(d.reqs["status"] == oracle.SCHEDULED)
-    lit = _algorithm1_literal(w, s.acc, s.v)
-    for i in range(n):
-        assert (int(d.reqs["model"][i]), int(d.reqs["order"][i])) == lit[i]
+    apps_present = sorted(set(int(x) for x in w.app))
+    nr = int(d.n_rounds[0])
+    rounds = d.rounds[0, :nr]
+    assert sorted(int(x) for x in rounds["app"]) == apps_present           # one round per group
+    t0 = int(w.t0_ns[0])
+    prio = {g: float(np.mean([s.v[i] * math.exp(-(int(w.deadline_ns[i]) - t0) * 1e-9 / w.prio_time_scale_s)
+                              for i in range(n) if w.app[i] == g])) for g in apps_present}
+    assert [int(x) for x in rounds["app"]] == sorted(apps_present, key=lambda g: (-prio[g], g))
+    prev = -1
+    for r in rounds:
+        g_app = int(r["app"])
+        members = [i for i in range(n) if w.app[i] == g_app]
+        assert r["n_members"] == len(members)
+        utils = []
+        for j in range(m):
+            g = first_model(w, g_app) + j
+            e = int(r["t_start_ns"]) + (int(w.swap_ns[0, g]) if g != prev else 0) + int(w.lat_alpha_ns[0, g]) \
+                + int(w.lat_beta_ns[0, g]) * len(members)
+            utils.append(sum(s.acc[i, j] for i in members if not (w.deadline_ns[i] < e)))
+        assert int(r["model"]) - first_model(w, g_app) == int(np.argmax(utils))
+        assert r["utility"] == pytest.approx(max(utils), rel=1e-12)
+        by_key = sorted(members, key=lambda i: (int(w.deadline_ns[i]), i))
+        orders = [int(d.reqs["order"][i]) for i in by_key]
+        assert orders == list(range(orders[0], orders[0] + len(members)))
+        prev = int(r["model"])
 
 
 # ------------------------------------------------------------------ brute force on tiny queues
