@@ -142,17 +142,24 @@ sp_status sp_set_clock(sp_ctx *ctx, int32_t instance, int64_t t_ns, int32_t load
 sp_status sp_set_clocks(sp_ctx *ctx, const int64_t *t_ns, const int32_t *loaded_model);
 
 /*
- * Scores n requests (Section 4.1 and Eq. 9, Eq. 12's variance factor) and makes them the context's request
- * table with ids 0..n-1 (a second call without sp_reset() in between fails with SP_ESTATE).
- * All pointers are DEVICE pointers and are BORROWED until sp_reset(), sp_load_profiles() or sp_destroy():
- * the scheduler reads deadlines and, for near-ties, the raw features again.
+ * Scores n requests (Section 4.1 and Eq. 9, Eq. 12's variance factor) and adds them to the context's request table.
+ * The first call after sp_reset() / sp_load_profiles() starts a table with ids 0..n-1.  A further call APPENDS: the new
+ * requests get the ids that follow (Section 3.2: requests are enqueued while the scheduler runs), earlier results and
+ * the scheduler's state stay, and the next sp_schedule_round() sees the new requests (snapshot mode: at once; trace
+ * mode: from their arrival time on, which must not precede the arrival of the last request already in the table).
+ * Appending is for single-instance contexts (n_instances == 1; otherwise SP_ESTATE), at most 4,096 calls per table.
+ * All pointers are DEVICE pointers and are BORROWED until sp_reset(), sp_load_profiles() or sp_destroy(): the
+ * scheduler reads deadlines and, for near-ties, the raw features again.  (From the first append on the context keeps
+ * its own copy of app / arrival_ns / deadline_ns, 20 bytes per request; the feature matrices stay the caller's.)
  *   feats       [n][D] row-major, float or bf16 as in the profiles; 16-byte aligned
  *   app         [n] application of each request, 0..A-1
  *   arrival_ns  [n]; deadline_ns [n]
  *   instance    [n] instance of each request, non-decreasing; NULL when I == 1.  In trace mode arrivals
  *               must be non-decreasing inside an instance.
- *   acc_out     [n][Mmax] float, optional (NULL): receives the data-aware accuracies, columns >= M_app are 0.
- * Violations found on the device (bad app/instance, order) surface as SP_EINVAL from sp_check().
+ *   acc_out     [n][Mmax] float, optional (NULL): receives the data-aware accuracies of THESE n requests, columns
+ *               >= M_app are 0.
+ * Violations found on the device (bad app/instance, order) surface as SP_EINVAL from sp_check(); the table is then
+ * unusable until sp_reset().
  */
 sp_status sp_score(sp_ctx *ctx, int64_t n, const void *feats, const int32_t *app, const int64_t *arrival_ns,
                    const int64_t *deadline_ns, const int32_t *instance, float *acc_out);

@@ -21,6 +21,7 @@ using namespace sp;
 namespace {
 
 constexpr double kDefaultGuardUtility = 2e-5, kDefaultGuardPriority = 2e-6;
+constexpr size_t kMaxSegments = 4096;   // sp_score calls that may build one request table
 
 struct Buf {                     // a device allocation that only grows
     void *p = nullptr;
@@ -61,6 +62,12 @@ struct sp_ctx {
     Buf state, zbuf, flags, stats, cnt, gstart, cursor, small_start, tiled_start, small_tiles, scan_partial, wt_image, gemm_tiles, gemm_counter;
     // per-request buffers
     Buf acc32, v32, acc64, v64, exact, recs, perm, q_id0, q_id1, q_dl0, q_dl1, q_pw0, q_pw1, sort_scratch;
+    // requests appended to a scored table: the context's own copies of application / arrival / deadline, the list of
+    // the calls' feature matrices, grouping scratch of an append, temporaries of the queue relocation
+    bool own_requests = false;
+    std::vector<FeatSeg> segs;
+    std::vector<Buf> seg_copies;
+    Buf t_app, t_arrival, t_deadline, a_cnt, a_cursor, a_gstart, r_id, r_dl, r_pw;
     // staging of sp_run_host
     Buf h_feats, h_app, h_arrival, h_deadline, h_instance, h_t0, h_loaded, h_rounds, h_ndone;
 };
@@ -93,16 +100,44 @@ sp_status ensure(sp_ctx *c, Buf &b, size_t bytes) {
     return SP_OK;
 }
 
+// Like ensure(), but the first keep_bytes of the old allocation survive; capacity grows geometrically.
+sp_status grow(sp_ctx *c, Buf &b, size_t keep_bytes, size_t bytes) {
+    if (bytes <= b.bytes && b.p) return SP_OK;
+    if (keep_bytes == 0 || !b.p) return ensure(c, b, bytes > 2 * b.bytes ? bytes : 2 * b.bytes);
+    const size_t cap = bytes > 2 * b.bytes ? bytes : 2 * b.bytes;
+    void *np = nullptr;
+    SP_CUDA(c, cudaMalloc(&np, cap));
+    cudaError_t e = cudaMemcpyAsync(np, b.p, keep_bytes, cudaMemcpyDeviceToDevice, c->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+    if (e != cudaSuccess) { cudaFree(np); return fail(c, SP_ECUDA, std::string("grow: ") + cudaGetErrorString(e)); }
+    cudaFree(b.p);
+    b.p = np; b.bytes = cap;
+    return SP_OK;
+}
+
 void release(Buf &b) {
     if (b.p) cudaFree(b.p);
     b.p = nullptr; b.bytes = 0;
 }
+
+// Forgets the request table (host side): the buffers stay allocated for the next one.
+void drop_table(sp_ctx *c);
 
 #define SP_TRY(expr)                       \
     do {                                   \
         sp_status s_ = (expr);             \
         if (s_ != SP_OK) return s_;        \
     } while (0)
+
+void drop_table(sp_ctx *c) {
+    c->have_table = false;
+    c->sched_started = false;
+    c->own_requests = false;
+    c->tb.n = 0;
+    c->segs.clear();
+    for (Buf &b : c->seg_copies) release(b);     // cudaFree waits for kernels that may still read them
+    c->seg_copies.clear();
+}
 
 sp_status upload(sp_ctx *c, Buf &b, const void *host, size_t bytes) {
     SP_TRY(ensure(c, b, bytes));
@@ -176,10 +211,10 @@ double drain_events(std::vector<cudaEvent_t> &list, int64_t *calls) {
 int small_ct_for(int C) { return C <= 10 ? 5 : C <= 20 ? 10 : C <= 32 ? 16 : C <= 64 ? 32 : 0; }
 
 template <int CT>
-sp_status launch_small(sp_ctx *c, int grid, float *acc_out) {
+sp_status launch_small(sp_ctx *c, const DevTable &tv, int grid, float *acc_out) {
     auto kern = k_score_small<CT>;
     SP_CUDA(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->small_smem));
-    kern<<<grid, kSmallThreads, c->small_smem, c->stream>>>(c->P, c->tb, (const int4 *)c->small_tiles.p, acc_out);
+    kern<<<grid, kSmallThreads, c->small_smem, c->stream>>>(c->P, tv, (const int4 *)c->small_tiles.p, acc_out);
     return launched(c, "k_score_small");
 }
 
@@ -244,6 +279,131 @@ sp_status launch_mma(sp_ctx *c, const CUtensorMap &map, const mma::Params &prm) 
     return prm.P.prior ? launch_mma_p<CT, true>(c, map, prm) : launch_mma_p<CT, false>(c, map, prm);
 }
 
+
+// Launches the scoring kernel the loaded profiles select over the rows of `tv` (a table of its own: rows 0..tv.n-1,
+// grouping counts and prefix already in tv.cnt / tv.gstart).
+sp_status score_rows(sp_ctx *c, const DevTable &tv, float *acc_out) {
+    const DevProfiles &P = c->P;
+    const int64_t n = tv.n;
+    const size_t nkeys = (size_t)P.I * P.A;
+    const unsigned gb = (unsigned)((n + 255) / 256);
+    int grid = 0;
+    if (c->small_ct || c->mma_ct) {
+        if (n / kSmallRows + P.I > 0x7fffffff / 2) return fail(c, SP_EINVAL, "too many requests for one call");
+        grid = (int)(n / kSmallRows + P.I);
+        SP_TRY(ensure(c, c->small_tiles, (size_t)grid * sizeof(int4)));
+        k_small_tiles<<<(grid + 255) / 256, 256, 0, c->stream>>>(P, tv, (const int32_t *)c->small_start.p, grid,
+                                                                 (int4 *)c->small_tiles.p, (const int *)c->flags.p);
+        SP_TRY(launched(c, "k_small_tiles"));
+    }
+    int n_tiles = 0;
+    if (c->gemm_on) {
+        k_group_scatter<<<gb, 256, 0, c->stream>>>(P, tv, (const int *)c->flags.p);
+        SP_TRY(launched(c, "k_group_scatter"));
+        if (n / gemm::kGRows + (int64_t)nkeys > 0x3fffffff) return fail(c, SP_EINVAL, "too many requests for one call");
+        n_tiles = (int)(n / gemm::kGRows + (int64_t)nkeys);
+        SP_TRY(ensure(c, c->gemm_tiles, (size_t)n_tiles * sizeof(int4)));
+        SP_TRY(ensure(c, c->gemm_counter, 16));
+        SP_CUDA(c, cudaMemsetAsync(c->gemm_tiles.p, 0xFF, (size_t)n_tiles * sizeof(int4), c->stream));
+        SP_CUDA(c, cudaMemsetAsync(c->gemm_counter.p, 0, 16, c->stream));
+        gemm::k_gemm_tiles<<<(unsigned)((nkeys + 255) / 256), 256, 0, c->stream>>>((int)nkeys, tv.cnt, tv.gstart, (int4 *)c->gemm_tiles.p,
+                                                                                (int *)c->gemm_counter.p, (const int *)c->flags.p);
+        SP_TRY(launched(c, "k_gemm_tiles"));
+    }
+    CUtensorMap x_map;
+    if (c->mma_ct) SP_TRY(feature_map(c, &x_map, tv.feats, n, P.D));
+    SP_TRY(mark(c, c->ev_score));
+    if (c->mma_ct) {
+        mma::Params prm{P, tv, (const int4 *)c->small_tiles.p, grid, acc_out, (int *)c->flags.p};
+        switch (c->mma_ct) {
+            case 8: SP_TRY(launch_mma<8>(c, x_map, prm)); break;
+            case 16: SP_TRY(launch_mma<16>(c, x_map, prm)); break;
+            case 24: SP_TRY(launch_mma<24>(c, x_map, prm)); break;
+            case 32: SP_TRY(launch_mma<32>(c, x_map, prm)); break;
+            case 48: SP_TRY(launch_mma<48>(c, x_map, prm)); break;
+            default: SP_TRY(launch_mma<64>(c, x_map, prm)); break;
+        }
+    } else if (c->small_ct) {
+        switch (c->small_ct) {
+            case 5: SP_TRY(launch_small<5>(c, tv, grid, acc_out)); break;
+            case 10: SP_TRY(launch_small<10>(c, tv, grid, acc_out)); break;
+            case 16: SP_TRY(launch_small<16>(c, tv, grid, acc_out)); break;
+            default: SP_TRY(launch_small<32>(c, tv, grid, acc_out)); break;
+        }
+    } else if (c->gemm_on) {
+        gemm::GParams gp{P, tv, (const int4 *)c->gemm_tiles.p, n_tiles, c->gemm_cp, P.I * P.A * c->gemm_cp, acc_out, (int *)c->flags.p};
+        const int ggrid = n_tiles < c->n_sms ? n_tiles : c->n_sms;
+        if (c->gemm_f32) {
+            SP_CUDA(c, cudaFuncSetAttribute(gemm::k_score_gemm<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::GCfg<true>::bytes));
+            gemm::k_score_gemm<true><<<ggrid, gemm::GCfg<true>::Threads, gemm::GCfg<true>::bytes, c->stream>>>(c->wt_map, c->r_map, c->b_map, gp);
+        } else {
+            SP_CUDA(c, cudaFuncSetAttribute(gemm::k_score_gemm<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::GCfg<false>::bytes));
+            gemm::k_score_gemm<false><<<ggrid, gemm::GCfg<false>::Threads, gemm::GCfg<false>::bytes, c->stream>>>(c->wt_map, c->r_map, c->b_map, gp);
+        }
+        SP_TRY(launched(c, "k_score_gemm"));
+    } else {
+        k_group_scatter<<<gb, 256, 0, c->stream>>>(P, tv, (const int *)c->flags.p);
+        SP_TRY(launched(c, "k_group_scatter"));
+        grid = (int)(n / kTiledRows + (int64_t)nkeys);
+        if (P.dtype == SP_BF16)
+            k_score_tiled<true><<<grid, kTiledThreads, 0, c->stream>>>(P, tv, (const int32_t *)c->tiled_start.p, acc_out,
+                                                                    (const int *)c->flags.p);
+        else
+            k_score_tiled<false><<<grid, kTiledThreads, 0, c->stream>>>(P, tv, (const int32_t *)c->tiled_start.p, acc_out,
+                                                                     (const int *)c->flags.p);
+        SP_TRY(launched(c, "k_score_tiled"));
+    }
+    return mark(c, c->ev_score);
+}
+
+// Appending requests changes the size of every application's queue region (regions are laid out back to back, sized by
+// the number of requests of the application scored so far).  One block: the live part of every queue is copied out
+// (phase 1) and back in at the start of its new region in queue copy 0 (phase 2); heads, tails and region starts follow.
+__global__ void __launch_bounds__(1024)
+k_queue_regrow(InstState *state, int A, int64_t *qstart, const int32_t *add_cnt, int64_t *q_id0, int64_t *q_id1,
+               int64_t *q_dl0, int64_t *q_dl1, double *q_pw0, double *q_pw1, int64_t *t_id, int64_t *t_dl, double *t_pw,
+               const int *flags) {
+    __shared__ int64_t s_old[kMaxApps + 1], s_new[kMaxApps + 1], s_live[kMaxApps + 1];
+    __shared__ int s_head[kMaxApps], s_cur[kMaxApps];
+    if (flags[1]) return;                    // the appended rows were rejected: the table is unusable until sp_reset
+    const int tid = threadIdx.x, NT = blockDim.x;
+    if (tid == 0) {
+        s_new[0] = 0; s_live[0] = 0;
+        for (int a = 0; a < A; ++a) {
+            s_old[a] = qstart[a];
+            s_new[a + 1] = s_new[a] + (qstart[a + 1] - qstart[a]) + add_cnt[a];
+            s_live[a + 1] = s_live[a] + (state->tail[a] - state->head[a]);
+            s_head[a] = state->head[a]; s_cur[a] = state->cur[a];
+        }
+    }
+    __syncthreads();
+    const int64_t total = s_live[A];
+    for (int64_t f = tid; f < total; f += NT) {
+        int a = 0;
+        while (f >= s_live[a + 1]) ++a;
+        const int64_t src = s_old[a] + s_head[a] + (f - s_live[a]);
+        t_id[f] = (s_cur[a] ? q_id1 : q_id0)[src];
+        t_dl[f] = (s_cur[a] ? q_dl1 : q_dl0)[src];
+        t_pw[f] = (s_cur[a] ? q_pw1 : q_pw0)[src];
+    }
+    __threadfence_block();
+    __syncthreads();
+    for (int64_t f = tid; f < total; f += NT) {
+        int a = 0;
+        while (f >= s_live[a + 1]) ++a;
+        const int64_t dst = s_new[a] + (f - s_live[a]);
+        q_id0[dst] = t_id[f]; q_dl0[dst] = t_dl[f]; q_pw0[dst] = t_pw[f];
+    }
+    __syncthreads();
+    if (tid == 0) {
+        for (int a = 0; a < A; ++a) {
+            state->tail[a] = (int32_t)(s_live[a + 1] - s_live[a]); state->head[a] = 0; state->cur[a] = 0;
+            qstart[a] = s_new[a];
+        }
+        qstart[A] = s_new[A];
+    }
+}
+
 }  // namespace
 
 // =================================================================================================
@@ -282,8 +442,10 @@ void sp_destroy(sp_ctx *c) {
                   &c->small_start, &c->tiled_start, &c->small_tiles, &c->scan_partial, &c->wt_image, &c->gemm_tiles, &c->gemm_counter, &c->acc32, &c->v32, &c->acc64, &c->v64, &c->exact, &c->recs,
                   &c->perm, &c->q_id0, &c->q_id1, &c->q_dl0, &c->q_dl1, &c->q_pw0, &c->q_pw1, &c->sort_scratch,
                   &c->h_feats, &c->h_app, &c->h_arrival, &c->h_deadline, &c->h_instance, &c->h_t0, &c->h_loaded,
-                  &c->h_rounds, &c->h_ndone};
+                  &c->h_rounds, &c->h_ndone, &c->t_app, &c->t_arrival, &c->t_deadline, &c->a_cnt, &c->a_cursor,
+                  &c->a_gstart, &c->r_id, &c->r_dl, &c->r_pw};
     for (Buf *b : all) release(*b);
+    for (Buf &b : c->seg_copies) release(b);
     delete c;
 }
 
@@ -340,7 +502,7 @@ sp_status sp_load_profiles(sp_ctx *c, const sp_profiles *p) {
     if (ss.end > 96 * 1024) return fail(c, SP_EINVAL, "models_per_app x largest batch size is too large for one block");
 
     c->have_profiles = false;
-    c->have_table = false;
+    drop_table(c);
     c->hp.models_per_app.assign(p->models_per_app, p->models_per_app + A);
     c->hp.batch_sizes.assign(p->batch_sizes, p->batch_sizes + nB);
     const size_t esz = p->feat_dtype == SP_BF16 ? 2 : 4;
@@ -506,9 +668,7 @@ sp_status sp_reset(sp_ctx *c) {
     SP_TRY(launched(c, "k_state_reset"));
     SP_CUDA(c, cudaMemsetAsync((int *)c->flags.p + 1, 0, sizeof(int), c->stream));
     SP_CUDA(c, cudaMemsetAsync(c->stats.p, 0, 4 * sizeof(unsigned long long), c->stream));
-    c->have_table = false;
-    c->sched_started = false;
-    c->tb.n = 0;
+    drop_table(c);
     return SP_OK;
 }
 
@@ -516,127 +676,120 @@ sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, 
                    const int64_t *deadline_ns, const int32_t *instance, float *acc_out) {
     if (!c) return SP_EINVAL;
     if (!c->have_profiles) return fail(c, SP_ESTATE, "no profiles loaded");
-    if (c->have_table) return fail(c, SP_ESTATE, "requests already scored; call sp_reset first");
+    const bool append = c->have_table;
+    if (append && c->P.I != 1)
+        return fail(c, SP_ESTATE, "requests can be appended to a single-instance context only; call sp_reset first");
     if (n < 0 || n > ((int64_t)1 << 40)) return fail(c, SP_EINVAL, "n out of range");
     if (n > 0 && (!feats || !app || !arrival_ns || !deadline_ns)) return fail(c, SP_EINVAL, "a request array is NULL");
     if (c->P.I > 1 && n > 0 && !instance) return fail(c, SP_EINVAL, "instance is required when n_instances > 1");
     if (((uintptr_t)feats & 15) != 0) return fail(c, SP_EINVAL, "feats must be 16-byte aligned");
+    if (append && n == 0) return SP_OK;
     SP_CUDA(c, cudaSetDevice(c->device));
     const DevProfiles &P = c->P;
-    const size_t nn = (size_t)(n > 0 ? n : 1), nkeys = (size_t)P.I * P.A;
-    SP_TRY(ensure(c, c->acc32, nn * P.Mmax * 4));
-    SP_TRY(ensure(c, c->v32, nn * 4));
-    SP_TRY(ensure(c, c->acc64, nn * P.Mmax * 8));
-    SP_TRY(ensure(c, c->v64, nn * 8));
-    SP_TRY(ensure(c, c->exact, nn));
-    SP_TRY(ensure(c, c->recs, nn * sizeof(sp_req_rec)));
-    SP_TRY(ensure(c, c->perm, nn * 8));
-    SP_TRY(ensure(c, c->q_id0, nn * 8));
-    SP_TRY(ensure(c, c->q_id1, nn * 8));
-    SP_TRY(ensure(c, c->q_dl0, nn * 8));
-    SP_TRY(ensure(c, c->q_dl1, nn * 8));
-    SP_TRY(ensure(c, c->q_pw0, nn * 8));
-    SP_TRY(ensure(c, c->q_pw1, nn * 8));
-    SP_TRY(ensure(c, c->sort_scratch, nn * sizeof(SortKey)));
+    const int64_t n_old = append ? c->tb.n : 0, n_tot = n_old + n;
+    if (append && c->segs.size() >= kMaxSegments)
+        return fail(c, SP_ESTATE, "too many sp_score calls on one table (4096); call sp_reset and score the pending requests again");
+    const size_t nn = (size_t)(n_tot > 0 ? n_tot : 1), nkeys = (size_t)P.I * P.A;
+    // per-request buffers of the context: rows 0..n_old-1 are kept when requests are appended
+    struct { Buf *b; size_t row_bytes; bool keep; } per_row[] = {
+        {&c->acc32, (size_t)P.Mmax * 4, true}, {&c->v32, 4, true}, {&c->acc64, (size_t)P.Mmax * 8, true}, {&c->v64, 8, true},
+        {&c->exact, 1, true}, {&c->recs, sizeof(sp_req_rec), true}, {&c->perm, 8, false},
+        {&c->q_id0, 8, true}, {&c->q_id1, 8, true}, {&c->q_dl0, 8, true}, {&c->q_dl1, 8, true},
+        {&c->q_pw0, 8, true}, {&c->q_pw1, 8, true}, {&c->sort_scratch, sizeof(SortKey), false}};
+    for (auto &e : per_row) {
+        if (append && e.keep) SP_TRY(grow(c, *e.b, (size_t)n_old * e.row_bytes, nn * e.row_bytes));
+        else SP_TRY(ensure(c, *e.b, nn * e.row_bytes));
+    }
     DevTable &tb = c->tb;
-    tb.n = n; tb.feats = feats; tb.app = app; tb.arrival = arrival_ns; tb.deadline = deadline_ns;
-    tb.instance = P.I > 1 ? instance : nullptr;
+    if (append) {
+        // The scheduler reads application, arrival and deadline by request id, and a table made by several calls has
+        // them in several caller arrays: from the first append on the context keeps its own copies (20 bytes per
+        // request), and the feature matrices of the calls are found through a segment list.
+        const bool migrate = !c->own_requests;
+        SP_TRY(grow(c, c->t_app, migrate ? 0 : (size_t)n_old * 4, nn * 4));
+        SP_TRY(grow(c, c->t_arrival, migrate ? 0 : (size_t)n_old * 8, nn * 8));
+        SP_TRY(grow(c, c->t_deadline, migrate ? 0 : (size_t)n_old * 8, nn * 8));
+        if (migrate) {
+            if (n_old > 0) {
+                SP_CUDA(c, cudaMemcpyAsync(c->t_app.p, tb.app, (size_t)n_old * 4, cudaMemcpyDeviceToDevice, c->stream));
+                SP_CUDA(c, cudaMemcpyAsync(c->t_arrival.p, tb.arrival, (size_t)n_old * 8, cudaMemcpyDeviceToDevice, c->stream));
+                SP_CUDA(c, cudaMemcpyAsync(c->t_deadline.p, tb.deadline, (size_t)n_old * 8, cudaMemcpyDeviceToDevice, c->stream));
+            }
+            c->segs.clear();
+            c->segs.push_back(FeatSeg{0, tb.feats});
+            c->own_requests = true;
+        }
+        SP_CUDA(c, cudaMemcpyAsync((int32_t *)c->t_app.p + n_old, app, (size_t)n * 4, cudaMemcpyDeviceToDevice, c->stream));
+        SP_CUDA(c, cudaMemcpyAsync((int64_t *)c->t_arrival.p + n_old, arrival_ns, (size_t)n * 8, cudaMemcpyDeviceToDevice, c->stream));
+        SP_CUDA(c, cudaMemcpyAsync((int64_t *)c->t_deadline.p + n_old, deadline_ns, (size_t)n * 8, cudaMemcpyDeviceToDevice, c->stream));
+        c->segs.push_back(FeatSeg{n_old, feats});
+        // the list is read by kernels of earlier calls that may still run: a new copy per call, the old ones are
+        // released with the table
+        Buf seg_dev;
+        SP_TRY(ensure(c, seg_dev, c->segs.size() * sizeof(FeatSeg)));
+        c->seg_copies.push_back(seg_dev);
+        SP_CUDA(c, cudaMemcpyAsync(seg_dev.p, c->segs.data(), c->segs.size() * sizeof(FeatSeg), cudaMemcpyHostToDevice, c->stream));
+        SP_CUDA(c, cudaStreamSynchronize(c->stream));      // the host vector may move at the next append
+        tb.feats = nullptr; tb.segs = (const FeatSeg *)seg_dev.p; tb.n_segs = (int)c->segs.size();
+        tb.app = (const int32_t *)c->t_app.p; tb.arrival = (const int64_t *)c->t_arrival.p;
+        tb.deadline = (const int64_t *)c->t_deadline.p;
+        SP_TRY(ensure(c, c->a_cnt, nkeys * 4));
+        SP_TRY(ensure(c, c->a_cursor, nkeys * 4));
+        SP_TRY(ensure(c, c->a_gstart, (nkeys + 1) * 8));
+        SP_TRY(ensure(c, c->r_id, nn * 8));
+        SP_TRY(ensure(c, c->r_dl, nn * 8));
+        SP_TRY(ensure(c, c->r_pw, nn * 8));
+    } else {
+        tb.feats = feats; tb.segs = nullptr; tb.n_segs = 0; tb.app = app; tb.arrival = arrival_ns; tb.deadline = deadline_ns;
+        tb.instance = P.I > 1 ? instance : nullptr;
+    }
+    tb.n = n_tot;
     tb.acc32 = (float *)c->acc32.p; tb.v32 = (float *)c->v32.p; tb.acc64 = (double *)c->acc64.p;
     tb.v64 = (double *)c->v64.p; tb.exact = (unsigned char *)c->exact.p; tb.recs = (sp_req_rec *)c->recs.p;
     tb.cnt = (int32_t *)c->cnt.p; tb.gstart = (int64_t *)c->gstart.p; tb.perm = (int64_t *)c->perm.p;
     tb.cursor = (int32_t *)c->cursor.p;
+    tb.qstart = (const int64_t *)c->gstart.p;
 
-    SP_CUDA(c, cudaMemsetAsync(tb.cnt, 0, nkeys * 4, c->stream));
-    SP_CUDA(c, cudaMemsetAsync(tb.cursor, 0, nkeys * 4, c->stream));
+    // The rows this call scores, as a table of their own: results go to rows n_old.. of the context's buffers; the
+    // grouping scratch of an append is separate from the queue regions the scheduler works on.
+    DevTable tv = tb;
+    tv.n = n; tv.feats = feats; tv.segs = nullptr; tv.n_segs = 0; tv.app = app; tv.arrival = arrival_ns; tv.deadline = deadline_ns;
+    tv.acc32 = tb.acc32 + n_old * P.Mmax; tv.v32 = tb.v32 + n_old; tv.exact = tb.exact + n_old; tv.recs = tb.recs + n_old;
+    if (append) { tv.cnt = (int32_t *)c->a_cnt.p; tv.cursor = (int32_t *)c->a_cursor.p; tv.gstart = (int64_t *)c->a_gstart.p; }
+
+    SP_CUDA(c, cudaMemsetAsync(tv.cnt, 0, nkeys * 4, c->stream));
+    SP_CUDA(c, cudaMemsetAsync(tv.cursor, 0, nkeys * 4, c->stream));
     const unsigned gb = (unsigned)((n + 255) / 256);
     if (n > 0) {
-        k_group_count<<<gb, 256, 0, c->stream>>>(P, tb, c->opt.trace_mode, (int *)c->flags.p);
+        k_group_count<<<gb, 256, 0, c->stream>>>(P, tv, c->opt.trace_mode, (int *)c->flags.p,
+                                                 append && n_old > 0 ? (const int64_t *)c->t_arrival.p + (n_old - 1) : nullptr);
         SP_TRY(launched(c, "k_group_count"));
     }
     if (nkeys <= 4 * (size_t)kScanChunk) {
-        k_group_scan<<<1, 1024, 0, c->stream>>>((int)nkeys, P.A, tb.cnt, tb.gstart, (int32_t *)c->tiled_start.p,
+        k_group_scan<<<1, 1024, 0, c->stream>>>((int)nkeys, P.A, tv.cnt, tv.gstart, (int32_t *)c->tiled_start.p,
                                                 (int32_t *)c->small_start.p);
         SP_TRY(launched(c, "k_group_scan"));
     } else {                                           // many keys: per-block totals, then one scan block per chunk
         const int nblk = (int)(nkeys / kScanChunk + 1);    // covers index nkeys (the grand total) as well
         SP_TRY(ensure(c, c->scan_partial, (size_t)3 * nblk * sizeof(long long)));
-        k_group_partials<<<nblk, kScanChunk, 0, c->stream>>>((int)nkeys, P.A, tb.cnt, (long long *)c->scan_partial.p);
+        k_group_partials<<<nblk, kScanChunk, 0, c->stream>>>((int)nkeys, P.A, tv.cnt, (long long *)c->scan_partial.p);
         SP_TRY(launched(c, "k_group_partials"));
-        k_group_scan_blocks<<<nblk, kScanChunk, 0, c->stream>>>((int)nkeys, P.A, tb.cnt, (const long long *)c->scan_partial.p,
-                                                              tb.gstart, (int32_t *)c->tiled_start.p, (int32_t *)c->small_start.p);
+        k_group_scan_blocks<<<nblk, kScanChunk, 0, c->stream>>>((int)nkeys, P.A, tv.cnt, (const long long *)c->scan_partial.p,
+                                                              tv.gstart, (int32_t *)c->tiled_start.p, (int32_t *)c->small_start.p);
         SP_TRY(launched(c, "k_group_scan_blocks"));
     }
-    if (n > 0) {
-        int grid = 0;
-        if (c->small_ct || c->mma_ct) {
-            if (n / kSmallRows + P.I > 0x7fffffff / 2) return fail(c, SP_EINVAL, "too many requests for one call");
-            grid = (int)(n / kSmallRows + P.I);
-            SP_TRY(ensure(c, c->small_tiles, (size_t)grid * sizeof(int4)));
-            k_small_tiles<<<(grid + 255) / 256, 256, 0, c->stream>>>(P, tb, (const int32_t *)c->small_start.p, grid,
-                                                                     (int4 *)c->small_tiles.p, (const int *)c->flags.p);
-            SP_TRY(launched(c, "k_small_tiles"));
-        }
-        int n_tiles = 0;
-        if (c->gemm_on) {
-            k_group_scatter<<<gb, 256, 0, c->stream>>>(P, tb, (const int *)c->flags.p);
-            SP_TRY(launched(c, "k_group_scatter"));
-            if (n / gemm::kGRows + (int64_t)nkeys > 0x3fffffff) return fail(c, SP_EINVAL, "too many requests for one call");
-            n_tiles = (int)(n / gemm::kGRows + (int64_t)nkeys);
-            SP_TRY(ensure(c, c->gemm_tiles, (size_t)n_tiles * sizeof(int4)));
-            SP_TRY(ensure(c, c->gemm_counter, 16));
-            SP_CUDA(c, cudaMemsetAsync(c->gemm_tiles.p, 0xFF, (size_t)n_tiles * sizeof(int4), c->stream));
-            SP_CUDA(c, cudaMemsetAsync(c->gemm_counter.p, 0, 16, c->stream));
-            gemm::k_gemm_tiles<<<(unsigned)((nkeys + 255) / 256), 256, 0, c->stream>>>((int)nkeys, tb.cnt, tb.gstart, (int4 *)c->gemm_tiles.p,
-                                                                                    (int *)c->gemm_counter.p, (const int *)c->flags.p);
-            SP_TRY(launched(c, "k_gemm_tiles"));
-        }
-        CUtensorMap x_map;
-        if (c->mma_ct) SP_TRY(feature_map(c, &x_map, feats, n, P.D));
-        SP_TRY(mark(c, c->ev_score));
-        if (c->mma_ct) {
-            mma::Params prm{P, tb, (const int4 *)c->small_tiles.p, grid, acc_out, (int *)c->flags.p};
-            switch (c->mma_ct) {
-                case 8: SP_TRY(launch_mma<8>(c, x_map, prm)); break;
-                case 16: SP_TRY(launch_mma<16>(c, x_map, prm)); break;
-                case 24: SP_TRY(launch_mma<24>(c, x_map, prm)); break;
-                case 32: SP_TRY(launch_mma<32>(c, x_map, prm)); break;
-                case 48: SP_TRY(launch_mma<48>(c, x_map, prm)); break;
-                default: SP_TRY(launch_mma<64>(c, x_map, prm)); break;
-            }
-        } else if (c->small_ct) {
-            switch (c->small_ct) {
-                case 5: SP_TRY(launch_small<5>(c, grid, acc_out)); break;
-                case 10: SP_TRY(launch_small<10>(c, grid, acc_out)); break;
-                case 16: SP_TRY(launch_small<16>(c, grid, acc_out)); break;
-                default: SP_TRY(launch_small<32>(c, grid, acc_out)); break;
-            }
-        } else if (c->gemm_on) {
-            gemm::GParams gp{P, tb, (const int4 *)c->gemm_tiles.p, n_tiles, c->gemm_cp, P.I * P.A * c->gemm_cp, acc_out, (int *)c->flags.p};
-            const int ggrid = n_tiles < c->n_sms ? n_tiles : c->n_sms;
-            if (c->gemm_f32) {
-                SP_CUDA(c, cudaFuncSetAttribute(gemm::k_score_gemm<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::GCfg<true>::bytes));
-                gemm::k_score_gemm<true><<<ggrid, gemm::kGThreads, gemm::GCfg<true>::bytes, c->stream>>>(c->wt_map, c->r_map, c->b_map, gp);
-            } else {
-                SP_CUDA(c, cudaFuncSetAttribute(gemm::k_score_gemm<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::GCfg<false>::bytes));
-                gemm::k_score_gemm<false><<<ggrid, gemm::kGThreads, gemm::GCfg<false>::bytes, c->stream>>>(c->wt_map, c->r_map, c->b_map, gp);
-            }
-            SP_TRY(launched(c, "k_score_gemm"));
-        } else {
-            k_group_scatter<<<gb, 256, 0, c->stream>>>(P, tb, (const int *)c->flags.p);
-            SP_TRY(launched(c, "k_group_scatter"));
-            grid = (int)(n / kTiledRows + (int64_t)nkeys);
-            if (P.dtype == SP_BF16)
-                k_score_tiled<true><<<grid, kTiledThreads, 0, c->stream>>>(P, tb, (const int32_t *)c->tiled_start.p, acc_out,
-                                                                        (const int *)c->flags.p);
-            else
-                k_score_tiled<false><<<grid, kTiledThreads, 0, c->stream>>>(P, tb, (const int32_t *)c->tiled_start.p, acc_out,
-                                                                         (const int *)c->flags.p);
-            SP_TRY(launched(c, "k_score_tiled"));
-        }
-        SP_TRY(mark(c, c->ev_score));
+    if (n > 0) SP_TRY(score_rows(c, tv, acc_out));
+    if (append) {
+        // make room in every application's queue region for its new requests; live entries move to the new regions
+        k_queue_regrow<<<1, 1024, 0, c->stream>>>((InstState *)c->state.p, P.A, (int64_t *)c->gstart.p, (const int32_t *)c->a_cnt.p,
+                                                  (int64_t *)c->q_id0.p, (int64_t *)c->q_id1.p, (int64_t *)c->q_dl0.p,
+                                                  (int64_t *)c->q_dl1.p, (double *)c->q_pw0.p, (double *)c->q_pw1.p,
+                                                  (int64_t *)c->r_id.p, (int64_t *)c->r_dl.p, (double *)c->r_pw.p,
+                                                  (const int *)c->flags.p);
+        SP_TRY(launched(c, "k_queue_regrow"));
     }
     c->have_table = true;
-    c->sched_started = false;
+    if (!append) c->sched_started = false;
     return SP_OK;
 }
 
@@ -891,7 +1044,7 @@ extern "C" sp_status sp_score_static(int device, void *cuda_stream, const sp_sta
     // the array keeps the previous call's contents: clear the parts that are accumulated into
     SP_STATIC_CUDA(cudaMemsetAsync(s, 0, offsetof(StaticScratch, tiled_start), stream));
     const unsigned gb = (unsigned)((n + 255) / 256);
-    k_group_count<<<gb, 256, 0, stream>>>(P, tb, 0, s->flags);
+    k_group_count<<<gb, 256, 0, stream>>>(P, tb, 0, s->flags, nullptr);
     k_group_scan<<<1, 1024, 0, stream>>>(A, A, s->cnt, s->gstart, s->tiled_start, s->small_start);
     k_group_scatter<<<gb, 256, 0, stream>>>(P, tb, s->flags);
     const int grid = (int)(n / kTiledRows + A);

@@ -12,7 +12,9 @@ constexpr int kSmallRows = 128;   // requests per tile of the small-head scoring
 
 // Validation of the request table, initial request records, requests per (instance, application).
 // flags[0]: device status (DevErr), flags[1]: 1 when the request table failed validation.
-__global__ void k_group_count(DevProfiles P, DevTable tb, int trace_mode, int *flags) {
+// prev_arrival: arrival time of the last request already in the table when these rows are appended to it (nullptr
+// for the first rows of a table); in trace mode the appended rows must not arrive before it.
+__global__ void k_group_count(DevProfiles P, DevTable tb, int trace_mode, int *flags, const int64_t *prev_arrival) {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= tb.n) return;
     if (tb.recs) {                           // the request starts pending, without an fp64 re-scoring (a table
@@ -23,6 +25,7 @@ __global__ void k_group_count(DevProfiles P, DevTable tb, int trace_mode, int *f
     const int a = tb.app[i];
     const int inst = tb.instance ? tb.instance[i] : 0;
     bool bad = a < 0 || a >= P.A || inst < 0 || inst >= P.I;
+    if (!bad && i == 0 && trace_mode && prev_arrival && *prev_arrival > tb.arrival[0]) bad = true;
     if (!bad && i > 0) {
         const int prev = tb.instance ? tb.instance[i - 1] : 0;
         if (prev > inst) bad = true;

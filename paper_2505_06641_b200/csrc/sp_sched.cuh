@@ -128,12 +128,14 @@ __device__ void exact_row(const SchedParams &sp, int inst, int64_t id, double *z
     const int a = sp.tb.app[id];
     const int64_t head = (int64_t)inst * P.A + a;
     const int C = P.C, D = P.D;
+    int64_t frow;
+    const void *fmat = feat_matrix(sp.tb, id, frow);
     for (int c0 = 0; c0 < C; c0 += 32) {
         const int c = c0 + lane;
         double z = c < C ? (double)P.bias[head * C + c] : 0.0;
         if (c < C)
             for (int d = 0; d < D; ++d) {
-                const double x = (double)load_feat(sp.tb.feats, P.dtype, id * D + d);
+                const double x = (double)load_feat(fmat, P.dtype, frow * D + d);
                 const double w = (double)load_feat(P.W, P.dtype, (head * D + d) * C + c);
                 z = __dadd_rn(z, __dmul_rn(x, w));
             }
@@ -322,10 +324,10 @@ __device__ void sched_instance(const SchedParams &sp, const int inst) {
         if (tid == 0 && sp.n_done) sp.n_done[inst] = 0;
         return;
     }
-    const int64_t r0 = tb.gstart[(int64_t)inst * A], r1 = tb.gstart[(int64_t)(inst + 1) * A];
+    const int64_t r0 = tb.qstart[(int64_t)inst * A], r1 = tb.qstart[(int64_t)(inst + 1) * A];
     const int64_t n_inst = r1 - r0;
     if (tid == 0) st = sp.state[inst];
-    if (tid <= A) s_base[tid] = tb.gstart[(int64_t)inst * A + tid];
+    if (tid <= A) s_base[tid] = tb.qstart[(int64_t)inst * A + tid];
     __syncthreads();
 
     const double tau = P.tau;

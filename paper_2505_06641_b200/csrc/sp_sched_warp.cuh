@@ -96,7 +96,7 @@ __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const 
     uint32_t *s_ida = reinterpret_cast<uint32_t *>(mine + L.ida);
     double *pref = reinterpret_cast<double *>(mine + L.pref);
 
-    const int64_t r0 = tb.gstart[(int64_t)inst * A], r1 = tb.gstart[(int64_t)(inst + 1) * A];
+    const int64_t r0 = tb.qstart[(int64_t)inst * A], r1 = tb.qstart[(int64_t)(inst + 1) * A];
     const int n_inst = (int)(r1 - r0);
     InstState *stp = &sp.state[inst];
     if (stp->started) return true;                                    // not a fresh instance: the block resumes it
@@ -346,7 +346,7 @@ __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const 
         for (int a = 0; a < A; ++a) {
             const int h = __shfl_sync(0xffffffffu, head, a), t = __shfl_sync(0xffffffffu, tail, a);
             const int s0 = __shfl_sync(0xffffffffu, seg0, a);
-            const int64_t base = tb.gstart[(int64_t)inst * A + a];
+            const int64_t base = tb.qstart[(int64_t)inst * A + a];
             for (int k = h + lane; k < t; k += 32) {
                 sp.q_id[0][base + (k - s0)] = r0 + (s_ida[k] & 0xFFFFFFu);
                 sp.q_dl[0][base + (k - s0)] = s_dl[k];

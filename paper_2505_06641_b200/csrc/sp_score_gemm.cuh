@@ -40,8 +40,8 @@ using namespace sp::mma;
 constexpr int kGRows = 128;                 // requests per tile = MMA M
 constexpr int kASlabBytes = kGRows * 128;   // 16 KB: 128 rows x 128 bytes
 constexpr int kGBProducerWarp = 0, kGMmaWarp = 1, kGAWarp0 = 2, kGEpiWarp0 = 6;
-constexpr int kGThreads = 32 * 14;
-constexpr int kGAThreads = 128, kGEpiThreads = 256;
+constexpr int kGAThreads = 128;
+constexpr int kGMaxEpiGroups = 4;
 constexpr int kMergeFloats = 2 + kMaxModelsPerApp;    // running max, running sum, running sums per model
 constexpr int kGMaxA = 5, kGMaxB = 3;      // largest A / B ring of the two flavours
 
@@ -63,6 +63,13 @@ __device__ __forceinline__ float sum_f32x2(unsigned long long v) {
 
 template <bool F32>
 struct GCfg {
+    // Epilogue warpgroups (each takes an equal share of the columns of every chunk) and the logit columns a thread
+    // holds in registers at a time.  Measured: the fp32 flavour is 14 % faster with four groups (its chunk has to be
+    // finished while only three operand slabs are in flight), the bf16 flavour 2 % slower than with two.
+    static constexpr int EpiGroups = F32 ? 4 : 2;
+    static constexpr int EpiBlk = F32 ? 16 : 32;
+    static constexpr int EpiThreads = 128 * EpiGroups;
+    static constexpr int Threads = 32 * 6 + EpiThreads;
     static constexpr int NC = F32 ? 208 : 256;                 // logit columns per chunk = MMA N (2 accumulators <= 512 columns)
     static constexpr int KSlab = F32 ? 32 : 64;                // features per slab row (128 bytes)
     static constexpr int KStep = F32 ? 8 : 16;                 // features per MMA
@@ -85,8 +92,8 @@ struct GCfg {
     static constexpr int b_ring = a_ring + AStages * kASlabBytes;             // [BStages] slabs of NC (x 2) rows
     static constexpr int rtab = b_ring + BStages * BSlot;                     // [2][16][NC] floats
     static constexpr int bias = rtab + 2 * RBytes;                            // [2][NC] floats
-    static constexpr int merge = bias + 2 * BiasSlot;                        // [128][kMergeFloats]
-    static constexpr int bars = (merge + kGRows * kMergeFloats * 4 + 15) & ~15;
+    static constexpr int merge = bias + 2 * BiasSlot;                        // [EpiGroups - 1][128][kMergeFloats]
+    static constexpr int bars = (merge + (EpiGroups - 1) * kGRows * kMergeFloats * 4 + 15) & ~15;
     static constexpr int n_bars = 2 * kGMaxA + 2 * kGMaxB + 8 + 3;
     static constexpr int misc = bars + n_bars * 8;
     static constexpr int end = misc + 16;
@@ -193,12 +200,13 @@ __global__ void k_gemm_tiles(int n_keys, const int32_t *__restrict__ cnt, const 
 }
 
 template <bool F32>
-__global__ void __launch_bounds__(kGThreads, 1)
+__global__ void __launch_bounds__(GCfg<F32>::Threads, 1)
 k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__ CUtensorMap r_map,
              const __grid_constant__ CUtensorMap b_map, const GParams prm) {
     using G = GCfg<F32>;
     constexpr int kNC = G::NC, kKSlab = G::KSlab, kAStages = G::AStages, kBStages = G::BStages;
     constexpr int kBSlabBytes = G::BSlabBytes, kRBytes = G::RBytes, kBiasBytes = G::BiasBytes;
+    constexpr int kGEpiGroups = G::EpiGroups, kGEpiBlk = G::EpiBlk, kGEpiThreads = G::EpiThreads;
     using GSmem = G;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw_u32 = smem_u32(smem_raw);
@@ -222,8 +230,8 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
             mbar_init(bar(gbar_acc_full(b)), 1); mbar_init(bar(gbar_acc_empty(b)), kGEpiThreads);
             mbar_init(bar(gbar_r_full(b)), 1); mbar_init(bar(gbar_r_free(b)), kGEpiThreads);
         }
-        mbar_init(bar(kGBarMergeReady), kGEpiThreads / 2);
-        mbar_init(bar(kGBarMergeDone), kGEpiThreads / 2);
+        mbar_init(bar(kGBarMergeReady), kGEpiThreads - 128);
+        mbar_init(bar(kGBarMergeDone), 128);
         mbar_init(bar(kGBarDrain), 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -382,15 +390,18 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
         cp_async_wait<0>();
         while (ok && signalled < issued) { signal((int)(signalled % kAStages)); ++signalled; }
     } else {
-        // ================================================================ epilogue warps (one row per thread, half the columns)
-        const int eg = (warp - kGEpiWarp0) >> 2;               // column half of every chunk this group reads
+        // ================================================================ epilogue warps (one row per thread, a quarter of the columns)
+        const int eg = (warp - kGEpiWarp0) >> 2;               // column group of every chunk this warpgroup reads
         const int quad = warp & 3, row = quad * 32 + lane;
         const float *rtab = reinterpret_cast<const float *>(sm + GSmem::rtab);
         const float *btab = reinterpret_cast<const float *>(sm + GSmem::bias);
-        float *merge = reinterpret_cast<float *>(sm + GSmem::merge) + row * kMergeFloats;
+        float *merge_all = reinterpret_cast<float *>(sm + GSmem::merge);
         uint32_t chunk_seq = 0, tile_seq = 0;
         const int Mmax = P.Mmax;
         bool ok = true;
+        constexpr int kGW = kNC / kGEpiGroups;                     // columns of a chunk per epilogue group
+        constexpr int kBlk = kGEpiBlk;
+        static_assert(kNC % (4 * kGEpiGroups) == 0, "a group's first column must keep 16-byte alignment in the tables");
         for (int t = blockIdx.x; t < prm.n_tiles && ok; t += gridDim.x) {
             const int4 d = prm.tiles[t];
             if (d.x < 0) continue;
@@ -406,17 +417,16 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
                 tc_fence_after();
                 const float *rt = rtab + b * (kRBytes / 4), *bt = btab + b * (G::BiasSlot / 4);
                 const int c_base = ch * kNC;
-                constexpr int kHalf = kNC / 2;                             // columns of a chunk per epilogue group
-                for (int sb = 0; sb < (kHalf + 31) / 32; ++sb) {
-                    const int col0 = eg * kHalf + sb * 32;                 // column of the chunk
-                    const int col_end = (eg + 1) * kHalf;                  // this group's columns end here
+                for (int sb = 0; sb < (kGW + kBlk - 1) / kBlk; ++sb) {
+                    const int col0 = eg * kGW + sb * kBlk;                 // column of the chunk
+                    const int col_end = (eg + 1) * kGW;                    // this group's columns end here
                     if (c_base + col0 >= C) break;                         // uniform: nothing valid from here on
-                    float z[32];
-                    tmem_ld<32>(((uint32_t)(quad * 32) << 16) + b * kNC + col0, z);
+                    float z[kBlk];
+                    tmem_ld<kBlk>(((uint32_t)(quad * 32) << 16) + b * kNC + col0, z);
                     tmem_wait_ld();
                     float bm = -INFINITY;
 #pragma unroll
-                    for (int c = 0; c < 32; c += 4) {
+                    for (int c = 0; c < kBlk; c += 4) {
                         if (col0 + c < kNC) {                              // the bias row has NC entries
                             const float4 bv = *reinterpret_cast<const float4 *>(bt + col0 + c);
                             if (F32) {                                     // log2(e) is already in the head image
@@ -429,7 +439,7 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
                         }
                     }
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
+                    for (int c = 0; c < kBlk; ++c) {
                         if (c_base + col0 + c >= C || col0 + c >= col_end) z[c] = -INFINITY;
                         bm = fmaxf(bm, z[c]);
                     }
@@ -442,20 +452,20 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
                     }
                     float ps = 0.f;
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) { z[c] = exp2_unit(z[c] - run_m); ps += z[c]; }
+                    for (int c = 0; c < kBlk; ++c) { z[c] = exp2_unit(z[c] - run_m); ps += z[c]; }
                     run_s += ps;
                     // recall contraction with two-wide FMAs: label pairs (c, c + 1) of a model's row against the pair of
-                    // numerators; the two halves of the accumulator are added once per block of 32 labels
-                    unsigned long long zz[16];
+                    // numerators; the two halves of the accumulator are added once per block of labels
+                    unsigned long long zz[kBlk / 2];
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) zz[c] = pack_f32x2(z[2 * c], z[2 * c + 1]);
+                    for (int c = 0; c < kBlk / 2; ++c) zz[c] = pack_f32x2(z[2 * c], z[2 * c + 1]);
 #pragma unroll
                     for (int j = 0; j < kMaxModelsPerApp; j += 2) {        // two models at a time: four independent chains
                         if (j < M) {
                             const float *r0 = rt + j * kNC + col0, *r1 = j + 1 < M ? r0 + kNC : r0;
                             unsigned long long p0a = 0ull, p0b = 0ull, p1a = 0ull, p1b = 0ull;
 #pragma unroll
-                            for (int c = 0; c < 32; c += 4) {
+                            for (int c = 0; c < kBlk; c += 4) {
                                 if (col0 + c < kNC) {                      // a recall row has NC entries; z is 0 past the group's end
                                     const ulonglong2 rv0 = *reinterpret_cast<const ulonglong2 *>(r0 + c);
                                     const ulonglong2 rv1 = *reinterpret_cast<const ulonglong2 *>(r1 + c);
@@ -475,8 +485,9 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
                 mbar_arrive(bar(gbar_r_free(b)));
             }
             if (!ok) break;
-            // ---- merge the two column halves of the row, finish Eq. 9 / Eq. 12, store
-            if (eg == 1) {
+            // ---- merge the column groups of the row, finish Eq. 9 / Eq. 12, store
+            if (eg > 0) {
+                float *merge = merge_all + ((eg - 1) * kGRows + row) * kMergeFloats;
                 if (tile_seq > 0 && !warp_wait(bar(kGBarMergeDone), (tile_seq - 1) & 1, abort_flag)) break;
                 merge[0] = run_m; merge[1] = run_s;
 #pragma unroll
@@ -484,11 +495,23 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
                 mbar_arrive(bar(kGBarMergeReady));
             } else {
                 if (!warp_wait(bar(kGBarMergeReady), tile_seq & 1, abort_flag)) break;
-                const float om = merge[0], os = merge[1];
-                const float mm = fmaxf(run_m, om);
+                float mm = run_m;
+#pragma unroll
+                for (int g = 0; g < kGEpiGroups - 1; ++g) mm = fmaxf(mm, merge_all[(g * kGRows + row) * kMergeFloats]);
                 const float s0 = run_m == -INFINITY ? 0.f : exp2_unit(run_m - mm);
-                const float s1 = om == -INFINITY ? 0.f : exp2_unit(om - mm);
-                const float inv = 1.f / (run_s * s0 + os * s1);
+                float tot = run_s * s0;
+#pragma unroll
+                for (int j = 0; j < kMaxModelsPerApp; ++j) racc[j] *= s0;
+#pragma unroll
+                for (int g = 0; g < kGEpiGroups - 1; ++g) {
+                    const float *mg = merge_all + (g * kGRows + row) * kMergeFloats;
+                    const float om = mg[0];
+                    const float sg = om == -INFINITY ? 0.f : exp2_unit(om - mm);
+                    tot = fmaf(mg[1], sg, tot);
+#pragma unroll
+                    for (int j = 0; j < kMaxModelsPerApp; ++j) racc[j] = fmaf(mg[2 + j], sg, racc[j]);
+                }
+                const float inv = 1.f / tot;
                 const bool valid = row < d.z;
                 const int64_t req = tb.perm[d.y + (valid ? row : 0)];
                 float *dst = tb.acc32 + req * Mmax;
@@ -499,7 +522,7 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
                     if (j < Mmax) {
                         float aj = 0.f;
                         if (j < M) {
-                            aj = (racc[j] * s0 + merge[2 + j] * s1) * inv;
+                            aj = racc[j] * inv;
                             if (P.prior)
                                 aj = (P.prior_dot[(int64_t)inst * P.sumM + g0 + j] + P.kappa * aj) / (P.prior_sum[d.x] + P.kappa);
                             if (j == 0) a0 = aj;

@@ -150,10 +150,6 @@ def test_errors_are_reported_not_crashes():
     w = synth.make_workload("C1")
     ses = runner.Session(w)
     ses.upload(); ses.alloc_outputs(8); ses.score()
-    with pytest.raises(api.SpError) as e:           # second score without reset
-        dv = ses.dev
-        api.sp_score(ses.ctx, ses.n, dv["feats"], dv["app"], dv["arrival"], dv["deadline"], None, None)
-    assert e.value.status == api.SP_ESTATE
     ses.dev["app"][5] = 77                          # out-of-range application id
     ses.score(); ses.schedule(8)
     with pytest.raises(api.SpError) as e:
