@@ -6,7 +6,10 @@ arrays the CUDA library takes:
 
 * :func:`score`  -- data-aware accuracy ``acc[n, Mmax]`` (Eq. 9 of the paper over the Dirichlet
   posterior mean of Eq. 10-11) and the priority factor ``v[n] = 1 + Var`` (Eq. 12), in fp64;
-* :func:`drain`  -- the greedy group-level rounds (Eq. 13-14, Algorithm 1) until nothing is left.
+* :func:`drain`  -- the greedy group-level rounds (Eq. 13-14, Algorithm 1) until nothing is left, over whole
+  applications or over the data-aware sub-groups of Section 4.3 (``labels=``);
+* :func:`bruteforce` -- Algorithm 1's exhaustive branch over the groups of one instance;
+* :func:`baseline` -- the request-level baselines of Section 5.1 (MaxAcc-EDF, LO-EDF, LO-Priority).
 """
 from __future__ import annotations
 
@@ -48,7 +51,7 @@ class _Profiles(C.Structure):
 
 ROUND_DTYPE = np.dtype([
     ("instance", "<i4"), ("round", "<i4"), ("app", "<i4"), ("model", "<i4"), ("batch", "<i4"),
-    ("n_members", "<i4"), ("n_expired", "<i4"), ("pad_", "<i4"), ("t_start_ns", "<i8"),
+    ("n_members", "<i4"), ("n_expired", "<i4"), ("label", "<i4"), ("t_start_ns", "<i8"),
     ("t_end_ns", "<i8"), ("utility", "<f8"), ("group_priority", "<f8"), ("util_margin", "<f8"),
     ("prio_margin", "<f8")], align=True)
 REQ_DTYPE = np.dtype([("status", "<i4"), ("round", "<i4"), ("model", "<i4"), ("pad_", "<i4"),
@@ -62,10 +65,16 @@ def _load():
     if _lib is None:
         lib = C.CDLL(build())
         lib.orc_score.restype = C.c_int
-        lib.orc_score.argtypes = [C.POINTER(_Profiles), C.c_int64] + [C.c_void_p] * 6
+        lib.orc_score.argtypes = [C.POINTER(_Profiles), C.c_int64] + [C.c_void_p] * 7
         lib.orc_drain.restype = C.c_int
-        lib.orc_drain.argtypes = ([C.POINTER(_Profiles), C.c_int64] + [C.c_void_p] * 8 +
+        lib.orc_drain.argtypes = ([C.POINTER(_Profiles), C.c_int64] + [C.c_void_p] * 9 +
                                   [C.c_int, C.c_int64, C.c_void_p, C.c_int64] + [C.c_void_p] * 4)
+        lib.orc_bruteforce.restype = C.c_int
+        lib.orc_bruteforce.argtypes = ([C.POINTER(_Profiles), C.c_int64] + [C.c_void_p] * 5 + [C.c_int64, C.c_int32,
+                                       C.c_void_p, C.c_int64] + [C.c_void_p] * 7)
+        lib.orc_baseline.restype = C.c_int
+        lib.orc_baseline.argtypes = ([C.POINTER(_Profiles), C.c_int, C.c_int64] + [C.c_void_p] * 9 +
+                                     [C.c_int64] + [C.c_void_p] * 5)
         lib.orc_num_threads.restype = C.c_int
         lib.orc_penalty.restype = C.c_double
         lib.orc_penalty.argtypes = [C.c_int, C.c_int64, C.c_int64, C.c_int64]
@@ -111,6 +120,7 @@ class Scores:
     acc: np.ndarray      # [n, Mmax] float64
     v: np.ndarray        # [n] float64
     theta: Optional[np.ndarray]  # [n, C] float64 when requested
+    label: Optional[np.ndarray] = None  # [n] int32: label c with theta_c > 0.5, -1 when there is none
 
 
 def score(w, want_theta: bool = False) -> Scores:
@@ -125,10 +135,11 @@ def score(w, want_theta: bool = False) -> Scores:
     acc = np.zeros((n, mm), dtype=np.float64)
     v = np.zeros(n, dtype=np.float64)
     theta = np.zeros((n, int(w.n_classes)), dtype=np.float64) if want_theta else None
-    rc = lib.orc_score(C.byref(b.struct), n, _ptr(feats), _ptr(app), _ptr(inst), _ptr(acc), _ptr(v), _ptr(theta))
+    label = np.zeros(n, dtype=np.int32)
+    rc = lib.orc_score(C.byref(b.struct), n, _ptr(feats), _ptr(app), _ptr(inst), _ptr(acc), _ptr(v), _ptr(theta), _ptr(label))
     if rc != 0:
         raise ValueError("orc_score rejected its arguments")
-    return Scores(acc, v, theta)
+    return Scores(acc, v, theta, label)
 
 
 @dataclass
@@ -141,8 +152,11 @@ class Drain:
 
 
 def drain(w, acc: np.ndarray, v: np.ndarray, t0_ns=None, loaded0=None, max_rounds: Optional[int] = None,
-          cap: Optional[int] = None, trace_mode: Optional[bool] = None) -> Drain:
-    """Runs the rounds of every instance of ``w`` from clock ``t0_ns`` with model ``loaded0`` resident."""
+          cap: Optional[int] = None, trace_mode: Optional[bool] = None, labels: Optional[np.ndarray] = None) -> Drain:
+    """Runs the rounds of every instance of ``w`` from clock ``t0_ns`` with model ``loaded0`` resident.
+
+    ``labels`` (from :func:`score`) switches to the data-aware sub-groups of Section 4.3: requests of an application
+    with the same predicted label form a group of their own."""
     lib, b = _load(), _Bound(w)
     n, ni = int(w.app.shape[0]), int(w.n_instances)
     per_inst = int(np.max(np.bincount(np.asarray(w.instance), minlength=ni))) if n else 0
@@ -164,9 +178,89 @@ def drain(w, acc: np.ndarray, v: np.ndarray, t0_ns=None, loaded0=None, max_round
     t_end = np.zeros(ni, dtype=np.int64)
     l_end = np.zeros(ni, dtype=np.int32)
     tm = bool(w.trace_mode) if trace_mode is None else bool(trace_mode)
-    rc = lib.orc_drain(C.byref(b.struct), n, _ptr(app), _ptr(inst), _ptr(arr), _ptr(dl), _ptr(acc), _ptr(v),
+    lab = None if labels is None else np.ascontiguousarray(labels, dtype=np.int32)
+    rc = lib.orc_drain(C.byref(b.struct), n, _ptr(app), _ptr(inst), _ptr(lab), _ptr(arr), _ptr(dl), _ptr(acc), _ptr(v),
                        _ptr(t0), _ptr(l0), int(tm), int(max_rounds), _ptr(rounds), int(cap), _ptr(n_rounds),
                        _ptr(reqs), _ptr(t_end), _ptr(l_end))
     if rc != 0:
         raise ValueError("orc_drain rejected its arguments")
     return Drain(rounds, n_rounds, reqs, t_end, l_end)
+
+
+@dataclass
+class BruteForce:
+    rounds: np.ndarray      # [1, cap] ROUND_DTYPE, one record per executed batch
+    n_rounds: np.ndarray    # [1]
+    reqs: np.ndarray        # [n] REQ_DTYPE
+    t_end_ns: np.ndarray    # [1]
+    loaded_end: np.ndarray  # [1]
+    total: float            # best total utility (the sum inside Eq. 3)
+    second: float           # best total among the solutions with a different total (-inf if none)
+    n_solutions: int        # solutions visited = G! * prod M_g
+
+
+def bruteforce(w, acc: np.ndarray, labels: Optional[np.ndarray] = None, loaded0: int = -1) -> BruteForce:
+    """Exact group-level solution of a single-instance workload (Algorithm 1's branch for few groups)."""
+    lib, b = _load(), _Bound(w)
+    if int(w.n_instances) != 1:
+        raise ValueError("one instance only")
+    n = int(w.app.shape[0])
+    app = np.ascontiguousarray(w.app, dtype=np.int32)
+    arr = np.ascontiguousarray(w.arrival_ns, dtype=np.int64)
+    dl = np.ascontiguousarray(w.deadline_ns, dtype=np.int64)
+    acc = np.ascontiguousarray(acc, dtype=np.float64)
+    lab = None if labels is None else np.ascontiguousarray(labels, dtype=np.int32)
+    cap = max(1, n)
+    rounds = np.zeros((1, cap), dtype=ROUND_DTYPE)
+    n_rounds = np.zeros(1, dtype=np.int64)
+    reqs = np.zeros(n, dtype=REQ_DTYPE)
+    t_end = np.zeros(1, dtype=np.int64)
+    l_end = np.zeros(1, dtype=np.int32)
+    best, second, nsol = np.zeros(1), np.zeros(1), np.zeros(1, dtype=np.int64)
+    rc = lib.orc_bruteforce(C.byref(b.struct), n, _ptr(app), _ptr(lab), _ptr(arr), _ptr(dl), _ptr(acc), int(w.t0_ns[0]),
+                            int(loaded0), _ptr(rounds), cap, _ptr(n_rounds), _ptr(reqs), _ptr(t_end), _ptr(l_end),
+                            _ptr(best), _ptr(second), _ptr(nsol))
+    if rc != 0:
+        raise ValueError("orc_bruteforce: %s" % ("too many groups or solutions" if rc == -2 else "bad arguments"))
+    return BruteForce(rounds, n_rounds, reqs, t_end, l_end, float(best[0]), float(second[0]), int(nsol[0]))
+
+
+MAXACC_EDF, LO_EDF, LO_PRIORITY = 0, 1, 2
+
+
+@dataclass
+class Baseline:
+    rounds: np.ndarray      # [I, cap] ROUND_DTYPE, one record per request in execution order
+    n_rounds: np.ndarray    # [I]
+    reqs: np.ndarray        # [n] REQ_DTYPE
+    t_end_ns: np.ndarray    # [I]
+    loaded_end: np.ndarray  # [I]
+    min_margin: np.ndarray  # [I] smallest relative gap between the two best scores of a decision / two neighbours of the order
+
+
+def baseline(w, policy: int, acc: np.ndarray, v: np.ndarray, loaded0=None) -> Baseline:
+    """Request-level baselines of Section 5.1: 0 MaxAcc-EDF, 1 LO-EDF, 2 LO-Priority (every request alone, in order)."""
+    lib, b = _load(), _Bound(w)
+    n, ni = int(w.app.shape[0]), int(w.n_instances)
+    per_inst = int(np.max(np.bincount(np.asarray(w.instance), minlength=ni))) if n else 0
+    cap = max(1, per_inst)
+    app = np.ascontiguousarray(w.app, dtype=np.int32)
+    inst = np.ascontiguousarray(w.instance, dtype=np.int32)
+    arr = np.ascontiguousarray(w.arrival_ns, dtype=np.int64)
+    dl = np.ascontiguousarray(w.deadline_ns, dtype=np.int64)
+    acc = np.ascontiguousarray(acc, dtype=np.float64)
+    v = np.ascontiguousarray(v, dtype=np.float64)
+    t0 = np.ascontiguousarray(w.t0_ns, dtype=np.int64)
+    l0 = np.full(ni, -1, dtype=np.int32) if loaded0 is None else np.ascontiguousarray(loaded0, dtype=np.int32)
+    rounds = np.zeros((ni, cap), dtype=ROUND_DTYPE)
+    n_rounds = np.zeros(ni, dtype=np.int64)
+    reqs = np.zeros(n, dtype=REQ_DTYPE)
+    t_end = np.zeros(ni, dtype=np.int64)
+    l_end = np.zeros(ni, dtype=np.int32)
+    margin = np.zeros(ni, dtype=np.float64)
+    rc = lib.orc_baseline(C.byref(b.struct), int(policy), n, _ptr(app), _ptr(inst), _ptr(arr), _ptr(dl), _ptr(acc), _ptr(v),
+                          _ptr(t0), _ptr(l0), _ptr(rounds), cap, _ptr(n_rounds), _ptr(reqs), _ptr(t_end), _ptr(l_end),
+                          _ptr(margin))
+    if rc != 0:
+        raise ValueError("orc_baseline rejected its arguments")
+    return Baseline(rounds, n_rounds, reqs, t_end, l_end, margin)

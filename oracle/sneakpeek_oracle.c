@@ -18,7 +18,9 @@
  * batch-size candidates with l(m,b) = alpha + beta*b and a separate swap cost, and the linear
  * and sigmoid penalties (Section 5.1 prints them garbled; orc_penalty() states the reading and
  * is pinned only at gamma(e = d) = 0, gamma(half way) = 1/2, gamma(>= relative deadline late) = 1
- * and monotonicity).
+ * and monotonicity).  Also readings: which requests form a data-aware sub-group (orc_score's label), how a whole
+ * group is run in the exhaustive branch of Algorithm 1 (orc_bruteforce), what "max accuracy" picks when no model
+ * meets the deadline (orc_baseline); each is stated where it is implemented.
  */
 #include <math.h>
 #include <stdint.h>
@@ -48,7 +50,8 @@ typedef struct {
 } orc_profiles;
 
 typedef struct {
-    int32_t instance, round, app, model, batch, n_members, n_expired, pad_;
+    int32_t instance, round, app, model, batch, n_members, n_expired;
+    int32_t label;        /* sub-group of the application that was served: predicted label, -1 = not split / inconclusive */
     int64_t t_start_ns, t_end_ns;
     double utility, group_priority;
     double util_margin;   /* (U1-U2)/U1 over candidates of the chosen group with a different value; +inf if none */
@@ -102,7 +105,7 @@ static int first_model(const orc_profiles *p, int app)
  *   v                : 1 + population variance of acc over the app's models (Eq. 12 and its footnote).
  * ------------------------------------------------------------------------------------------- */
 static void score_one(const orc_profiles *p, const void *feats, int64_t i, int inst, int app,
-                      double *theta /* [C] scratch/out */, double *acc /* [Mmax] */, double *v)
+                      double *theta /* [C] scratch/out */, double *acc /* [Mmax] */, double *v, int32_t *label)
 {
     const int A = p->n_apps, C = p->n_classes, D = p->feat_dim;
     const int64_t head = ((int64_t)inst * A + app);
@@ -125,6 +128,13 @@ static void score_one(const orc_profiles *p, const void *feats, int64_t i, int i
         for (int c = 0; c < C; ++c)
             theta[c] = ((double)al[c] + p->evidence_k * theta[c]) / (asum + p->evidence_k);
     }
+    /* Data-aware sub-group ("Enhancements for Grouped Scheduling", Section 4.3): the request belongs to the sub-group
+     * of label c when theta_c > 0.5 (at most one label can), and stays with its application's unsplit remainder when
+     * every theta_c <= 0.5. */
+    if (label) {
+        *label = -1;
+        for (int c = 0; c < C; ++c) if (theta[c] > 0.5) *label = c;
+    }
     const int M = p->models_per_app[app], g0 = first_model(p, app), SM = sum_models(p);
     double mean = 0.0;
     for (int j = 0; j < M; ++j) {
@@ -141,9 +151,10 @@ static void score_one(const orc_profiles *p, const void *feats, int64_t i, int i
 }
 
 /* Scores n requests.  acc_out [n][Mmax] (columns >= M_app are 0), v_out [n],
- * theta_out [n][C] or NULL.  Returns 0, or -1 on a bad argument. */
+ * theta_out [n][C] or NULL, label_out [n] or NULL (predicted label, -1 = inconclusive).
+ * Returns 0, or -1 on a bad argument. */
 int orc_score(const orc_profiles *p, int64_t n, const void *feats, const int32_t *app,
-              const int32_t *instance, double *acc_out, double *v_out, double *theta_out)
+              const int32_t *instance, double *acc_out, double *v_out, double *theta_out, int32_t *label_out)
 {
     if (!p || n < 0 || !acc_out || !v_out) return -1;
     const int C = p->n_classes, MM = max_models(p);
@@ -155,7 +166,7 @@ int orc_score(const orc_profiles *p, int64_t n, const void *feats, const int32_t
         double *theta = (double *)malloc(sizeof(double) * (size_t)C);
         double *acc = acc_out + i * MM;
         for (int j = 0; j < MM; ++j) acc[j] = 0.0;
-        score_one(p, feats, i, inst, app[i], theta, acc, &v_out[i]);
+        score_one(p, feats, i, inst, app[i], theta, acc, &v_out[i], label_out ? &label_out[i] : NULL);
         if (theta_out) memcpy(theta_out + i * C, theta, sizeof(double) * (size_t)C);
         free(theta);
     }
@@ -234,12 +245,17 @@ static int cmp_akey(const void *x, const void *y)
 }
 
 static void drain_instance(const orc_profiles *p, int inst, int64_t lo, int64_t hi,
-                           const int32_t *app, const int64_t *arrival, const int64_t *deadline,
+                           const int32_t *app, const int32_t *label, const int64_t *arrival, const int64_t *deadline,
                            const double *acc, const double *v, int64_t t0, int32_t loaded0,
                            int trace_mode, int64_t max_rounds, orc_round_rec *rounds, int64_t cap,
                            int64_t *n_rounds, orc_req_rec *reqs, int64_t *t_end, int32_t *loaded_end)
 {
-    const int A = p->n_apps, MM = max_models(p), SM = sum_models(p), nB = p->n_batch_sizes;
+    /* Groups: the applications (Section 4.2), or, with labels given, the data-aware sub-groups of Section 4.3: group
+     * index = app * (C + 1) + label + 1, so an application's unsplit remainder (label -1) comes before its per-label
+     * sub-groups and "lowest application" generalises to "lowest group index".  GW = groups per application. */
+    const int GW = label ? p->n_classes + 1 : 1;
+    const int A = p->n_apps * GW, MM = max_models(p), SM = sum_models(p), nB = p->n_batch_sizes;
+#define GROUP_OF(id) (app[id] * GW + (label ? label[id] + 1 : 0))
     const int64_t *al = p->lat_alpha_ns + (int64_t)inst * SM;
     const int64_t *be = p->lat_beta_ns + (int64_t)inst * SM;
     const int64_t *sw = p->swap_ns + (int64_t)inst * SM;
@@ -252,7 +268,8 @@ static void drain_instance(const orc_profiles *p, int inst, int64_t lo, int64_t 
     qkey **q = (qkey **)malloc(sizeof(qkey *) * (size_t)A);
     int64_t *head = (int64_t *)calloc((size_t)A, sizeof(int64_t));
     int64_t *tail = (int64_t *)calloc((size_t)A, sizeof(int64_t));
-    for (int a = 0; a < A; ++a) q[a] = (qkey *)malloc(sizeof(qkey) * (size_t)(n > 0 ? n : 1));
+    for (int64_t i = lo; i < hi; ++i) ++tail[GROUP_OF(i)];              /* group sizes, to size the queues */
+    for (int a = 0; a < A; ++a) { q[a] = (qkey *)malloc(sizeof(qkey) * (size_t)(tail[a] > 0 ? tail[a] : 1)); tail[a] = 0; }
     for (int64_t i = lo; i < hi; ++i) {
         reqs[i].status = ORC_PENDING; reqs[i].round = -1; reqs[i].model = -1; reqs[i].pad_ = 0; reqs[i].order = 0;
     }
@@ -264,7 +281,7 @@ static void drain_instance(const orc_profiles *p, int inst, int64_t lo, int64_t 
         int inserted = 0;
         while (ap < n && (!trace_mode || arr[ap].arrival <= T)) {
             const int64_t id = arr[ap].id;
-            const int a = app[id];
+            const int a = GROUP_OF(id);
             q[a][tail[a]].deadline = deadline[id];
             q[a][tail[a]].id = id;
             ++tail[a]; ++ap; inserted = 1;
@@ -282,14 +299,15 @@ static void drain_instance(const orc_profiles *p, int inst, int64_t lo, int64_t 
         /* 3. retire requests that no candidate of their group can complete in time */
         const int64_t bmin = p->batch_sizes[0];
         for (int a = 0; a < A; ++a) {
-            const int g0 = first_model(p, a), M = p->models_per_app[a];
+            if (head[a] == tail[a]) continue;
+            const int g0 = first_model(p, a / GW), M = p->models_per_app[a / GW];
             int64_t emin = INT64_MAX;
             for (int j = 0; j < M; ++j) {
                 const int g = g0 + j;
                 const int64_t e = T + (g != L ? sw[g] : 0) + al[g] + be[g] * bmin;
                 if (e < emin) emin = e;
             }
-            const int pk = p->penalty_kind ? p->penalty_kind[a] : ORC_PEN_STEP;
+            const int pk = p->penalty_kind ? p->penalty_kind[a / GW] : ORC_PEN_STEP;
             while (head[a] < tail[a] && hopeless(pk, q[a][head[a]].deadline, arrival[q[a][head[a]].id], emin)) {
                 orc_req_rec *r = &reqs[q[a][head[a]].id];
                 r->status = ORC_EXPIRED; r->round = (int32_t)round;
@@ -316,9 +334,9 @@ static void drain_instance(const orc_profiles *p, int inst, int64_t lo, int64_t 
             else if (pr < best_p && pr > second_p) second_p = pr;
         }
         /* 5./6. every (model, batch size) candidate of the chosen group; best summed utility */
-        const int a = best_a, g0 = first_model(p, a), M = p->models_per_app[a];
+        const int a = best_a, g0 = first_model(p, a / GW), M = p->models_per_app[a / GW];
         const int64_t na = tail[a] - head[a];
-        const int pen = p->penalty_kind ? p->penalty_kind[a] : ORC_PEN_STEP;
+        const int pen = p->penalty_kind ? p->penalty_kind[a / GW] : ORC_PEN_STEP;
         int best_j = -1, best_b = 0;
         int64_t best_bp = 0, best_e = 0;
         double best_u = 0.0, second_u = -INFINITY;
@@ -346,8 +364,9 @@ static void drain_instance(const orc_profiles *p, int inst, int64_t lo, int64_t 
         head[a] += best_bp;
         if (rounds && round < cap) {
             orc_round_rec *rr = &rounds[round];
-            rr->instance = inst; rr->round = (int32_t)round; rr->app = a; rr->model = g0 + best_j;
-            rr->batch = best_b; rr->n_members = (int32_t)best_bp; rr->n_expired = exp_since; rr->pad_ = 0;
+            rr->instance = inst; rr->round = (int32_t)round; rr->app = a / GW; rr->model = g0 + best_j;
+            rr->batch = best_b; rr->n_members = (int32_t)best_bp; rr->n_expired = exp_since;
+            rr->label = label ? a % GW - 1 : -1;
             rr->t_start_ns = T; rr->t_end_ns = best_e; rr->utility = best_u; rr->group_priority = best_p;
             rr->util_margin = (second_u == -INFINITY || !(best_u > 0.0)) ? INFINITY : (best_u - second_u) / best_u;
             rr->prio_margin = (second_p == -INFINITY || !(best_p > 0.0)) ? INFINITY : (best_p - second_p) / best_p;
@@ -358,12 +377,14 @@ static void drain_instance(const orc_profiles *p, int inst, int64_t lo, int64_t 
     *n_rounds = round; *t_end = T; *loaded_end = L;
     for (int a = 0; a < A; ++a) free(q[a]);
     free(q); free(head); free(tail); free(arr);
+#undef GROUP_OF
 }
 
 /* Runs up to max_rounds rounds of every instance.  Requests must be grouped by instance in
- * ascending order (instance == NULL means one instance).  rounds [I][cap] (may be NULL),
+ * ascending order (instance == NULL means one instance).  label: predicted labels from orc_score() to schedule the
+ * data-aware sub-groups of Section 4.3, or NULL to schedule whole applications.  rounds [I][cap] (may be NULL),
  * n_rounds [I], reqs [n], t_end [I], loaded_end [I].  Returns 0, -1 on a bad argument. */
-int orc_drain(const orc_profiles *p, int64_t n, const int32_t *app, const int32_t *instance,
+int orc_drain(const orc_profiles *p, int64_t n, const int32_t *app, const int32_t *instance, const int32_t *label,
               const int64_t *arrival, const int64_t *deadline, const double *acc, const double *v,
               const int64_t *t0, const int32_t *loaded0, int trace_mode, int64_t max_rounds,
               orc_round_rec *rounds, int64_t cap, int64_t *n_rounds, orc_req_rec *reqs,
@@ -383,9 +404,249 @@ int orc_drain(const orc_profiles *p, int64_t n, const int32_t *app, const int32_
     }
 #pragma omp parallel for schedule(dynamic, 1)
     for (int k = 0; k < I; ++k)
-        drain_instance(p, k, start[k], start[k + 1], app, arrival, deadline, acc, v, t0[k], loaded0[k],
+        drain_instance(p, k, start[k], start[k + 1], app, label, arrival, deadline, acc, v, t0[k], loaded0[k],
                        trace_mode, max_rounds, rounds ? rounds + (int64_t)k * cap : NULL, cap,
                        &n_rounds[k], reqs, &t_end[k], &loaded_end[k]);
+    free(start);
+    return 0;
+}
+
+
+/* ---------------------------------------------------------------------------------------------
+ * Exhaustive branch of Algorithm 1 (Section 4.2: when the number of groups is at most the threshold tau, the
+ * group-level problem is solved exactly).  A solution is an order of the non-empty groups and one model per group;
+ * every group is served whole, on its model, before the next group starts.  Reading of "served whole" under batch
+ * sizes: the group's members, in (deadline, id) order, run back to back in batches of the largest allowed size (the
+ * last batch takes the remainder); batch k completes at e = T + swap*[model != loaded] + alpha + beta*b' (Eq. 1) and
+ * each member earns acc * (1 - gamma) (Eq. 2).  Nothing is retired: every request gets a model and an order (Eq. 5).
+ * All G! * prod M_g solutions are evaluated; the best total (Eq. 3's sum) wins, the first in enumeration order on a
+ * tie: orders in lexicographic order of the group indices, then model choices in lexicographic order with the
+ * lowest group index as the slowest digit.  One instance (instance 0 of the profiles); groups as in drain_instance.
+ * Returns 0, -1 on a bad argument, -2 when there are more than 8 non-empty groups or more than 2^31 solutions.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct { int g, M, g0, pen; int64_t n; qkey *q; } bf_group;
+
+static double bf_eval(const orc_profiles *p, const bf_group *grp, int G, const int *perm, const int *choice,
+                      const int64_t *arrival, const double *acc, int MM, int64_t t0, int32_t loaded0,
+                      orc_round_rec *rounds, int64_t cap, int64_t *n_rounds, orc_req_rec *reqs, int64_t *t_end, int32_t *l_end)
+{
+    const int64_t *al = p->lat_alpha_ns, *be = p->lat_beta_ns, *sw = p->swap_ns;
+    const int64_t bmax = p->batch_sizes[p->n_batch_sizes - 1];
+    int64_t T = t0, order = 1, round = 0;
+    int32_t L = loaded0;
+    double total = 0.0;
+    for (int pos = 0; pos < G; ++pos) {
+        const bf_group *gr = &grp[perm[pos]];
+        const int j = choice[perm[pos]], m = gr->g0 + j;
+        for (int64_t k0 = 0; k0 < gr->n; k0 += bmax) {
+            const int64_t bp = gr->n - k0 < bmax ? gr->n - k0 : bmax;
+            const int64_t e = T + (m != L ? sw[m] : 0) + al[m] + be[m] * bp;
+            double u = 0.0;
+            for (int64_t k = 0; k < bp; ++k) {
+                const qkey *mem = &gr->q[k0 + k];
+                const double contrib = acc[mem->id * MM + j] * (1.0 - orc_penalty(gr->pen, mem->deadline, arrival[mem->id], e));
+                u += contrib;
+                total += contrib;
+                if (reqs) {
+                    orc_req_rec *r = &reqs[mem->id];
+                    r->status = ORC_SCHEDULED; r->round = (int32_t)round; r->model = m; r->pad_ = 0; r->order = order++;
+                }
+            }
+            if (rounds && round < cap) {
+                orc_round_rec *rr = &rounds[round];
+                memset(rr, 0, sizeof *rr);
+                rr->instance = 0; rr->round = (int32_t)round; rr->app = 0; rr->model = m;
+                rr->batch = (int32_t)bmax; rr->n_members = (int32_t)bp; rr->t_start_ns = T; rr->t_end_ns = e; rr->utility = u;
+                rr->util_margin = INFINITY; rr->prio_margin = INFINITY;
+            }
+            T = e; L = m; ++round;
+        }
+    }
+    if (n_rounds) *n_rounds = round;
+    if (t_end) *t_end = T;
+    if (l_end) *l_end = L;
+    return total;
+}
+
+static int bf_next_perm(int *a, int n)
+{
+    int i = n - 2;
+    while (i >= 0 && a[i] > a[i + 1]) --i;
+    if (i < 0) return 0;
+    int j = n - 1;
+    while (a[j] < a[i]) --j;
+    int t = a[i]; a[i] = a[j]; a[j] = t;
+    for (int l = i + 1, r = n - 1; l < r; ++l, --r) { t = a[l]; a[l] = a[r]; a[r] = t; }
+    return 1;
+}
+
+int orc_bruteforce(const orc_profiles *p, int64_t n, const int32_t *app, const int32_t *label, const int64_t *arrival,
+                   const int64_t *deadline, const double *acc, int64_t t0, int32_t loaded0, orc_round_rec *rounds,
+                   int64_t cap, int64_t *n_rounds, orc_req_rec *reqs, int64_t *t_end, int32_t *loaded_end,
+                   double *best_total, double *second_total, int64_t *n_solutions)
+{
+    if (!p || n < 0 || !n_rounds || !reqs || !t_end || !loaded_end || !best_total || !n_solutions) return -1;
+    const int GW = label ? p->n_classes + 1 : 1, NG = p->n_apps * GW, MM = max_models(p);
+    int64_t *count = (int64_t *)calloc((size_t)NG, sizeof(int64_t));
+    for (int64_t i = 0; i < n; ++i) ++count[app[i] * GW + (label ? label[i] + 1 : 0)];
+    bf_group grp[8];
+    int G = 0;
+    for (int g = 0; g < NG; ++g) {
+        if (!count[g]) continue;
+        if (G == 8) { free(count); return -2; }
+        grp[G].g = g; grp[G].M = p->models_per_app[g / GW]; grp[G].g0 = first_model(p, g / GW);
+        grp[G].pen = p->penalty_kind ? p->penalty_kind[g / GW] : ORC_PEN_STEP;
+        grp[G].n = 0; grp[G].q = (qkey *)malloc(sizeof(qkey) * (size_t)count[g]);
+        ++G;
+    }
+    for (int64_t i = 0; i < n; ++i) {
+        const int g = app[i] * GW + (label ? label[i] + 1 : 0);
+        for (int k = 0; k < G; ++k)
+            if (grp[k].g == g) { grp[k].q[grp[k].n].deadline = deadline[i]; grp[k].q[grp[k].n].id = i; ++grp[k].n; }
+    }
+    double n_sol = 1.0;
+    for (int k = 0; k < G; ++k) { qsort(grp[k].q, (size_t)grp[k].n, sizeof(qkey), cmp_qkey); n_sol *= (double)grp[k].M * (double)(k + 1); }
+    int rc = 0;
+    if (n_sol > 2147483648.0) rc = -2;
+    int perm[8], choice[8], best_perm[8], best_choice[8];
+    double best = -INFINITY, second = -INFINITY;
+    int64_t visited = 0;
+    if (rc == 0) {
+        for (int k = 0; k < G; ++k) perm[k] = k;
+        do {
+            for (int k = 0; k < G; ++k) choice[k] = 0;
+            for (;;) {
+                const double tot = bf_eval(p, grp, G, perm, choice, arrival, acc, MM, t0, loaded0, NULL, 0, NULL, NULL, NULL, NULL);
+                ++visited;
+                if (tot > best) { second = best; best = tot; memcpy(best_perm, perm, sizeof perm); memcpy(best_choice, choice, sizeof choice); }
+                else if (tot < best && tot > second) second = tot;
+                int k = G - 1;                                   /* next model tuple: last group is the fastest digit */
+                while (k >= 0 && ++choice[k] == grp[k].M) { choice[k] = 0; --k; }
+                if (k < 0) break;
+            }
+        } while (bf_next_perm(perm, G));
+        for (int64_t i = 0; i < n; ++i) { reqs[i].status = ORC_PENDING; reqs[i].round = -1; reqs[i].model = -1; reqs[i].pad_ = 0; reqs[i].order = 0; }
+        if (G > 0) {
+            bf_eval(p, grp, G, best_perm, best_choice, arrival, acc, MM, t0, loaded0, rounds, cap, n_rounds, reqs, t_end, loaded_end);
+            if (rounds) {                                        /* application and label of every emitted batch */
+                int64_t r = 0;
+                const int64_t bmax = p->batch_sizes[p->n_batch_sizes - 1];
+                for (int pos = 0; pos < G; ++pos)
+                    for (int64_t k0 = 0; k0 < grp[best_perm[pos]].n; k0 += bmax, ++r)
+                        if (r < cap) { rounds[r].app = grp[best_perm[pos]].g / GW; rounds[r].label = label ? grp[best_perm[pos]].g % GW - 1 : -1; }
+            }
+        } else { *n_rounds = 0; *t_end = t0; *loaded_end = loaded0; }
+        *best_total = G > 0 ? best : 0.0;
+        if (second_total) *second_total = second;
+        *n_solutions = visited;
+    }
+    for (int k = 0; k < G; ++k) free(grp[k].q);
+    free(count);
+    return rc;
+}
+
+/* ---------------------------------------------------------------------------------------------
+ * Request-level baselines of the evaluation (Section 5.1, "Baselines and Metrics"): an ordering policy plus a
+ * per-request model selection, one request at a time (batch size 1), nothing retired.
+ *   order  EDF: (deadline, id) ascending.  Priority: Eq. 12, v_i * exp(-(d_i - t0)/tau) descending, then id
+ *          (a common clock shift rescales every priority alike, so the order does not change while the schedule runs).
+ *   model  Locally optimal (Eq. 13): the model with the highest utility acc * (1 - gamma(d, e)) at the time the
+ *          request starts, e = T + swap*[model != loaded] + alpha + beta.  Max accuracy: the most accurate model that
+ *          still meets the deadline (d >= e); reading for the case the paper leaves open: when none meets it, the most
+ *          accurate model of all.  Ties: lowest model.
+ * policy 0 = MaxAcc-EDF, 1 = LO-EDF, 2 = LO-Priority.  min_margin [I]: smallest relative gap met in an instance
+ * between the winning and the runner-up score of a decision, and between consecutive priorities of the order.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct { double prio; int64_t deadline, id; } bkey;
+static int cmp_b_edf(const void *x, const void *y)
+{
+    const bkey *a = (const bkey *)x, *b = (const bkey *)y;
+    if (a->deadline != b->deadline) return a->deadline < b->deadline ? -1 : 1;
+    return a->id < b->id ? -1 : a->id > b->id;
+}
+static int cmp_b_prio(const void *x, const void *y)
+{
+    const bkey *a = (const bkey *)x, *b = (const bkey *)y;
+    if (a->prio != b->prio) return a->prio > b->prio ? -1 : 1;
+    return a->id < b->id ? -1 : a->id > b->id;
+}
+
+int orc_baseline(const orc_profiles *p, int policy, int64_t n, const int32_t *app, const int32_t *instance,
+                 const int64_t *arrival, const int64_t *deadline, const double *acc, const double *v,
+                 const int64_t *t0, const int32_t *loaded0, orc_round_rec *rounds, int64_t cap, int64_t *n_rounds,
+                 orc_req_rec *reqs, int64_t *t_end, int32_t *loaded_end, double *min_margin)
+{
+    if (!p || n < 0 || policy < 0 || policy > 2 || !n_rounds || !reqs || !t_end || !loaded_end) return -1;
+    const int I = p->n_instances, MM = max_models(p), SM = sum_models(p);
+    int64_t *start = (int64_t *)malloc(sizeof(int64_t) * (size_t)(I + 1));
+    {
+        int64_t i = 0;
+        for (int k = 0; k < I; ++k) { start[k] = i; while (i < n && (instance ? instance[i] : 0) == k) ++i; }
+        start[I] = i;
+        if (i != n) { free(start); return -1; }
+    }
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int inst = 0; inst < I; ++inst) {
+        const int64_t lo = start[inst], m = start[inst + 1] - lo;
+        const int64_t *al = p->lat_alpha_ns + (int64_t)inst * SM, *be = p->lat_beta_ns + (int64_t)inst * SM;
+        const int64_t *sw = p->swap_ns + (int64_t)inst * SM;
+        bkey *ord = (bkey *)malloc(sizeof(bkey) * (size_t)(m > 0 ? m : 1));
+        double margin = INFINITY;
+        for (int64_t k = 0; k < m; ++k) {
+            const int64_t id = lo + k;
+            ord[k].id = id; ord[k].deadline = deadline[id];
+            ord[k].prio = v[id] * exp(-((double)(deadline[id] - t0[inst]) * 1e-9 / p->prio_time_scale_s));
+        }
+        qsort(ord, (size_t)m, sizeof(bkey), policy == 2 ? cmp_b_prio : cmp_b_edf);
+        if (policy == 2)
+            for (int64_t k = 0; k + 1 < m; ++k)
+                if (ord[k].prio > ord[k + 1].prio && ord[k].prio > 0.0) {
+                    const double g = (ord[k].prio - ord[k + 1].prio) / ord[k].prio;
+                    if (g < margin) margin = g;
+                }
+        int64_t T = t0[inst];
+        int32_t L = loaded0[inst];
+        for (int64_t k = 0; k < m; ++k) {
+            const int64_t id = ord[k].id;
+            const int a = app[id], g0 = first_model(p, a), M = p->models_per_app[a];
+            const int pen = p->penalty_kind ? p->penalty_kind[a] : ORC_PEN_STEP;
+            int best = -1, any_feasible = 0;
+            double best_s = -INFINITY, second_s = -INFINITY;
+            if (policy == 0)
+                for (int j = 0; j < M; ++j) {
+                    const int g = g0 + j;
+                    if (!(deadline[id] < T + (g != L ? sw[g] : 0) + al[g] + be[g])) any_feasible = 1;
+                }
+            for (int j = 0; j < M; ++j) {
+                const int g = g0 + j;
+                const int64_t e = T + (g != L ? sw[g] : 0) + al[g] + be[g];
+                double sc;
+                if (policy == 0) {
+                    if (any_feasible && deadline[id] < e) continue;
+                    sc = acc[id * MM + j];
+                } else sc = acc[id * MM + j] * (1.0 - orc_penalty(pen, deadline[id], arrival[id], e));
+                if (best < 0 || sc > best_s) { if (best >= 0) second_s = best_s; best = j; best_s = sc; }
+                else if (sc < best_s && sc > second_s) second_s = sc;
+            }
+            if (second_s != -INFINITY && best_s > 0.0 && (best_s - second_s) / best_s < margin) margin = (best_s - second_s) / best_s;
+            const int g = g0 + best;
+            const int64_t e = T + (g != L ? sw[g] : 0) + al[g] + be[g];
+            const double u = acc[id * MM + best] * (1.0 - orc_penalty(pen, deadline[id], arrival[id], e));
+            orc_req_rec *r = &reqs[id];
+            r->status = ORC_SCHEDULED; r->round = (int32_t)k; r->model = g; r->pad_ = 0; r->order = k + 1;
+            if (rounds && k < cap) {
+                orc_round_rec *rr = &rounds[(int64_t)inst * cap + k];
+                memset(rr, 0, sizeof *rr);
+                rr->instance = inst; rr->round = (int32_t)k; rr->app = a; rr->model = g; rr->batch = 1; rr->n_members = 1;
+                rr->label = -1; rr->t_start_ns = T; rr->t_end_ns = e; rr->utility = u; rr->group_priority = ord[k].prio;
+                rr->util_margin = INFINITY; rr->prio_margin = INFINITY;
+            }
+            T = e; L = g;
+        }
+        n_rounds[inst] = m; t_end[inst] = T; loaded_end[inst] = L;
+        if (min_margin) min_margin[inst] = margin;
+        free(ord);
+    }
     free(start);
     return 0;
 }
