@@ -181,6 +181,35 @@ sp_status sp_get_scores(sp_ctx *ctx, int64_t first, int64_t n, float *acc, float
 sp_status sp_schedule_round(sp_ctx *ctx, int32_t max_rounds, sp_round_rec *rounds_out, int64_t cap,
                             int32_t *n_done);
 
+/*
+ * Three more ways to schedule a freshly scored SNAPSHOT table (no round run on it yet, not trace mode; otherwise
+ * SP_ESTATE).  All three first compute the fp64 scores and the data-aware label of every request in one pass over the
+ * whole table and take every decision on those, run the table to completion in one call, and write records like
+ * sp_schedule_round() (rounds_out DEVICE [I][cap] or NULL, n_done DEVICE [I] or NULL; sp_round_rec.exact carries the
+ * sub-group: bits 8 and up hold predicted label + 1, 0 = the application's unsplit remainder or no sub-groups).
+ *
+ * sp_schedule_split: the greedy rounds of Algorithm 1 over data-aware sub-groups (Section 4.3, "Enhancements for Grouped
+ *   Scheduling"): requests of an application whose posterior gives one label more than one half form a group of their
+ *   own, the others stay together; Eq. 14, the purge and the (model, batch size) candidates apply per sub-group.  Ties
+ *   between groups go to the lowest application, then the unsplit remainder, then the lowest label.
+ * sp_schedule_exhaustive: Algorithm 1's branch for few groups (Section 4.2): every order of the non-empty groups
+ *   (applications, or sub-groups when split != 0) times every model per group; a group is served whole on its model,
+ *   members in (deadline, id) order in batches of the largest allowed size, nothing is retired; the best total utility
+ *   wins (ties: first in lexicographic order of the group order, then of the model choices).  Single-instance contexts;
+ *   at most 8 non-empty groups and 2^31 solutions (SP_EINVAL beyond).  Synchronous.  total_out / n_solutions_out: HOST,
+ *   optional.
+ * sp_schedule_baseline: the request-level baselines of Section 5.1, one request at a time in EDF or Eq. 12 priority
+ *   order: SP_BASE_MAXACC_EDF (most accurate model that meets the deadline, else the most accurate of all),
+ *   SP_BASE_LO_EDF and SP_BASE_LO_PRIORITY (Eq. 13: highest utility at the time the request starts).  Nothing is retired.
+ * sp_get_labels: the labels (-1 = none above one half) to a DEVICE buffer, after one of the three calls.
+ */
+enum { SP_BASE_MAXACC_EDF = 0, SP_BASE_LO_EDF = 1, SP_BASE_LO_PRIORITY = 2 };
+sp_status sp_schedule_split(sp_ctx *ctx, sp_round_rec *rounds_out, int64_t cap, int32_t *n_done);
+sp_status sp_schedule_exhaustive(sp_ctx *ctx, int32_t split, sp_round_rec *rounds_out, int64_t cap, int32_t *n_done,
+                                 double *total_out, int64_t *n_solutions_out);
+sp_status sp_schedule_baseline(sp_ctx *ctx, int32_t policy, sp_round_rec *rounds_out, int64_t cap, int32_t *n_done);
+sp_status sp_get_labels(sp_ctx *ctx, int64_t first, int64_t n, int32_t *labels);
+
 /* Copies the records of requests first..first+n-1 to a DEVICE buffer. */
 sp_status sp_get_requests(sp_ctx *ctx, int64_t first, int64_t n, sp_req_rec *out);
 /* Copies every instance's clock and resident model to DEVICE buffers t_ns [I], loaded_model [I]. */

@@ -110,7 +110,7 @@ class _Bound:
         k = self.keep
         self.struct = _Profiles(
             int(w.n_instances), int(w.n_apps), int(w.n_classes), int(w.feat_dim), int(w.feat_dtype),
-            _ptr(k["mpa"]), _ptr(k["head_w"]), _ptr(k["head_b"]), _ptr(k["prior"]), float(w.evidence_k),
+            _ptr(k["mpa"]), _ptr(k["head_w"]), _ptr(k["head_b"]), _ptr(k["prior"]), float(np.float32(w.evidence_k)),   # the interface takes kappa as a float
             _ptr(k["recall"]), _ptr(k["al"]), _ptr(k["be"]), _ptr(k["sw"]), _ptr(k["bs"]),
             int(k["bs"].shape[0]), float(w.prio_time_scale_s), _ptr(k["pen"]))
 

@@ -30,7 +30,9 @@ assert ROUND_DTYPE.itemsize == 64 and REQ_DTYPE.itemsize == 24
 
 EXPORTS = ["sp_create", "sp_destroy", "sp_last_error", "sp_load_profiles", "sp_default_options", "sp_set_options", "sp_set_clock",
            "sp_set_clocks", "sp_score", "sp_get_scores", "sp_schedule_round", "sp_get_requests", "sp_get_clocks",
-           "sp_reset", "sp_check", "sp_get_stats", "sp_run_host", "sp_score_static"]
+           "sp_reset", "sp_check", "sp_get_stats", "sp_run_host", "sp_score_static", "sp_schedule_split",
+           "sp_schedule_exhaustive", "sp_schedule_baseline", "sp_get_labels"]
+SP_BASE_MAXACC_EDF, SP_BASE_LO_EDF, SP_BASE_LO_PRIORITY = 0, 1, 2
 
 
 class SpError(RuntimeError):
@@ -99,6 +101,10 @@ def load_library():
     lib.sp_check.argtypes = [vp]
     lib.sp_get_stats.argtypes = [vp, C.POINTER(_Stats)]
     lib.sp_run_host.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp, vp, i32, vp, vp, i64, vp]
+    lib.sp_schedule_split.argtypes = [vp, vp, i64, vp]
+    lib.sp_schedule_exhaustive.argtypes = [vp, i32, vp, i64, vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+    lib.sp_schedule_baseline.argtypes = [vp, i32, vp, i64, vp]
+    lib.sp_get_labels.argtypes = [vp, i64, i64, vp]
     lib.sp_score_static.argtypes = [C.c_int, vp, C.POINTER(_StaticHead), i64, vp, vp, vp, vp, C.c_char_p, i32]
     for name in EXPORTS:
         if name not in ("sp_destroy", "sp_last_error", "sp_default_options"):
@@ -194,6 +200,26 @@ def sp_get_scores(ctx: int, first: int, n: int, acc=None, v=None) -> None:
 
 def sp_schedule_round(ctx: int, max_rounds: int, rounds_out=None, cap: int = 0, n_done=None) -> None:
     _ok(ctx, load_library().sp_schedule_round(ctx, int(max_rounds), _dev(rounds_out), int(cap), _dev(n_done)))
+
+
+def sp_schedule_split(ctx: int, rounds_out=None, cap: int = 0, n_done=None) -> None:
+    _ok(ctx, load_library().sp_schedule_split(ctx, _dev(rounds_out), int(cap), _dev(n_done)))
+
+
+def sp_schedule_exhaustive(ctx: int, split: bool, rounds_out=None, cap: int = 0, n_done=None):
+    """Returns (best total utility, number of solutions visited)."""
+    total, nsol = C.c_double(), C.c_int64()
+    _ok(ctx, load_library().sp_schedule_exhaustive(ctx, int(bool(split)), _dev(rounds_out), int(cap), _dev(n_done),
+                                                   C.byref(total), C.byref(nsol)))
+    return total.value, nsol.value
+
+
+def sp_schedule_baseline(ctx: int, policy: int, rounds_out=None, cap: int = 0, n_done=None) -> None:
+    _ok(ctx, load_library().sp_schedule_baseline(ctx, int(policy), _dev(rounds_out), int(cap), _dev(n_done)))
+
+
+def sp_get_labels(ctx: int, first: int, n: int, labels) -> None:
+    _ok(ctx, load_library().sp_get_labels(ctx, int(first), int(n), _dev(labels)))
 
 
 def sp_get_requests(ctx: int, first: int, n: int, out) -> None:

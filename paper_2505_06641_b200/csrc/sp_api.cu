@@ -15,6 +15,7 @@
 #include "sp_sched.cuh"
 #include "sp_sched_warp.cuh"
 #include "sp_presort.cuh"
+#include "sp_policies.cuh"
 
 using namespace sp;
 
@@ -68,6 +69,9 @@ struct sp_ctx {
     std::vector<FeatSeg> segs;
     std::vector<Buf> seg_copies;
     Buf t_app, t_arrival, t_deadline, a_cnt, a_cursor, a_gstart, r_id, r_dl, r_pw;
+    // policies decided on fp64 scores: labels, group tables, exhaustive search
+    Buf labels, g_key, g_start, g_head, g_count, exh_info, exh_total, exh_sol;
+    bool have_exact_all = false;
     // staging of sp_run_host
     Buf h_feats, h_app, h_arrival, h_deadline, h_instance, h_t0, h_loaded, h_rounds, h_ndone;
 };
@@ -133,6 +137,7 @@ void drop_table(sp_ctx *c) {
     c->have_table = false;
     c->sched_started = false;
     c->own_requests = false;
+    c->have_exact_all = false;
     c->tb.n = 0;
     c->segs.clear();
     for (Buf &b : c->seg_copies) release(b);     // cudaFree waits for kernels that may still read them
@@ -404,6 +409,75 @@ k_queue_regrow(InstState *state, int A, int64_t *qstart, const int32_t *add_cnt,
     }
 }
 
+// Sorts the n keys in the context's sort scratch with the whole GPU (bitonic network, see sp_presort.cuh).
+sp_status presort_network(sp_ctx *c, int64_t n) {
+    SortKey *keys = (SortKey *)c->sort_scratch.p;
+    const unsigned nblk = (unsigned)((n + kPresortChunk - 1) / kPresortChunk);
+    const size_t psm = (size_t)kPresortChunk * sizeof(SortKey);
+    SP_CUDA(c, cudaFuncSetAttribute(k_presort_local, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm));
+    k_presort_local<<<nblk, kPresortThreads, psm, c->stream>>>(keys, n, 2, kPresortChunk);
+    SP_TRY(launched(c, "k_presort_local"));
+    int64_t p2 = 1;
+    while (p2 < n) p2 <<= 1;
+    const int64_t n_pairs = p2 >> 1;
+    for (int64_t k = 2 * (int64_t)kPresortChunk; k <= p2; k <<= 1) {
+        for (int64_t j = k >> 1; j >= kPresortChunk; j >>= 1) {
+            k_presort_global<<<(unsigned)((n_pairs + 255) / 256), 256, 0, c->stream>>>(keys, n, k, j, n_pairs);
+            SP_TRY(launched(c, "k_presort_global"));
+        }
+        k_presort_local<<<nblk, kPresortThreads, psm, c->stream>>>(keys, n, k, k);
+        SP_TRY(launched(c, "k_presort_local"));
+    }
+    return SP_OK;
+}
+
+// Common start of the calls that schedule on fp64 scores: the table must be fresh and in snapshot mode; every request
+// gets its fp64 scores and label (one grid-wide pass, kept until the table changes); the group tables are sized.
+sp_status policy_prologue(sp_ctx *c, const char *who, GroupParams *gp, bool use_labels, sp_round_rec *rounds_out, int64_t cap,
+                          int32_t *n_done) {
+    if (!c->have_table) return fail(c, SP_ESTATE, "no scored requests");
+    if (c->opt.trace_mode) return fail(c, SP_ESTATE, std::string(who) + " works on a snapshot: trace mode is not supported");
+    if (c->sched_started) return fail(c, SP_ESTATE, std::string(who) + " needs a table no round has run on yet; call sp_reset and score again");
+    if (cap < 0) return fail(c, SP_EINVAL, "cap must be >= 0");
+    SP_CUDA(c, cudaSetDevice(c->device));
+    const DevProfiles &P = c->P;
+    const int64_t n = c->tb.n;
+    const size_t nn = (size_t)(n > 0 ? n : 1);
+    SP_TRY(ensure(c, c->labels, nn * 4));
+    SP_TRY(ensure(c, c->g_key, (nn + P.I) * 4));
+    SP_TRY(ensure(c, c->g_start, (nn + P.I) * 4));
+    SP_TRY(ensure(c, c->g_head, (nn + P.I) * 4));
+    SP_TRY(ensure(c, c->g_count, (size_t)P.I * 4));
+    if (!c->have_exact_all && n > 0) {
+        int warps = 8;
+        while (warps > 1 && (size_t)warps * P.C * 8 > 200 * 1024) warps >>= 1;
+        const size_t smem = (size_t)warps * P.C * 8;
+        SP_CUDA(c, cudaFuncSetAttribute(k_exact_all, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        int64_t blocks = (n + warps - 1) / warps;
+        if (blocks > (int64_t)c->n_sms * 8) blocks = (int64_t)c->n_sms * 8;
+        k_exact_all<<<(unsigned)blocks, warps * 32, smem, c->stream>>>(P, c->tb, (int32_t *)c->labels.p, (const int *)c->flags.p);
+        SP_TRY(launched(c, "k_exact_all"));
+        c->have_exact_all = true;
+    }
+    *gp = GroupParams{};
+    gp->P = P; gp->tb = c->tb; gp->state = (InstState *)c->state.p;
+    gp->labels = use_labels ? (const int32_t *)c->labels.p : nullptr;
+    gp->q_id = (int64_t *)c->q_id0.p; gp->q_dl = (int64_t *)c->q_dl0.p; gp->q_pw = (double *)c->q_pw0.p;
+    gp->keys = (SortKey *)c->sort_scratch.p;
+    gp->g_key = (int32_t *)c->g_key.p; gp->g_start = (int32_t *)c->g_start.p; gp->g_head = (int32_t *)c->g_head.p;
+    gp->g_count = (int32_t *)c->g_count.p;
+    gp->flags = (int *)c->flags.p; gp->stats = (unsigned long long *)c->stats.p;
+    gp->rounds_out = rounds_out; gp->cap = rounds_out ? cap : 0; gp->n_done = n_done;
+    gp->bmax = P.batch[P.nB - 1];
+    const int64_t per_inst = P.I > 1 ? (n + P.I - 1) / P.I * 2 : n;
+    int sort_cap = P.I > 1 ? 1024 : 4096;
+    while (sort_cap > 64 && sort_cap / 2 >= per_inst) sort_cap /= 2;
+    gp->sort_cap = sort_cap;
+    gp->presorted = 0;
+    c->sched_started = true;
+    return SP_OK;
+}
+
 }  // namespace
 
 // =================================================================================================
@@ -443,7 +517,8 @@ void sp_destroy(sp_ctx *c) {
                   &c->perm, &c->q_id0, &c->q_id1, &c->q_dl0, &c->q_dl1, &c->q_pw0, &c->q_pw1, &c->sort_scratch,
                   &c->h_feats, &c->h_app, &c->h_arrival, &c->h_deadline, &c->h_instance, &c->h_t0, &c->h_loaded,
                   &c->h_rounds, &c->h_ndone, &c->t_app, &c->t_arrival, &c->t_deadline, &c->a_cnt, &c->a_cursor,
-                  &c->a_gstart, &c->r_id, &c->r_dl, &c->r_pw};
+                  &c->a_gstart, &c->r_id, &c->r_dl, &c->r_pw, &c->labels, &c->g_key, &c->g_start, &c->g_head, &c->g_count,
+                  &c->exh_info, &c->exh_total, &c->exh_sol};
     for (Buf *b : all) release(*b);
     for (Buf &b : c->seg_copies) release(b);
     delete c;
@@ -874,31 +949,109 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
     }
     // One large snapshot instance: its keys are sorted by the whole GPU first (k_sched would use one block for it).
     if (P.I == 1 && !c->opt.trace_mode && !c->sched_started && max_rounds > 0 && c->tb.n > sort_cap && c->tb.n < ((int64_t)1 << 31)) {
-        const int64_t n = c->tb.n;
-        SortKey *keys = (SortKey *)c->sort_scratch.p;
-        k_presort_keys<<<(unsigned)((n + 255) / 256), 256, 0, c->stream>>>(c->tb, keys, n);
+        k_presort_keys<<<(unsigned)((c->tb.n + 255) / 256), 256, 0, c->stream>>>(c->tb, (SortKey *)c->sort_scratch.p, c->tb.n);
         SP_TRY(launched(c, "k_presort_keys"));
-        const unsigned nblk = (unsigned)((n + kPresortChunk - 1) / kPresortChunk);
-        const size_t psm = (size_t)kPresortChunk * sizeof(SortKey);
-        SP_CUDA(c, cudaFuncSetAttribute(k_presort_local, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm));
-        k_presort_local<<<nblk, kPresortThreads, psm, c->stream>>>(keys, n, 2, kPresortChunk);
-        SP_TRY(launched(c, "k_presort_local"));
-        int64_t p2 = 1;
-        while (p2 < n) p2 <<= 1;
-        const int64_t n_pairs = p2 >> 1;
-        for (int64_t k = 2 * (int64_t)kPresortChunk; k <= p2; k <<= 1) {
-            for (int64_t j = k >> 1; j >= kPresortChunk; j >>= 1) {
-                k_presort_global<<<(unsigned)((n_pairs + 255) / 256), 256, 0, c->stream>>>(keys, n, k, j, n_pairs);
-                SP_TRY(launched(c, "k_presort_global"));
-            }
-            k_presort_local<<<nblk, kPresortThreads, psm, c->stream>>>(keys, n, k, k);
-            SP_TRY(launched(c, "k_presort_local"));
-        }
+        SP_TRY(presort_network(c, c->tb.n));
         sp.presorted = 1;
     }
     if (max_rounds > 0) c->sched_started = true;
     sched_kernel<<<P.I, nt, L.end, c->stream>>>(sp);
     SP_TRY(launched(c, "k_sched"));
+    return mark(c, c->ev_sched);
+}
+
+sp_status sp_get_labels(sp_ctx *c, int64_t first, int64_t n, int32_t *labels) {
+    if (!c) return SP_EINVAL;
+    if (!c->have_table || !c->have_exact_all) return fail(c, SP_ESTATE, "labels exist after sp_schedule_split, sp_schedule_exhaustive or sp_schedule_baseline");
+    if (first < 0 || n < 0 || first + n > c->tb.n || (n && !labels)) return fail(c, SP_EINVAL, "request range out of bounds");
+    SP_CUDA(c, cudaSetDevice(c->device));
+    if (n) SP_CUDA(c, cudaMemcpyAsync(labels, (const int32_t *)c->labels.p + first, (size_t)n * 4, cudaMemcpyDeviceToDevice, c->stream));
+    return SP_OK;
+}
+
+sp_status sp_schedule_split(sp_ctx *c, sp_round_rec *rounds_out, int64_t cap, int32_t *n_done) {
+    if (!c) return SP_EINVAL;
+    GroupParams gp;
+    SP_TRY(policy_prologue(c, "sp_schedule_split", &gp, true, rounds_out, cap, n_done));
+    const DevProfiles &P = c->P;
+    if (P.I == 1 && c->tb.n > gp.sort_cap && c->tb.n < ((int64_t)1 << 31)) {
+        k_group_keys<<<(unsigned)((c->tb.n + 255) / 256), 256, 0, c->stream>>>(gp, c->tb.n);
+        SP_TRY(launched(c, "k_group_keys"));
+        SP_TRY(presort_network(c, c->tb.n));
+        gp.presorted = 1;
+    }
+    const int nt = P.I > 1 ? 128 : 1024;
+    const GroupSchedSmem L(gp.sort_cap, P.Mmax, gp.bmax, P.sumM, nt / 32);
+    if (L.end > 220 * 1024) return fail(c, SP_EINVAL, "models_per_app x largest batch size is too large for one block");
+    SP_CUDA(c, cudaFuncSetAttribute(k_sched_groups, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)L.end));
+    SP_TRY(mark(c, c->ev_sched));
+    k_sched_groups<<<P.I, nt, L.end, c->stream>>>(gp);
+    SP_TRY(launched(c, "k_sched_groups"));
+    return mark(c, c->ev_sched);
+}
+
+sp_status sp_schedule_exhaustive(sp_ctx *c, int32_t split, sp_round_rec *rounds_out, int64_t cap, int32_t *n_done,
+                                 double *total_out, int64_t *n_solutions_out) {
+    if (!c) return SP_EINVAL;
+    if (c->have_profiles && c->P.I != 1) return fail(c, SP_ESTATE, "the exhaustive branch is for single-instance contexts");
+    GroupParams gp;
+    SP_TRY(policy_prologue(c, "sp_schedule_exhaustive", &gp, split != 0, rounds_out, cap, n_done));
+    SP_TRY(ensure(c, c->exh_info, sizeof(ExhInfo)));
+    ExhInfo *info_d = (ExhInfo *)c->exh_info.p;
+    if (c->tb.n > gp.sort_cap && c->tb.n < ((int64_t)1 << 31)) {
+        k_group_keys<<<(unsigned)((c->tb.n + 255) / 256), 256, 0, c->stream>>>(gp, c->tb.n);
+        SP_TRY(launched(c, "k_group_keys"));
+        SP_TRY(presort_network(c, c->tb.n));
+        gp.presorted = 1;
+    }
+    const size_t psm = (size_t)gp.sort_cap * sizeof(SortKey);
+    SP_CUDA(c, cudaFuncSetAttribute(k_exh_prepare, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm));
+    SP_TRY(mark(c, c->ev_sched));
+    k_exh_prepare<<<1, 1024, psm, c->stream>>>(gp, info_d);
+    SP_TRY(launched(c, "k_exh_prepare"));
+    ExhInfo info;
+    SP_CUDA(c, cudaMemcpyAsync(&info, info_d, sizeof info, cudaMemcpyDeviceToHost, c->stream));
+    SP_CUDA(c, cudaStreamSynchronize(c->stream));
+    if (info.status != 0) {
+        c->sched_started = false;
+        return fail(c, SP_EINVAL, "the exhaustive branch takes at most 8 non-empty groups and 2^31 solutions (found " +
+                                      std::to_string(info.n_groups) + " groups)");
+    }
+    const int n_blocks = (int)((info.n_solutions + 255) / 256);
+    SP_TRY(ensure(c, c->exh_total, (size_t)(n_blocks > 0 ? n_blocks : 1) * 8));
+    SP_TRY(ensure(c, c->exh_sol, (size_t)(n_blocks > 0 ? n_blocks : 1) * 8));
+    if (n_blocks > 0) {
+        k_exh_search<<<n_blocks, 256, 0, c->stream>>>(gp, info_d, (double *)c->exh_total.p, (long long *)c->exh_sol.p);
+        SP_TRY(launched(c, "k_exh_search"));
+    }
+    k_exh_finish<<<1, 256, 0, c->stream>>>(gp, info_d, (const double *)c->exh_total.p, (const long long *)c->exh_sol.p, n_blocks);
+    SP_TRY(launched(c, "k_exh_finish"));
+    SP_TRY(mark(c, c->ev_sched));
+    SP_CUDA(c, cudaMemcpyAsync(&info, info_d, sizeof info, cudaMemcpyDeviceToHost, c->stream));
+    SP_CUDA(c, cudaStreamSynchronize(c->stream));
+    if (total_out) *total_out = info.best_total;
+    if (n_solutions_out) *n_solutions_out = info.n_solutions;
+    return SP_OK;
+}
+
+sp_status sp_schedule_baseline(sp_ctx *c, int32_t policy, sp_round_rec *rounds_out, int64_t cap, int32_t *n_done) {
+    if (!c) return SP_EINVAL;
+    if (policy < SP_BASE_MAXACC_EDF || policy > SP_BASE_LO_PRIORITY) return fail(c, SP_EINVAL, "policy must be one of SP_BASE_*");
+    BaselineParams bp;
+    SP_TRY(policy_prologue(c, "sp_schedule_baseline", &bp.gp, false, rounds_out, cap, n_done));
+    bp.policy = policy;
+    const DevProfiles &P = c->P;
+    if (P.I == 1 && c->tb.n > bp.gp.sort_cap && c->tb.n < ((int64_t)1 << 31)) {
+        k_baseline_keys<<<(unsigned)((c->tb.n + 255) / 256), 256, 0, c->stream>>>(bp, c->tb.n);
+        SP_TRY(launched(c, "k_baseline_keys"));
+        SP_TRY(presort_network(c, c->tb.n));
+        bp.gp.presorted = 1;
+    }
+    const size_t psm = (size_t)bp.gp.sort_cap * sizeof(SortKey);
+    SP_CUDA(c, cudaFuncSetAttribute(k_baseline, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)psm));
+    SP_TRY(mark(c, c->ev_sched));
+    k_baseline<<<P.I, P.I > 1 ? 128 : 1024, psm, c->stream>>>(bp);
+    SP_TRY(launched(c, "k_baseline"));
     return mark(c, c->ev_sched);
 }
 

@@ -121,15 +121,16 @@ __device__ __forceinline__ double block_sum(double v, double *red) {
 }
 
 // fp64 re-scoring of one request by one warp, written to acc64 / v64.  Plain definition of Section 4.1 /
-// Eq. 9 / Eq. 12 with separate multiplies and adds (no fused multiply-add).
-__device__ void exact_row(const SchedParams &sp, int inst, int64_t id, double *zrow) {
-    const DevProfiles &P = sp.P;
+// Eq. 9 / Eq. 12 with separate multiplies and adds (no fused multiply-add).  zrow: C doubles of scratch owned by the
+// warp.  label (optional): receives the request's data-aware sub-group (Section 4.3): the label c whose posterior
+// theta_c exceeds one half, or -1 when none does.
+__device__ void exact_row_core(const DevProfiles &P, const DevTable &tb, int inst, int64_t id, double *zrow, int32_t *label) {
     const int lane = threadIdx.x & 31;
-    const int a = sp.tb.app[id];
+    const int a = tb.app[id];
     const int64_t head = (int64_t)inst * P.A + a;
     const int C = P.C, D = P.D;
     int64_t frow;
-    const void *fmat = feat_matrix(sp.tb, id, frow);
+    const void *fmat = feat_matrix(tb, id, frow);
     for (int c0 = 0; c0 < C; c0 += 32) {
         const int c = c0 + lane;
         double z = c < C ? (double)P.bias[head * C + c] : 0.0;
@@ -150,17 +151,22 @@ __device__ void exact_row(const SchedParams &sp, int inst, int64_t id, double *z
     for (int o = 16; o >= 1; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     __syncwarp();
     double asum = 0.0;
-    if (P.prior) asum = (double)P.prior_sum[head];   // refined below in fp64
     if (P.prior) {
         double t = 0.0;
         for (int c = lane; c < C; c += 32) t += (double)P.prior[head * C + c];
         for (int o = 16; o >= 1; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
         asum = t;
     }
+    int lab = -1;
     for (int c = lane; c < C; c += 32) {
         double th = zrow[c] / s;
         if (P.prior) th = ((double)P.prior[head * C + c] + (double)P.kappa * th) / (asum + (double)P.kappa);
         zrow[c] = th;
+        if (th > 0.5) lab = c;
+    }
+    if (label) {
+        for (int o = 16; o >= 1; o >>= 1) lab = max(lab, __shfl_xor_sync(0xffffffffu, lab, o));
+        if (lane == 0) *label = lab;
     }
     __syncwarp();
     const int m0 = P.mfirst[a], M = P.mfirst[a + 1] - m0;
@@ -181,12 +187,16 @@ __device__ void exact_row(const SchedParams &sp, int inst, int64_t id, double *z
     for (int j = 0; j < kMaxModelsPerApp; ++j)
         if (j < M) var += (accv[j] - mean) * (accv[j] - mean);
     if (lane == 0) {
-        for (int j = 0; j < P.Mmax; ++j) sp.tb.acc64[id * P.Mmax + j] = j < M ? accv[j] : 0.0;
-        sp.tb.v64[id] = 1.0 + var / (double)M;
+        for (int j = 0; j < P.Mmax; ++j) tb.acc64[id * P.Mmax + j] = j < M ? accv[j] : 0.0;
+        tb.v64[id] = 1.0 + var / (double)M;
         __threadfence_block();
-        sp.tb.exact[id] = 1;
+        tb.exact[id] = 1;
     }
     __syncwarp();
+}
+
+__device__ __forceinline__ void exact_row(const SchedParams &sp, int inst, int64_t id, double *zrow) {
+    exact_row_core(sp.P, sp.tb, inst, id, zrow, nullptr);
 }
 
 // Re-scores (if not done before) the requests at queue positions [k0, k1) of one queue buffer.
