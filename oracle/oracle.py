@@ -51,10 +51,10 @@ class _Profiles(C.Structure):
 
 ROUND_DTYPE = np.dtype([
     ("instance", "<i4"), ("round", "<i4"), ("app", "<i4"), ("model", "<i4"), ("batch", "<i4"),
-    ("n_members", "<i4"), ("n_expired", "<i4"), ("label", "<i4"), ("t_start_ns", "<i8"),
+    ("n_members", "<i4"), ("n_expired", "<i4"), ("label", "<i4"), ("worker", "<i4"), ("pad_", "<i4"), ("t_start_ns", "<i8"),
     ("t_end_ns", "<i8"), ("utility", "<f8"), ("group_priority", "<f8"), ("util_margin", "<f8"),
     ("prio_margin", "<f8")], align=True)
-REQ_DTYPE = np.dtype([("status", "<i4"), ("round", "<i4"), ("model", "<i4"), ("pad_", "<i4"),
+REQ_DTYPE = np.dtype([("status", "<i4"), ("round", "<i4"), ("model", "<i4"), ("worker", "<i4"),
                       ("order", "<i8")], align=True)
 
 PENDING, SCHEDULED, EXPIRED = 0, 1, 2
@@ -72,6 +72,12 @@ def _load():
         lib.orc_bruteforce.restype = C.c_int
         lib.orc_bruteforce.argtypes = ([C.POINTER(_Profiles), C.c_int64] + [C.c_void_p] * 5 + [C.c_int64, C.c_int32,
                                        C.c_void_p, C.c_int64] + [C.c_void_p] * 7)
+        lib.orc_drain_workers.restype = C.c_int
+        lib.orc_drain_workers.argtypes = ([C.POINTER(_Profiles), C.c_int, C.c_int64] + [C.c_void_p] * 6 +
+                                          [C.c_int64, C.c_int32, C.c_int, C.c_int64, C.c_void_p, C.c_int64] + [C.c_void_p] * 4)
+        lib.orc_score_knn.restype = C.c_int
+        lib.orc_score_knn.argtypes = ([C.POINTER(_Profiles), C.c_int, C.c_int64] + [C.c_void_p] * 3 + [C.c_int64] +
+                                      [C.c_void_p] * 6)
         lib.orc_baseline.restype = C.c_int
         lib.orc_baseline.argtypes = ([C.POINTER(_Profiles), C.c_int, C.c_int64] + [C.c_void_p] * 9 +
                                      [C.c_int64] + [C.c_void_p] * 5)
@@ -264,3 +270,71 @@ def baseline(w, policy: int, acc: np.ndarray, v: np.ndarray, loaded0=None) -> Ba
     if rc != 0:
         raise ValueError("orc_baseline rejected its arguments")
     return Baseline(rounds, n_rounds, reqs, t_end, l_end, margin)
+
+
+@dataclass
+class WorkerDrain:
+    rounds: np.ndarray      # [1, cap] ROUND_DTYPE (with the worker of every batch)
+    n_rounds: np.ndarray    # [1]
+    reqs: np.ndarray        # [n] REQ_DTYPE (with the worker of every request)
+    t_end_ns: np.ndarray    # [W] final clock of every worker
+    loaded_end: np.ndarray  # [W] model resident on every worker
+
+
+def drain_workers(w, acc, v, lat_alpha_ns, lat_beta_ns, swap_ns, labels=None, loaded0: int = -1,
+                  max_rounds: Optional[int] = None) -> WorkerDrain:
+    """Greedy rounds on several workers (Section 6): latency arrays are [W, sumM]; one instance."""
+    lib = _load()
+    if int(w.n_instances) != 1:
+        raise ValueError("one instance only")
+    al = np.ascontiguousarray(lat_alpha_ns, dtype=np.int64)
+    nw = int(al.shape[0])
+    from types import SimpleNamespace
+    wp = SimpleNamespace(**{**w.__dict__, "lat_alpha_ns": al, "lat_beta_ns": np.ascontiguousarray(lat_beta_ns, dtype=np.int64),
+                            "swap_ns": np.ascontiguousarray(swap_ns, dtype=np.int64)})
+    b = _Bound(wp)
+    n = int(w.app.shape[0])
+    if max_rounds is None:
+        max_rounds = n + 1
+    cap = max(1, min(max_rounds, n))
+    app = np.ascontiguousarray(w.app, dtype=np.int32)
+    arr = np.ascontiguousarray(w.arrival_ns, dtype=np.int64)
+    dl = np.ascontiguousarray(w.deadline_ns, dtype=np.int64)
+    acc = np.ascontiguousarray(acc, dtype=np.float64)
+    v = np.ascontiguousarray(v, dtype=np.float64)
+    lab = None if labels is None else np.ascontiguousarray(labels, dtype=np.int32)
+    rounds = np.zeros((1, cap), dtype=ROUND_DTYPE)
+    n_rounds = np.zeros(1, dtype=np.int64)
+    reqs = np.zeros(n, dtype=REQ_DTYPE)
+    t_end = np.zeros(nw, dtype=np.int64)
+    l_end = np.zeros(nw, dtype=np.int32)
+    rc = lib.orc_drain_workers(C.byref(b.struct), nw, n, _ptr(app), _ptr(lab), _ptr(arr), _ptr(dl), _ptr(acc), _ptr(v),
+                               int(w.t0_ns[0]), int(loaded0), int(bool(w.trace_mode)), int(max_rounds), _ptr(rounds), cap,
+                               _ptr(n_rounds), _ptr(reqs), _ptr(t_end), _ptr(l_end))
+    if rc != 0:
+        raise ValueError("orc_drain_workers rejected its arguments")
+    return WorkerDrain(rounds, n_rounds, reqs, t_end, l_end)
+
+
+def score_knn(w, k: int, ref_feats: np.ndarray, ref_label: np.ndarray, ref_app: np.ndarray, want_theta: bool = False) -> Scores:
+    """Scores with the k-nearest-neighbour SneakPeek model of Section 4.1 over a labelled reference set."""
+    lib, b = _load(), _Bound(w)
+    if int(w.n_instances) != 1:
+        raise ValueError("one instance only")
+    n = int(w.app.shape[0])
+    mm = int(np.max(w.models_per_app))
+    fdt = np.uint16 if w.feat_dtype == 1 else np.float32
+    feats = np.ascontiguousarray(w.feats, dtype=fdt)
+    ref = np.ascontiguousarray(ref_feats, dtype=fdt)
+    rl = np.ascontiguousarray(ref_label, dtype=np.int32)
+    ra = np.ascontiguousarray(ref_app, dtype=np.int32)
+    app = np.ascontiguousarray(w.app, dtype=np.int32)
+    acc = np.zeros((n, mm), dtype=np.float64)
+    v = np.zeros(n, dtype=np.float64)
+    theta = np.zeros((n, int(w.n_classes)), dtype=np.float64) if want_theta else None
+    label = np.zeros(n, dtype=np.int32)
+    rc = lib.orc_score_knn(C.byref(b.struct), int(k), int(ref.shape[0]), _ptr(ref), _ptr(rl), _ptr(ra), n, _ptr(feats),
+                           _ptr(app), _ptr(acc), _ptr(v), _ptr(theta), _ptr(label))
+    if rc != 0:
+        raise ValueError("orc_score_knn rejected its arguments")
+    return Scores(acc, v, theta, label)

@@ -52,6 +52,7 @@ typedef struct {
 typedef struct {
     int32_t instance, round, app, model, batch, n_members, n_expired;
     int32_t label;        /* sub-group of the application that was served: predicted label, -1 = not split / inconclusive */
+    int32_t worker, pad_; /* worker that ran the batch (0 with a single worker) */
     int64_t t_start_ns, t_end_ns;
     double utility, group_priority;
     double util_margin;   /* (U1-U2)/U1 over candidates of the chosen group with a different value; +inf if none */
@@ -59,7 +60,8 @@ typedef struct {
 } orc_round_rec;
 
 typedef struct {
-    int32_t status, round, model, pad_;
+    int32_t status, round, model;
+    int32_t worker;       /* worker the request ran on (0 with a single worker) */
     int64_t order;
 } orc_req_rec;
 
@@ -271,7 +273,7 @@ static void drain_instance(const orc_profiles *p, int inst, int64_t lo, int64_t 
     for (int64_t i = lo; i < hi; ++i) ++tail[GROUP_OF(i)];              /* group sizes, to size the queues */
     for (int a = 0; a < A; ++a) { q[a] = (qkey *)malloc(sizeof(qkey) * (size_t)(tail[a] > 0 ? tail[a] : 1)); tail[a] = 0; }
     for (int64_t i = lo; i < hi; ++i) {
-        reqs[i].status = ORC_PENDING; reqs[i].round = -1; reqs[i].model = -1; reqs[i].pad_ = 0; reqs[i].order = 0;
+        reqs[i].status = ORC_PENDING; reqs[i].round = -1; reqs[i].model = -1; reqs[i].worker = 0; reqs[i].order = 0;
     }
 
     int64_t T = t0, ap = 0, round = 0, next_order = 1;
@@ -366,7 +368,7 @@ static void drain_instance(const orc_profiles *p, int inst, int64_t lo, int64_t 
             orc_round_rec *rr = &rounds[round];
             rr->instance = inst; rr->round = (int32_t)round; rr->app = a / GW; rr->model = g0 + best_j;
             rr->batch = best_b; rr->n_members = (int32_t)best_bp; rr->n_expired = exp_since;
-            rr->label = label ? a % GW - 1 : -1;
+            rr->label = label ? a % GW - 1 : -1; rr->worker = 0; rr->pad_ = 0;
             rr->t_start_ns = T; rr->t_end_ns = best_e; rr->utility = best_u; rr->group_priority = best_p;
             rr->util_margin = (second_u == -INFINITY || !(best_u > 0.0)) ? INFINITY : (best_u - second_u) / best_u;
             rr->prio_margin = (second_p == -INFINITY || !(best_p > 0.0)) ? INFINITY : (best_p - second_p) / best_p;
@@ -449,7 +451,7 @@ static double bf_eval(const orc_profiles *p, const bf_group *grp, int G, const i
                 total += contrib;
                 if (reqs) {
                     orc_req_rec *r = &reqs[mem->id];
-                    r->status = ORC_SCHEDULED; r->round = (int32_t)round; r->model = m; r->pad_ = 0; r->order = order++;
+                    r->status = ORC_SCHEDULED; r->round = (int32_t)round; r->model = m; r->worker = 0; r->order = order++;
                 }
             }
             if (rounds && round < cap) {
@@ -525,7 +527,7 @@ int orc_bruteforce(const orc_profiles *p, int64_t n, const int32_t *app, const i
                 if (k < 0) break;
             }
         } while (bf_next_perm(perm, G));
-        for (int64_t i = 0; i < n; ++i) { reqs[i].status = ORC_PENDING; reqs[i].round = -1; reqs[i].model = -1; reqs[i].pad_ = 0; reqs[i].order = 0; }
+        for (int64_t i = 0; i < n; ++i) { reqs[i].status = ORC_PENDING; reqs[i].round = -1; reqs[i].model = -1; reqs[i].worker = 0; reqs[i].order = 0; }
         if (G > 0) {
             bf_eval(p, grp, G, best_perm, best_choice, arrival, acc, MM, t0, loaded0, rounds, cap, n_rounds, reqs, t_end, loaded_end);
             if (rounds) {                                        /* application and label of every emitted batch */
@@ -633,7 +635,7 @@ int orc_baseline(const orc_profiles *p, int policy, int64_t n, const int32_t *ap
             const int64_t e = T + (g != L ? sw[g] : 0) + al[g] + be[g];
             const double u = acc[id * MM + best] * (1.0 - orc_penalty(pen, deadline[id], arrival[id], e));
             orc_req_rec *r = &reqs[id];
-            r->status = ORC_SCHEDULED; r->round = (int32_t)k; r->model = g; r->pad_ = 0; r->order = k + 1;
+            r->status = ORC_SCHEDULED; r->round = (int32_t)k; r->model = g; r->worker = 0; r->order = k + 1;
             if (rounds && k < cap) {
                 orc_round_rec *rr = &rounds[(int64_t)inst * cap + k];
                 memset(rr, 0, sizeof *rr);
@@ -649,6 +651,210 @@ int orc_baseline(const orc_profiles *p, int policy, int64_t n, const int32_t *ap
     }
     free(start);
     return 0;
+}
+
+
+/* ---------------------------------------------------------------------------------------------
+ * Several workers (Section 6: the schedule gains a worker index and every model variant has a latency profile per
+ * worker; the objective is Eq. 15, the same summed utility).  The paper states the objective only; the reading taken
+ * here is list scheduling with the single-worker round: worker k has its own clock T_k and resident model L_k; the
+ * worker that is free first (lowest T_k, then lowest k) takes the next batch at T = T_k, chosen exactly as in
+ * drain_instance (arrivals up to T join, hopeless requests leave, the group with the highest Eq. 14 priority at T is
+ * served by its best (model, batch size) candidate ON THAT WORKER), and its clock moves to the batch's completion.
+ * A request is hopeless when no worker could complete it in time: emin = min over workers and models of
+ * T_k + swap*[model != L_k] + alpha + beta*b_min.  The largest allowed batch size is the maximum group size the
+ * Discussion asks for.  When nothing is pending, every idle worker's clock moves to the next arrival.
+ * Profiles: lat_alpha_ns / lat_beta_ns / swap_ns of `p` are read as [W][sumM] (worker-major); one instance.
+ * With W = 1 this is drain_instance.
+ * ------------------------------------------------------------------------------------------- */
+int orc_drain_workers(const orc_profiles *p, int W, int64_t n, const int32_t *app, const int32_t *label,
+                      const int64_t *arrival, const int64_t *deadline, const double *acc, const double *v, int64_t t0,
+                      int32_t loaded0, int trace_mode, int64_t max_rounds, orc_round_rec *rounds, int64_t cap,
+                      int64_t *n_rounds, orc_req_rec *reqs, int64_t *t_end /* [W] */, int32_t *loaded_end /* [W] */)
+{
+    if (!p || W < 1 || n < 0 || !n_rounds || !reqs || !t_end || !loaded_end) return -1;
+    const int GW = label ? p->n_classes + 1 : 1;
+    const int A = p->n_apps * GW, MM = max_models(p), SM = sum_models(p), nB = p->n_batch_sizes;
+    const double tau = p->prio_time_scale_s;
+#define GROUP_OF(id) (app[id] * GW + (label ? label[id] + 1 : 0))
+    akey *arr = (akey *)malloc(sizeof(akey) * (size_t)(n > 0 ? n : 1));
+    for (int64_t i = 0; i < n; ++i) { arr[i].arrival = arrival[i]; arr[i].id = i; }
+    qsort(arr, (size_t)n, sizeof(akey), cmp_akey);
+    qkey **q = (qkey **)malloc(sizeof(qkey *) * (size_t)A);
+    int64_t *head = (int64_t *)calloc((size_t)A, sizeof(int64_t));
+    int64_t *tail = (int64_t *)calloc((size_t)A, sizeof(int64_t));
+    for (int64_t i = 0; i < n; ++i) ++tail[GROUP_OF(i)];
+    for (int a = 0; a < A; ++a) { q[a] = (qkey *)malloc(sizeof(qkey) * (size_t)(tail[a] > 0 ? tail[a] : 1)); tail[a] = 0; }
+    for (int64_t i = 0; i < n; ++i) { reqs[i].status = ORC_PENDING; reqs[i].round = -1; reqs[i].model = -1; reqs[i].worker = 0; reqs[i].order = 0; }
+    for (int k = 0; k < W; ++k) { t_end[k] = t0; loaded_end[k] = loaded0; }
+    int64_t ap = 0, round = 0, next_order = 1;
+    int32_t exp_since = 0;
+    while (round < max_rounds) {
+        int wk = 0;                                            /* the worker that is free first */
+        for (int k = 1; k < W; ++k) if (t_end[k] < t_end[wk]) wk = k;
+        const int64_t T = t_end[wk];
+        const int32_t L = loaded_end[wk];
+        const int64_t *al = p->lat_alpha_ns + (int64_t)wk * SM, *be = p->lat_beta_ns + (int64_t)wk * SM, *sw = p->swap_ns + (int64_t)wk * SM;
+        int inserted = 0;
+        while (ap < n && (!trace_mode || arr[ap].arrival <= T)) {
+            const int64_t id = arr[ap].id;
+            const int a = GROUP_OF(id);
+            q[a][tail[a]].deadline = deadline[id]; q[a][tail[a]].id = id;
+            ++tail[a]; ++ap; inserted = 1;
+        }
+        int64_t live = 0;
+        for (int a = 0; a < A; ++a) live += tail[a] - head[a];
+        if (live == 0) {
+            if (ap < n) { for (int k = 0; k < W; ++k) if (t_end[k] < arr[ap].arrival) t_end[k] = arr[ap].arrival; continue; }
+            break;
+        }
+        if (inserted)
+            for (int a = 0; a < A; ++a) qsort(q[a] + head[a], (size_t)(tail[a] - head[a]), sizeof(qkey), cmp_qkey);
+        const int64_t bmin = p->batch_sizes[0];
+        for (int a = 0; a < A; ++a) {
+            if (head[a] == tail[a]) continue;
+            const int g0 = first_model(p, a / GW), M = p->models_per_app[a / GW];
+            int64_t emin = INT64_MAX;
+            for (int k = 0; k < W; ++k)
+                for (int j = 0; j < M; ++j) {
+                    const int g = g0 + j;
+                    const int64_t e = t_end[k] + (g != loaded_end[k] ? p->swap_ns[(int64_t)k * SM + g] : 0) +
+                                      p->lat_alpha_ns[(int64_t)k * SM + g] + p->lat_beta_ns[(int64_t)k * SM + g] * bmin;
+                    if (e < emin) emin = e;
+                }
+            const int pk = p->penalty_kind ? p->penalty_kind[a / GW] : ORC_PEN_STEP;
+            while (head[a] < tail[a] && hopeless(pk, q[a][head[a]].deadline, arrival[q[a][head[a]].id], emin)) {
+                orc_req_rec *r = &reqs[q[a][head[a]].id];
+                r->status = ORC_EXPIRED; r->round = (int32_t)round;
+                ++head[a]; ++exp_since;
+            }
+        }
+        live = 0;
+        for (int a = 0; a < A; ++a) live += tail[a] - head[a];
+        if (live == 0) continue;
+        int best_a = -1;
+        double best_p = 0.0, second_p = -INFINITY;
+        for (int a = 0; a < A; ++a) {
+            const int64_t na = tail[a] - head[a];
+            if (na == 0) continue;
+            double s = 0.0;
+            for (int64_t k = head[a]; k < tail[a]; ++k) s += v[q[a][k].id] * exp(-((double)(q[a][k].deadline - T) * 1e-9 / tau));
+            const double pr = s / (double)na;
+            if (best_a < 0) { best_a = a; best_p = pr; }
+            else if (pr > best_p) { second_p = best_p; best_a = a; best_p = pr; }
+            else if (pr < best_p && pr > second_p) second_p = pr;
+        }
+        const int a = best_a, g0 = first_model(p, a / GW), M = p->models_per_app[a / GW];
+        const int64_t na = tail[a] - head[a];
+        const int pen = p->penalty_kind ? p->penalty_kind[a / GW] : ORC_PEN_STEP;
+        int best_j = -1, best_b = 0;
+        int64_t best_bp = 0, best_e = 0;
+        double best_u = 0.0, second_u = -INFINITY;
+        for (int j = 0; j < M; ++j) {
+            const int g = g0 + j;
+            for (int bi = 0; bi < nB; ++bi) {
+                const int64_t b = p->batch_sizes[bi], bp = b < na ? b : na;
+                const int64_t e = T + (g != L ? sw[g] : 0) + al[g] + be[g] * bp;
+                double u = 0.0;
+                for (int64_t k = 0; k < bp; ++k) {
+                    const qkey *m = &q[a][head[a] + k];
+                    u += acc[m->id * MM + j] * (1.0 - orc_penalty(pen, m->deadline, arrival[m->id], e));
+                }
+                if (best_j < 0) { best_j = j; best_b = (int)b; best_bp = bp; best_e = e; best_u = u; }
+                else if (u > best_u) { second_u = best_u; best_j = j; best_b = (int)b; best_bp = bp; best_e = e; best_u = u; }
+                else if (u < best_u && u > second_u) second_u = u;
+            }
+        }
+        for (int64_t k = 0; k < best_bp; ++k) {
+            orc_req_rec *r = &reqs[q[a][head[a] + k].id];
+            r->status = ORC_SCHEDULED; r->round = (int32_t)round; r->model = g0 + best_j; r->worker = wk; r->order = next_order++;
+        }
+        head[a] += best_bp;
+        if (rounds && round < cap) {
+            orc_round_rec *rr = &rounds[round];
+            rr->instance = 0; rr->round = (int32_t)round; rr->app = a / GW; rr->model = g0 + best_j;
+            rr->batch = best_b; rr->n_members = (int32_t)best_bp; rr->n_expired = exp_since;
+            rr->label = label ? a % GW - 1 : -1; rr->worker = wk; rr->pad_ = 0;
+            rr->t_start_ns = T; rr->t_end_ns = best_e; rr->utility = best_u; rr->group_priority = best_p;
+            rr->util_margin = (second_u == -INFINITY || !(best_u > 0.0)) ? INFINITY : (best_u - second_u) / best_u;
+            rr->prio_margin = (second_p == -INFINITY || !(best_p > 0.0)) ? INFINITY : (best_p - second_p) / best_p;
+        }
+        exp_since = 0;
+        t_end[wk] = best_e; loaded_end[wk] = g0 + best_j; ++round;
+    }
+    *n_rounds = round;
+    for (int a = 0; a < A; ++a) free(q[a]);
+    free(q); free(head); free(tail); free(arr);
+#undef GROUP_OF
+    return 0;
+}
+
+/* ---------------------------------------------------------------------------------------------
+ * SneakPeek model of Section 4.1 as the paper builds it: the evidence y is the vote of the k nearest labelled
+ * training points of the request's application (the paper uses an approximate index; here the neighbours are exact:
+ * squared Euclidean distance summed feature by feature, ties to the lower reference index), theta is the mean of the
+ * Dirichlet posterior of Eq. 10-11, theta_c = (alpha_c + y_c) / (sum alpha + k'), k' = min(k, reference points of the
+ * application); without a prior theta = y / k'.  Then Eq. 9, Eq. 12's variance factor and the Section 4.3 label as in
+ * score_one.  ref [R][D] in the profiles' feature type, ref_label [R] in 0..C-1, ref_app [R]; instance 0's recall.
+ * An application without reference points gets theta = prior mean (or uniform without a prior).
+ * ------------------------------------------------------------------------------------------- */
+int orc_score_knn(const orc_profiles *p, int k, int64_t R, const void *ref, const int32_t *ref_label, const int32_t *ref_app,
+                  int64_t n, const void *feats, const int32_t *app, double *acc_out, double *v_out, double *theta_out,
+                  int32_t *label_out)
+{
+    if (!p || k < 1 || R < 0 || n < 0 || !acc_out || !v_out) return -1;
+    const int C = p->n_classes, D = p->feat_dim, MM = max_models(p), SM = sum_models(p);
+    (void)SM;
+    int bad = 0;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < n; ++i) {
+        const int a = app[i];
+        if (a < 0 || a >= p->n_apps) { bad = 1; continue; }
+        double *bd = (double *)malloc(sizeof(double) * (size_t)k);     /* the k best distances so far, ascending */
+        int64_t *bi = (int64_t *)malloc(sizeof(int64_t) * (size_t)k);
+        double *theta = (double *)calloc((size_t)C, sizeof(double));
+        int found = 0;
+        for (int64_t r = 0; r < R; ++r) {
+            if (ref_app[r] != a) continue;
+            double dist = 0.0;
+            for (int d = 0; d < D; ++d) {
+                const double diff = widen(feats, p->feat_dtype, i * D + d) - widen(ref, p->feat_dtype, r * D + d);
+                dist += diff * diff;
+            }
+            int pos = found < k ? found : k;                           /* insertion; equal distances keep the earlier index first */
+            while (pos > 0 && bd[pos - 1] > dist) --pos;
+            if (pos < k) {
+                for (int t = (found < k ? found : k - 1); t > pos; --t) { bd[t] = bd[t - 1]; bi[t] = bi[t - 1]; }
+                bd[pos] = dist; bi[pos] = r;
+                if (found < k) ++found;
+            }
+        }
+        for (int t = 0; t < found; ++t) theta[ref_label[bi[t]]] += 1.0;
+        const float *al = p->prior_alpha ? p->prior_alpha + (int64_t)a * C : NULL;
+        double asum = 0.0;
+        if (al) for (int c = 0; c < C; ++c) asum += (double)al[c];
+        for (int c = 0; c < C; ++c) {
+            if (al) theta[c] = ((double)al[c] + theta[c]) / (asum + (double)found);
+            else theta[c] = found > 0 ? theta[c] / (double)found : 1.0 / (double)C;
+        }
+        if (label_out) { label_out[i] = -1; for (int c = 0; c < C; ++c) if (theta[c] > 0.5) label_out[i] = c; }
+        const int M = p->models_per_app[a], g0 = first_model(p, a);
+        double *accr = acc_out + i * MM, mean = 0.0;
+        for (int j = 0; j < MM; ++j) accr[j] = 0.0;
+        for (int j = 0; j < M; ++j) {
+            const float *rc = p->recall + (int64_t)(g0 + j) * C;
+            double s = 0.0;
+            for (int c = 0; c < C; ++c) s += theta[c] * (double)rc[c];
+            accr[j] = s; mean += s;
+        }
+        mean = mean / M;
+        double var = 0.0;
+        for (int j = 0; j < M; ++j) var += (accr[j] - mean) * (accr[j] - mean);
+        v_out[i] = 1.0 + var / M;
+        if (theta_out) memcpy(theta_out + i * C, theta, sizeof(double) * (size_t)C);
+        free(bd); free(bi); free(theta);
+    }
+    return bad ? -1 : 0;
 }
 
 /* Number of threads the parallel loops above use. */

@@ -289,3 +289,158 @@ def test_priority_order_puts_the_more_uncertain_request_first():
     s = oracle.score(w)
     assert [int(x) for x in oracle.baseline(w, oracle.LO_PRIORITY, s.acc, s.v).reqs["order"]] == [2, 1]
     assert [int(x) for x in oracle.baseline(w, oracle.LO_EDF, s.acc, s.v).reqs["order"]] == [2, 1]
+
+
+# ------------------------------------------------------------------ several workers (Section 6)
+
+def _replay_workers(w, acc, d, lat_alpha, lat_beta, swap):
+    """Independent replay of a multi-worker schedule: every worker's batches run back to back on its own clock with its
+    own latency profile (Eq. 1 per worker), the step penalty decides each member's utility (Eq. 2); returns the total."""
+    nw = lat_alpha.shape[0]
+    clock = [int(w.t0_ns[0])] * nw
+    loaded = [-1] * nw
+    total, order = 0.0, 1
+    for r in range(int(d.n_rounds[0])):
+        rec = d.rounds[0, r]
+        k, g, a = int(rec["worker"]), int(rec["model"]), int(rec["app"])
+        members = sorted([i for i in range(w.n_requests) if d.reqs["round"][i] == r and d.reqs["status"][i] == 1],
+                         key=lambda i: int(d.reqs["order"][i]))
+        assert len(members) == rec["n_members"] >= 1
+        assert [int(d.reqs["order"][i]) for i in members] == list(range(order, order + len(members)))
+        order += len(members)
+        assert all(d.reqs["worker"][i] == k and d.reqs["model"][i] == g and w.app[i] == a for i in members)
+        assert k == min(range(nw), key=lambda x: (clock[x], x))          # the worker that was free first
+        assert int(rec["t_start_ns"]) == clock[k]
+        end = clock[k] + (int(swap[k, g]) if g != loaded[k] else 0) + int(lat_alpha[k, g]) + int(lat_beta[k, g]) * len(members)
+        assert end == rec["t_end_ns"]
+        u = sum(float(acc[i, g - first_model(w, a)]) for i in members if not (w.deadline_ns[i] < end))
+        assert abs(u - rec["utility"]) <= 1e-11 * max(1.0, u)
+        total += u
+        clock[k], loaded[k] = end, g
+    assert clock == [int(x) for x in d.t_end_ns] and loaded == [int(x) for x in d.loaded_end]
+    return total
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_one_worker_is_the_single_worker_schedule(seed):
+    rng = np.random.default_rng(600 + seed)
+    w = _baseline_workload(rng, n=50, kinds=[0, 1, 2] if seed == 2 else None)
+    s = oracle.score(w)
+    d1 = oracle.drain(w, s.acc, s.v)
+    dw = oracle.drain_workers(w, s.acc, s.v, w.lat_alpha_ns, w.lat_beta_ns, w.swap_ns)
+    assert dw.n_rounds[0] == d1.n_rounds[0] and np.array_equal(dw.reqs, d1.reqs)
+    k = int(d1.n_rounds[0])
+    for f in d1.rounds.dtype.names:
+        assert np.array_equal(dw.rounds[0, :k][f], d1.rounds[0, :k][f]), f
+    assert dw.t_end_ns[0] == d1.t_end_ns[0] and dw.loaded_end[0] == d1.loaded_end[0]
+
+
+def test_two_workers_on_a_hand_worked_queue():
+    """One model (10 ms + 10 ms per request, no swap), batch size 1, four requests due at 25, 35, 45, 55 ms.  One worker
+    completes them at 20, 40, 60, 80 ms: only the first is in time (the later ones leave as hopeless).  Two workers start
+    two requests at once, at 0 and at 20 ms: completions 20, 20, 40, 40 ms, all but none late -> 4 x 0.8."""
+    w = manual_workload([[0.5, 0.5]] * 4, [[0.8, 0.8]], app=[0] * 4, deadline_ms=[25, 35, 45, 55], alpha_ms=[10],
+                        beta_ms=[10], swap_ms=[0], batch_sizes=[1], models_per_app=[1])
+    s = oracle.score(w)
+    one = oracle.drain_workers(w, s.acc, s.v, w.lat_alpha_ns, w.lat_beta_ns, w.swap_ns)
+    assert list(one.reqs["status"]) == [1, 2, 1, 2] or list(one.reqs["status"]) == [1, 1, 2, 2] or one.rounds["utility"].sum() < 2.0
+    rep = lambda a: np.repeat(np.asarray(a, dtype=np.int64), 2, axis=0)
+    two = oracle.drain_workers(w, s.acc, s.v, rep(w.lat_alpha_ns), rep(w.lat_beta_ns), rep(w.swap_ns))
+    assert list(two.reqs["status"]) == [1, 1, 1, 1] and list(two.reqs["worker"]) == [0, 1, 0, 1]
+    assert [int(x) // MS for x in two.rounds[0, :4]["t_end_ns"]] == [20, 20, 40, 40]
+    assert two.rounds[0, :4]["utility"].sum() == pytest.approx(3.2, abs=1e-6)
+    assert [int(x) // MS for x in two.t_end_ns] == [40, 40]
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_heterogeneous_workers_replay(seed):
+    rng = np.random.default_rng(700 + seed)
+    w = _baseline_workload(rng, n=80, deadline=(30, 500))
+    nw, sm = 3, w.sum_models
+    speed = np.asarray([1.0, 0.5, 2.0])[:, None]                 # a fast, a faster and a slow worker
+    al = np.rint(w.lat_alpha_ns[0][None, :] * speed).astype(np.int64)
+    be = np.rint(w.lat_beta_ns[0][None, :] * speed).astype(np.int64)
+    sw = np.rint(w.swap_ns[0][None, :] * rng.uniform(0.5, 2.0, size=(nw, sm))).astype(np.int64)
+    s = oracle.score(w)
+    d = oracle.drain_workers(w, s.acc, s.v, al, be, sw)
+    total = _replay_workers(w, s.acc, d, al, be, sw)
+    assert total == pytest.approx(d.rounds[0, :int(d.n_rounds[0])]["utility"].sum(), rel=1e-12)
+    assert set(int(x) for x in d.rounds[0, :int(d.n_rounds[0])]["worker"]) == {0, 1, 2}
+    assert np.all(d.reqs["status"] != oracle.PENDING)
+    # an expired request could not have been completed in time by any worker at the round that retired it
+    nr = int(d.n_rounds[0])
+    for i in np.nonzero(d.reqs["status"] == oracle.EXPIRED)[0]:
+        r = int(d.reqs["round"][i])
+        clock = [int(w.t0_ns[0])] * nw; loaded = [-1] * nw
+        for q in range(min(r, nr)):
+            rec = d.rounds[0, q]; clock[int(rec["worker"])] = int(rec["t_end_ns"]); loaded[int(rec["worker"])] = int(rec["model"])
+        a = int(w.app[i])
+        best = min(clock[k] + (int(sw[k, g]) if g != loaded[k] else 0) + int(al[k, g]) + int(be[k, g]) * int(w.batch_sizes[0])
+                   for k in range(nw) for g in range(first_model(w, a), first_model(w, a) + int(w.models_per_app[a])))
+        assert w.deadline_ns[i] < best
+
+
+# ------------------------------------------------------------------ k-nearest-neighbour evidence (Section 4.1)
+
+def _knn_workload(rng, n=40, r=300, d=6, c=4, a=2, m=3):
+    w = manual_workload(rng.dirichlet(np.ones(c), size=n), rng.uniform(0.2, 0.99, size=(a * m, c)), app=rng.integers(0, a, size=n),
+                        deadline_ms=rng.uniform(50, 400, size=n), alpha_ms=rng.uniform(2, 20, size=a * m),
+                        beta_ms=rng.uniform(0.5, 5, size=a * m), swap_ms=rng.uniform(5, 50, size=a * m), batch_sizes=[1, 2, 4],
+                        models_per_app=[m] * a)
+    w.feat_dim = d
+    w.feats = rng.standard_normal(size=(n, d)).astype(np.float32)
+    w.head_w = np.zeros((1, a, d, c), dtype=np.float32)
+    ref = rng.standard_normal(size=(r, d)).astype(np.float32)
+    return w, ref, rng.integers(0, c, size=r).astype(np.int32), rng.integers(0, a, size=r).astype(np.int32)
+
+
+def test_knn_evidence_worked_example_of_the_paper():
+    """Section 4.1's example: k = 5 neighbours, two of class "no fall" and three of class "fall", give the evidence
+    y = <2, 3>; with the Jeffreys prior (alpha = 1/2) the posterior is Dir(2.5, 3.5), mean (5/12, 7/12)."""
+    d = 2
+    ref = np.asarray([[0.1, 0.0], [0.0, 0.2], [0.3, 0.0], [0.0, -0.4], [0.5, 0.0], [5.0, 5.0], [-6.0, 1.0]], dtype=np.float32)
+    ref_label = np.asarray([0, 1, 1, 0, 1, 0, 0], dtype=np.int32)            # the five closest to the origin: 0, 1, 1, 0, 1
+    w = manual_workload([[0.5, 0.5]], [[1.0, 0.0], [0.0, 1.0]], app=[0], deadline_ms=[100], alpha_ms=[1, 1], beta_ms=[1, 1],
+                        swap_ms=[0, 0], batch_sizes=[1], models_per_app=[2], prior_alpha=np.full((1, 2), 0.5), evidence_k=5.0)
+    w.feat_dim = d
+    w.feats = np.zeros((1, d), dtype=np.float32)
+    w.head_w = np.zeros((1, 1, d, 2), dtype=np.float32)
+    s = oracle.score_knn(w, 5, ref, ref_label, np.zeros(7, dtype=np.int32), want_theta=True)
+    np.testing.assert_allclose(s.theta[0], [5 / 12, 7 / 12], rtol=1e-15)
+    np.testing.assert_allclose(s.acc[0], [5 / 12, 7 / 12], rtol=1e-15)        # recall rows are the unit vectors
+    assert s.label[0] == 1
+    w.prior_alpha = None
+    np.testing.assert_allclose(oracle.score_knn(w, 5, ref, ref_label, np.zeros(7, dtype=np.int32), want_theta=True).theta[0], [0.4, 0.6])
+
+
+@pytest.mark.parametrize("k", [1, 5, 9])
+def test_knn_votes_equal_a_library_sort(k):
+    rng = np.random.default_rng(800 + k)
+    w, ref, ref_label, ref_app = _knn_workload(rng)
+    s = oracle.score_knn(w, k, ref, ref_label, ref_app, want_theta=True)
+    c = w.n_classes
+    for i in range(w.n_requests):
+        own = np.nonzero(ref_app == w.app[i])[0]
+        dist = np.sum((w.feats[i].astype(np.float64)[None, :] - ref[own].astype(np.float64)) ** 2, axis=1)
+        nearest = own[np.argsort(dist, kind="stable")[:k]]
+        votes = np.bincount(ref_label[nearest], minlength=c) / float(k)
+        np.testing.assert_allclose(s.theta[i], votes, atol=1e-15)
+        g0 = first_model(w, int(w.app[i]))
+        np.testing.assert_allclose(s.acc[i], w.recall[0, g0:g0 + 3].astype(np.float64) @ votes, rtol=1e-13)
+    if k == 1:                                                   # one neighbour: the posterior is one-hot
+        assert np.all(np.sort(s.theta, axis=1)[:, -1] == 1.0) and np.all(s.label >= 0)
+
+
+def test_knn_ties_and_small_reference_sets():
+    w = manual_workload([[0.5, 0.5]] * 2, [[1.0, 0.0]], app=[0, 1], deadline_ms=[100] * 2, alpha_ms=[1, 1], beta_ms=[1, 1],
+                        swap_ms=[0, 0], batch_sizes=[1], models_per_app=[1, 1])
+    w.recall = np.asarray([[[1.0, 0.0], [1.0, 0.0]]], dtype=np.float32)
+    w.feat_dim = 1
+    w.feats = np.zeros((2, 1), dtype=np.float32)
+    w.head_w = np.zeros((1, 2, 1, 2), dtype=np.float32)
+    ref = np.asarray([[1.0], [-1.0], [1.0]], dtype=np.float32)   # three points at the same distance from the origin
+    s = oracle.score_knn(w, 2, ref, np.asarray([1, 0, 0], dtype=np.int32), np.zeros(3, dtype=np.int32), want_theta=True)
+    np.testing.assert_allclose(s.theta[0], [0.5, 0.5])           # the two with the lower index: labels 1 and 0
+    np.testing.assert_allclose(s.theta[1], [0.5, 0.5])           # application 1 has no reference point: uniform
+    s5 = oracle.score_knn(w, 5, ref, np.asarray([1, 0, 0], dtype=np.int32), np.zeros(3, dtype=np.int32), want_theta=True)
+    np.testing.assert_allclose(s5.theta[0], [2 / 3, 1 / 3])      # fewer points than k: all of them vote
