@@ -94,7 +94,7 @@ typedef struct {
     int32_t status; /* SP_PENDING / SP_SCHEDULED / SP_EXPIRED */
     int32_t round;  /* round that scheduled or retired it, -1 while pending */
     int32_t model;  /* global model id, -1 unless scheduled */
-    int32_t pad_;
+    int32_t worker; /* worker that runs it (sp_schedule_workers), else 0 */
     int64_t order;  /* 1-based execution order inside its instance, 0 unless scheduled */
 } sp_req_rec;       /* 24 bytes */
 
@@ -164,6 +164,26 @@ sp_status sp_set_clocks(sp_ctx *ctx, const int64_t *t_ns, const int32_t *loaded_
 sp_status sp_score(sp_ctx *ctx, int64_t n, const void *feats, const int32_t *app, const int64_t *arrival_ns,
                    const int64_t *deadline_ns, const int32_t *instance, float *acc_out);
 
+/*
+ * The SneakPeek model as the paper builds it (Section 4.1): the evidence of a request is the vote of its k nearest
+ * labelled reference points among those of its application (exact neighbours: squared Euclidean distance in fp64, ties
+ * to the lower index), theta the mean of the Dirichlet posterior of Eq. 10-11 over the vote counts,
+ * theta_c = (alpha_c + y_c) / (sum alpha + k'), k' = min(k, reference points of the application); without a prior
+ * theta = y / k' (uniform when the application has no reference point).  sp_load_evidence copies the reference set (HOST
+ * arrays; single-instance contexts; dropped by sp_load_profiles).  sp_score_knn is sp_score() with that model in place
+ * of the linear head (head_w / head_b / evidence_k of the profiles are not used); it starts a table and cannot append.
+ */
+typedef struct {
+    int32_t k;                  /* neighbours, 1..1024 */
+    int64_t n_ref;              /* R reference points */
+    const void *ref_feats;      /* HOST [R][D], float or bf16 as in the profiles */
+    const int32_t *ref_label;   /* HOST [R], 0..C-1 */
+    const int32_t *ref_app;     /* HOST [R], 0..A-1 */
+} sp_knn_evidence;
+sp_status sp_load_evidence(sp_ctx *ctx, const sp_knn_evidence *evidence);
+sp_status sp_score_knn(sp_ctx *ctx, int64_t n, const void *feats, const int32_t *app, const int64_t *arrival_ns,
+                       const int64_t *deadline_ns, float *acc_out);
+
 /* Copies scores of requests first..first+n-1 to DEVICE buffers: acc [n][Mmax] float and/or v [n] float
  * (v = 1 + population variance of the request's accuracies); either may be NULL. */
 sp_status sp_get_scores(sp_ctx *ctx, int64_t first, int64_t n, float *acc, float *v);
@@ -182,8 +202,8 @@ sp_status sp_schedule_round(sp_ctx *ctx, int32_t max_rounds, sp_round_rec *round
                             int32_t *n_done);
 
 /*
- * Three more ways to schedule a freshly scored SNAPSHOT table (no round run on it yet, not trace mode; otherwise
- * SP_ESTATE).  All three first compute the fp64 scores and the data-aware label of every request in one pass over the
+ * More ways to schedule a freshly scored SNAPSHOT table (no round run on it yet, not trace mode; otherwise
+ * SP_ESTATE).  They first compute the fp64 scores and the data-aware label of every request in one pass over the
  * whole table and take every decision on those, run the table to completion in one call, and write records like
  * sp_schedule_round() (rounds_out DEVICE [I][cap] or NULL, n_done DEVICE [I] or NULL; sp_round_rec.exact carries the
  * sub-group: bits 8 and up hold predicted label + 1, 0 = the application's unsplit remainder or no sub-groups).
@@ -201,9 +221,22 @@ sp_status sp_schedule_round(sp_ctx *ctx, int32_t max_rounds, sp_round_rec *round
  * sp_schedule_baseline: the request-level baselines of Section 5.1, one request at a time in EDF or Eq. 12 priority
  *   order: SP_BASE_MAXACC_EDF (most accurate model that meets the deadline, else the most accurate of all),
  *   SP_BASE_LO_EDF and SP_BASE_LO_PRIORITY (Eq. 13: highest utility at the time the request starts).  Nothing is retired.
- * sp_get_labels: the labels (-1 = none above one half) to a DEVICE buffer, after one of the three calls.
+ * sp_get_labels: the labels (-1 = none above one half) to a DEVICE buffer, after one of these calls.
+ * sp_set_workers / sp_schedule_workers / sp_get_workers: several workers (Section 6: every model variant has a latency
+ *   profile per worker and the schedule gains a worker index).  sp_set_workers registers 1..64 workers with HOST arrays
+ *   [W][sumM] (copied; single-instance contexts; dropped by sp_load_profiles).  sp_schedule_workers runs the greedy
+ *   rounds (over applications, or sub-groups when split != 0) as list scheduling: every worker starts at the instance's
+ *   clock with its resident model; the worker that is free first (lowest clock, then lowest index) takes the next batch,
+ *   chosen as in a single-worker round from that worker's profile; a request is retired when no worker could complete
+ *   it in time.  sp_req_rec.worker and bits 2..7 of sp_round_rec.exact give the worker.  sp_get_workers copies the
+ *   workers' final clocks and resident models to DEVICE buffers t_ns [W], loaded [W]; the instance's clock becomes the
+ *   last completion.
  */
 enum { SP_BASE_MAXACC_EDF = 0, SP_BASE_LO_EDF = 1, SP_BASE_LO_PRIORITY = 2 };
+sp_status sp_set_workers(sp_ctx *ctx, int32_t n_workers, const int64_t *lat_alpha_ns, const int64_t *lat_beta_ns,
+                         const int64_t *swap_ns);
+sp_status sp_schedule_workers(sp_ctx *ctx, int32_t split, sp_round_rec *rounds_out, int64_t cap, int32_t *n_done);
+sp_status sp_get_workers(sp_ctx *ctx, int64_t *t_ns, int32_t *loaded);
 sp_status sp_schedule_split(sp_ctx *ctx, sp_round_rec *rounds_out, int64_t cap, int32_t *n_done);
 sp_status sp_schedule_exhaustive(sp_ctx *ctx, int32_t split, sp_round_rec *rounds_out, int64_t cap, int32_t *n_done,
                                  double *total_out, int64_t *n_solutions_out);

@@ -24,14 +24,15 @@ ROUND_DTYPE = np.dtype([
     ("instance", "<i4"), ("round", "<i4"), ("app", "<i4"), ("model", "<i4"), ("batch", "<i4"),
     ("n_members", "<i4"), ("n_expired", "<i4"), ("exact", "<i4"), ("t_start_ns", "<i8"), ("t_end_ns", "<i8"),
     ("utility", "<f8"), ("group_priority", "<f8")], align=True)
-REQ_DTYPE = np.dtype([("status", "<i4"), ("round", "<i4"), ("model", "<i4"), ("pad_", "<i4"), ("order", "<i8")],
+REQ_DTYPE = np.dtype([("status", "<i4"), ("round", "<i4"), ("model", "<i4"), ("worker", "<i4"), ("order", "<i8")],
                      align=True)
 assert ROUND_DTYPE.itemsize == 64 and REQ_DTYPE.itemsize == 24
 
 EXPORTS = ["sp_create", "sp_destroy", "sp_last_error", "sp_load_profiles", "sp_default_options", "sp_set_options", "sp_set_clock",
            "sp_set_clocks", "sp_score", "sp_get_scores", "sp_schedule_round", "sp_get_requests", "sp_get_clocks",
            "sp_reset", "sp_check", "sp_get_stats", "sp_run_host", "sp_score_static", "sp_schedule_split",
-           "sp_schedule_exhaustive", "sp_schedule_baseline", "sp_get_labels"]
+           "sp_schedule_exhaustive", "sp_schedule_baseline", "sp_get_labels", "sp_set_workers", "sp_schedule_workers",
+           "sp_get_workers", "sp_load_evidence", "sp_score_knn"]
 SP_BASE_MAXACC_EDF, SP_BASE_LO_EDF, SP_BASE_LO_PRIORITY = 0, 1, 2
 
 
@@ -66,6 +67,11 @@ class _Stats(C.Structure):
 class _StaticHead(C.Structure):
     _fields_ = [("n_apps", C.c_int32), ("n_classes", C.c_int32), ("feat_dim", C.c_int32), ("feat_dtype", C.c_int32),
                 ("models_per_app", C.c_void_p), ("head_w", C.c_void_p), ("head_b", C.c_void_p), ("recall", C.c_void_p)]
+
+
+class _KnnEvidence(C.Structure):
+    _fields_ = [("k", C.c_int32), ("n_ref", C.c_int64), ("ref_feats", C.c_void_p), ("ref_label", C.c_void_p),
+                ("ref_app", C.c_void_p)]
 
 
 _lib = None
@@ -105,6 +111,11 @@ def load_library():
     lib.sp_schedule_exhaustive.argtypes = [vp, i32, vp, i64, vp, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     lib.sp_schedule_baseline.argtypes = [vp, i32, vp, i64, vp]
     lib.sp_get_labels.argtypes = [vp, i64, i64, vp]
+    lib.sp_load_evidence.argtypes = [vp, C.POINTER(_KnnEvidence)]
+    lib.sp_score_knn.argtypes = [vp, i64, vp, vp, vp, vp, vp]
+    lib.sp_set_workers.argtypes = [vp, i32, vp, vp, vp]
+    lib.sp_schedule_workers.argtypes = [vp, i32, vp, i64, vp]
+    lib.sp_get_workers.argtypes = [vp, vp, vp]
     lib.sp_score_static.argtypes = [C.c_int, vp, C.POINTER(_StaticHead), i64, vp, vp, vp, vp, C.c_char_p, i32]
     for name in EXPORTS:
         if name not in ("sp_destroy", "sp_last_error", "sp_default_options"):
@@ -194,6 +205,19 @@ def sp_score(ctx: int, n: int, feats, app, arrival_ns, deadline_ns, instance=Non
                                      _dev(instance), _dev(acc_out)))
 
 
+def sp_load_evidence(ctx: int, k: int, ref_feats: np.ndarray, ref_label: np.ndarray, ref_app: np.ndarray) -> None:
+    """Reference set of the k-nearest-neighbour SneakPeek model (host arrays; bf16 features as uint16 bit patterns)."""
+    rf = np.ascontiguousarray(ref_feats)
+    rl, ra = np.ascontiguousarray(ref_label, dtype=np.int32), np.ascontiguousarray(ref_app, dtype=np.int32)
+    ev = _KnnEvidence(int(k), int(rf.shape[0]), _host(rf), _host(rl), _host(ra))
+    _ok(ctx, load_library().sp_load_evidence(ctx, C.byref(ev)))
+
+
+def sp_score_knn(ctx: int, n: int, feats, app, arrival_ns, deadline_ns, acc_out=None) -> None:
+    _ok(ctx, load_library().sp_score_knn(ctx, int(n), _dev(feats), _dev(app), _dev(arrival_ns), _dev(deadline_ns),
+                                         _dev(acc_out)))
+
+
 def sp_get_scores(ctx: int, first: int, n: int, acc=None, v=None) -> None:
     _ok(ctx, load_library().sp_get_scores(ctx, int(first), int(n), _dev(acc), _dev(v)))
 
@@ -216,6 +240,20 @@ def sp_schedule_exhaustive(ctx: int, split: bool, rounds_out=None, cap: int = 0,
 
 def sp_schedule_baseline(ctx: int, policy: int, rounds_out=None, cap: int = 0, n_done=None) -> None:
     _ok(ctx, load_library().sp_schedule_baseline(ctx, int(policy), _dev(rounds_out), int(cap), _dev(n_done)))
+
+
+def sp_set_workers(ctx: int, lat_alpha_ns: np.ndarray, lat_beta_ns: np.ndarray, swap_ns: np.ndarray) -> None:
+    """Registers W workers; the three arrays are host arrays [W, sumM] of int64 nanoseconds."""
+    al, be, sw = (np.ascontiguousarray(a, dtype=np.int64) for a in (lat_alpha_ns, lat_beta_ns, swap_ns))
+    _ok(ctx, load_library().sp_set_workers(ctx, int(al.shape[0]), _host(al), _host(be), _host(sw)))
+
+
+def sp_schedule_workers(ctx: int, split: bool, rounds_out=None, cap: int = 0, n_done=None) -> None:
+    _ok(ctx, load_library().sp_schedule_workers(ctx, int(bool(split)), _dev(rounds_out), int(cap), _dev(n_done)))
+
+
+def sp_get_workers(ctx: int, t_ns=None, loaded=None) -> None:
+    _ok(ctx, load_library().sp_get_workers(ctx, _dev(t_ns), _dev(loaded)))
 
 
 def sp_get_labels(ctx: int, first: int, n: int, labels) -> None:

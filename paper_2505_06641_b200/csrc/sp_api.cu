@@ -16,6 +16,7 @@
 #include "sp_sched_warp.cuh"
 #include "sp_presort.cuh"
 #include "sp_policies.cuh"
+#include "sp_knn.cuh"
 
 using namespace sp;
 
@@ -71,6 +72,12 @@ struct sp_ctx {
     Buf t_app, t_arrival, t_deadline, a_cnt, a_cursor, a_gstart, r_id, r_dl, r_pw;
     // policies decided on fp64 scores: labels, group tables, exhaustive search
     Buf labels, g_key, g_start, g_head, g_count, exh_info, exh_total, exh_sol;
+    // k-nearest-neighbour evidence (sp_load_evidence): reference set feature-major in fp64, grouped by application
+    int knn_k = 0;
+    int64_t knn_R = 0, knn_max_per_app = 0;
+    Buf knn_refT, knn_label, knn_start, knn_prior_total, knn_dist;
+    int n_workers = 0;           // workers registered with sp_set_workers (0 = none)
+    Buf w_alpha, w_beta, w_swap, w_T, w_L;
     bool have_exact_all = false;
     // staging of sp_run_host
     Buf h_feats, h_app, h_arrival, h_deadline, h_instance, h_t0, h_loaded, h_rounds, h_ndone;
@@ -361,6 +368,43 @@ sp_status score_rows(sp_ctx *c, const DevTable &tv, float *acc_out) {
     return mark(c, c->ev_score);
 }
 
+// k-nearest-neighbour scoring of the rows of `tv` (fresh single-instance table): fp64 throughout, so the rows also get
+// their exact scores and labels, and the policies that run on fp64 scores need no second pass.
+sp_status score_rows_knn(sp_ctx *c, const DevTable &tv, float *acc_out) {
+    const DevProfiles &P = c->P;
+    const size_t nn = (size_t)(tv.n > 0 ? tv.n : 1);
+    SP_TRY(ensure(c, c->labels, nn * 4));
+    int64_t blocks = (tv.n + kKnnWarps - 1) / kKnnWarps;
+    if (blocks > (int64_t)c->n_sms * 4) blocks = (int64_t)c->n_sms * 4;
+    const int64_t stride = c->knn_max_per_app > 0 ? c->knn_max_per_app : 1;
+    SP_TRY(ensure(c, c->knn_dist, (size_t)blocks * kKnnWarps * stride * 8));
+    KnnParams kp{};
+    kp.P = P; kp.tb = tv; kp.k = c->knn_k; kp.R = c->knn_R;
+    kp.refT = (const double *)c->knn_refT.p; kp.ref_label = (const int32_t *)c->knn_label.p;
+    kp.app_start = (const int64_t *)c->knn_start.p;
+    kp.prior_total = P.prior ? (const double *)c->knn_prior_total.p : nullptr;
+    kp.dist = (double *)c->knn_dist.p; kp.dist_stride = stride;
+    kp.labels = (int32_t *)c->labels.p; kp.acc_out = acc_out; kp.flags = (const int *)c->flags.p;
+    if (P.prior) {                                   // sum of the hyper-parameters per application, label by label in fp64
+        std::vector<float> al((size_t)P.A * P.C);
+        SP_CUDA(c, cudaMemcpyAsync(al.data(), P.prior, al.size() * 4, cudaMemcpyDeviceToHost, c->stream));
+        SP_CUDA(c, cudaStreamSynchronize(c->stream));
+        std::vector<double> tot((size_t)P.A, 0.0);
+        for (int a = 0; a < P.A; ++a)
+            for (int k = 0; k < P.C; ++k) tot[(size_t)a] += (double)al[(size_t)a * P.C + k];
+        SP_TRY(upload(c, c->knn_prior_total, tot.data(), tot.size() * 8));
+        SP_CUDA(c, cudaStreamSynchronize(c->stream));
+        kp.prior_total = (const double *)c->knn_prior_total.p;
+    }
+    const size_t smem = (size_t)kKnnWarps * (P.D + P.C) * 8;
+    SP_CUDA(c, cudaFuncSetAttribute(k_score_knn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    SP_TRY(mark(c, c->ev_score));
+    k_score_knn<<<(unsigned)blocks, kKnnWarps * 32, smem, c->stream>>>(kp);
+    SP_TRY(launched(c, "k_score_knn"));
+    c->have_exact_all = true;
+    return mark(c, c->ev_score);
+}
+
 // Appending requests changes the size of every application's queue region (regions are laid out back to back, sized by
 // the number of requests of the application scored so far).  One block: the live part of every queue is copied out
 // (phase 1) and back in at the start of its new region in queue copy 0 (phase 2); heads, tails and region starts follow.
@@ -518,7 +562,8 @@ void sp_destroy(sp_ctx *c) {
                   &c->h_feats, &c->h_app, &c->h_arrival, &c->h_deadline, &c->h_instance, &c->h_t0, &c->h_loaded,
                   &c->h_rounds, &c->h_ndone, &c->t_app, &c->t_arrival, &c->t_deadline, &c->a_cnt, &c->a_cursor,
                   &c->a_gstart, &c->r_id, &c->r_dl, &c->r_pw, &c->labels, &c->g_key, &c->g_start, &c->g_head, &c->g_count,
-                  &c->exh_info, &c->exh_total, &c->exh_sol};
+                  &c->exh_info, &c->exh_total, &c->exh_sol, &c->w_alpha, &c->w_beta, &c->w_swap, &c->w_T, &c->w_L,
+                  &c->knn_refT, &c->knn_label, &c->knn_start, &c->knn_prior_total, &c->knn_dist};
     for (Buf *b : all) release(*b);
     for (Buf &b : c->seg_copies) release(b);
     delete c;
@@ -577,6 +622,8 @@ sp_status sp_load_profiles(sp_ctx *c, const sp_profiles *p) {
     if (ss.end > 96 * 1024) return fail(c, SP_EINVAL, "models_per_app x largest batch size is too large for one block");
 
     c->have_profiles = false;
+    c->n_workers = 0;
+    c->knn_k = 0;
     drop_table(c);
     c->hp.models_per_app.assign(p->models_per_app, p->models_per_app + A);
     c->hp.batch_sizes.assign(p->batch_sizes, p->batch_sizes + nB);
@@ -747,11 +794,13 @@ sp_status sp_reset(sp_ctx *c) {
     return SP_OK;
 }
 
-sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, const int64_t *arrival_ns,
-                   const int64_t *deadline_ns, const int32_t *instance, float *acc_out) {
+static sp_status score_impl(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, const int64_t *arrival_ns,
+                            const int64_t *deadline_ns, const int32_t *instance, float *acc_out, bool knn) {
     if (!c) return SP_EINVAL;
     if (!c->have_profiles) return fail(c, SP_ESTATE, "no profiles loaded");
     const bool append = c->have_table;
+    if (knn && (append || c->knn_k < 1))
+        return fail(c, SP_ESTATE, append ? "sp_score_knn starts a table: call sp_reset first" : "no evidence loaded; call sp_load_evidence first");
     if (append && c->P.I != 1)
         return fail(c, SP_ESTATE, "requests can be appended to a single-instance context only; call sp_reset first");
     if (n < 0 || n > ((int64_t)1 << 40)) return fail(c, SP_EINVAL, "n out of range");
@@ -853,7 +902,7 @@ sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, 
                                                               tv.gstart, (int32_t *)c->tiled_start.p, (int32_t *)c->small_start.p);
         SP_TRY(launched(c, "k_group_scan_blocks"));
     }
-    if (n > 0) SP_TRY(score_rows(c, tv, acc_out));
+    if (n > 0) SP_TRY(knn ? score_rows_knn(c, tv, acc_out) : score_rows(c, tv, acc_out));
     if (append) {
         // make room in every application's queue region for its new requests; live entries move to the new regions
         k_queue_regrow<<<1, 1024, 0, c->stream>>>((InstState *)c->state.p, P.A, (int64_t *)c->gstart.p, (const int32_t *)c->a_cnt.p,
@@ -865,6 +914,59 @@ sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, 
     }
     c->have_table = true;
     if (!append) c->sched_started = false;
+    return SP_OK;
+}
+
+sp_status sp_score(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, const int64_t *arrival_ns,
+                   const int64_t *deadline_ns, const int32_t *instance, float *acc_out) {
+    return score_impl(c, n, feats, app, arrival_ns, deadline_ns, instance, acc_out, false);
+}
+
+sp_status sp_score_knn(sp_ctx *c, int64_t n, const void *feats, const int32_t *app, const int64_t *arrival_ns,
+                       const int64_t *deadline_ns, float *acc_out) {
+    return score_impl(c, n, feats, app, arrival_ns, deadline_ns, nullptr, acc_out, true);
+}
+
+sp_status sp_load_evidence(sp_ctx *c, const sp_knn_evidence *ev) {
+    if (!c) return SP_EINVAL;
+    if (!c->have_profiles) return fail(c, SP_ESTATE, "no profiles loaded");
+    if (c->P.I != 1) return fail(c, SP_ESTATE, "k-nearest-neighbour evidence is for single-instance contexts");
+    if (!ev || ev->k < 1 || ev->k > kKnnMaxK || ev->n_ref < 0 || (ev->n_ref > 0 && (!ev->ref_feats || !ev->ref_label || !ev->ref_app)))
+        return fail(c, SP_EINVAL, "bad evidence description (k must be 1..1024, arrays non-NULL)");
+    const DevProfiles &P = c->P;
+    const int64_t R = ev->n_ref;
+    if ((size_t)(P.D + P.C) * 8 * kKnnWarps > 200 * 1024) return fail(c, SP_EINVAL, "feat_dim + n_classes is too large for the neighbour kernel");
+    std::vector<int64_t> start((size_t)P.A + 1, 0);
+    for (int64_t r = 0; r < R; ++r) {
+        if (ev->ref_app[r] < 0 || ev->ref_app[r] >= P.A || ev->ref_label[r] < 0 || ev->ref_label[r] >= P.C)
+            return fail(c, SP_EINVAL, "reference point with an application or label out of range");
+        ++start[(size_t)ev->ref_app[r] + 1];
+    }
+    int64_t max_per_app = 0;
+    for (int a = 0; a < P.A; ++a) { max_per_app = start[a + 1] > max_per_app ? start[a + 1] : max_per_app; start[a + 1] += start[a]; }
+    // stable grouping by application (ties between equal distances go to the lower original index), feature-major, fp64
+    std::vector<int64_t> cursor(start.begin(), start.end() - 1);
+    std::vector<double> refT((size_t)(R > 0 ? R : 1) * P.D);
+    std::vector<int32_t> lab((size_t)(R > 0 ? R : 1));
+    for (int64_t r = 0; r < R; ++r) {
+        const int64_t pos = cursor[(size_t)ev->ref_app[r]]++;
+        lab[(size_t)pos] = ev->ref_label[r];
+        for (int d = 0; d < P.D; ++d) {
+            double val;
+            if (P.dtype == SP_BF16) {
+                const uint32_t bits = (uint32_t)((const uint16_t *)ev->ref_feats)[r * P.D + d] << 16;
+                float f; std::memcpy(&f, &bits, 4); val = (double)f;
+            } else val = (double)((const float *)ev->ref_feats)[r * P.D + d];
+            refT[(size_t)d * R + pos] = val;
+        }
+    }
+    SP_CUDA(c, cudaSetDevice(c->device));
+    SP_TRY(upload(c, c->knn_refT, refT.data(), refT.size() * 8));
+    SP_TRY(upload(c, c->knn_label, lab.data(), lab.size() * 4));
+    SP_TRY(upload(c, c->knn_start, start.data(), start.size() * 8));
+    SP_CUDA(c, cudaStreamSynchronize(c->stream));      // the host arrays may be freed on return
+    c->knn_R = R; c->knn_max_per_app = max_per_app;
+    c->knn_k = ev->k;
     return SP_OK;
 }
 
@@ -969,11 +1071,17 @@ sp_status sp_get_labels(sp_ctx *c, int64_t first, int64_t n, int32_t *labels) {
     return SP_OK;
 }
 
-sp_status sp_schedule_split(sp_ctx *c, sp_round_rec *rounds_out, int64_t cap, int32_t *n_done) {
-    if (!c) return SP_EINVAL;
+// Greedy rounds over groups (applications or data-aware sub-groups) on the profiles' worker or on the registered workers.
+static sp_status run_group_rounds(sp_ctx *c, const char *who, bool use_labels, bool use_workers, sp_round_rec *rounds_out,
+                                  int64_t cap, int32_t *n_done) {
     GroupParams gp;
-    SP_TRY(policy_prologue(c, "sp_schedule_split", &gp, true, rounds_out, cap, n_done));
+    SP_TRY(policy_prologue(c, who, &gp, use_labels, rounds_out, cap, n_done));
     const DevProfiles &P = c->P;
+    if (use_workers) {
+        gp.W = c->n_workers;
+        gp.w_alpha = (const int64_t *)c->w_alpha.p; gp.w_beta = (const int64_t *)c->w_beta.p; gp.w_swap = (const int64_t *)c->w_swap.p;
+        gp.w_T = (int64_t *)c->w_T.p; gp.w_L = (int32_t *)c->w_L.p;
+    }
     if (P.I == 1 && c->tb.n > gp.sort_cap && c->tb.n < ((int64_t)1 << 31)) {
         k_group_keys<<<(unsigned)((c->tb.n + 255) / 256), 256, 0, c->stream>>>(gp, c->tb.n);
         SP_TRY(launched(c, "k_group_keys"));
@@ -988,6 +1096,48 @@ sp_status sp_schedule_split(sp_ctx *c, sp_round_rec *rounds_out, int64_t cap, in
     k_sched_groups<<<P.I, nt, L.end, c->stream>>>(gp);
     SP_TRY(launched(c, "k_sched_groups"));
     return mark(c, c->ev_sched);
+}
+
+sp_status sp_schedule_split(sp_ctx *c, sp_round_rec *rounds_out, int64_t cap, int32_t *n_done) {
+    if (!c) return SP_EINVAL;
+    return run_group_rounds(c, "sp_schedule_split", true, false, rounds_out, cap, n_done);
+}
+
+sp_status sp_set_workers(sp_ctx *c, int32_t n_workers, const int64_t *lat_alpha_ns, const int64_t *lat_beta_ns, const int64_t *swap_ns) {
+    if (!c) return SP_EINVAL;
+    if (!c->have_profiles) return fail(c, SP_ESTATE, "no profiles loaded");
+    if (c->P.I != 1) return fail(c, SP_ESTATE, "several workers are for single-instance contexts");
+    if (n_workers < 1 || n_workers > kMaxWorkers) return fail(c, SP_EINVAL, "n_workers must be 1..64");
+    if (!lat_alpha_ns || !lat_beta_ns || !swap_ns) return fail(c, SP_EINVAL, "a worker profile array is NULL");
+    const int64_t nm = (int64_t)n_workers * c->P.sumM, lat_limit = (int64_t)1 << 50;
+    for (int64_t k = 0; k < nm; ++k)
+        if (lat_alpha_ns[k] < 0 || lat_beta_ns[k] < 0 || swap_ns[k] < 0 || lat_alpha_ns[k] > lat_limit ||
+            lat_beta_ns[k] > lat_limit / kMaxBatch || swap_ns[k] > lat_limit)
+            return fail(c, SP_EINVAL, "latency and swap profiles must be in [0, 2^50] ns");
+    SP_CUDA(c, cudaSetDevice(c->device));
+    SP_TRY(upload(c, c->w_alpha, lat_alpha_ns, (size_t)nm * 8));
+    SP_TRY(upload(c, c->w_beta, lat_beta_ns, (size_t)nm * 8));
+    SP_TRY(upload(c, c->w_swap, swap_ns, (size_t)nm * 8));
+    SP_TRY(ensure(c, c->w_T, (size_t)n_workers * 8));
+    SP_TRY(ensure(c, c->w_L, (size_t)n_workers * 4));
+    SP_CUDA(c, cudaStreamSynchronize(c->stream));     // the host arrays may be freed on return
+    c->n_workers = n_workers;
+    return SP_OK;
+}
+
+sp_status sp_schedule_workers(sp_ctx *c, int32_t split, sp_round_rec *rounds_out, int64_t cap, int32_t *n_done) {
+    if (!c) return SP_EINVAL;
+    if (c->n_workers < 1) return fail(c, SP_ESTATE, "no workers registered; call sp_set_workers first");
+    return run_group_rounds(c, "sp_schedule_workers", split != 0, true, rounds_out, cap, n_done);
+}
+
+sp_status sp_get_workers(sp_ctx *c, int64_t *t_ns, int32_t *loaded) {
+    if (!c) return SP_EINVAL;
+    if (c->n_workers < 1) return fail(c, SP_ESTATE, "no workers registered");
+    SP_CUDA(c, cudaSetDevice(c->device));
+    if (t_ns) SP_CUDA(c, cudaMemcpyAsync(t_ns, c->w_T.p, (size_t)c->n_workers * 8, cudaMemcpyDeviceToDevice, c->stream));
+    if (loaded) SP_CUDA(c, cudaMemcpyAsync(loaded, c->w_L.p, (size_t)c->n_workers * 4, cudaMemcpyDeviceToDevice, c->stream));
+    return SP_OK;
 }
 
 sp_status sp_schedule_exhaustive(sp_ctx *c, int32_t split, sp_round_rec *rounds_out, int64_t cap, int32_t *n_done,

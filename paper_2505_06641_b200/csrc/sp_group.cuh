@@ -18,7 +18,7 @@ __global__ void k_group_count(DevProfiles P, DevTable tb, int trace_mode, int *f
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= tb.n) return;
     if (tb.recs) {                           // the request starts pending, without an fp64 re-scoring (a table
-        sp_req_rec r; r.status = SP_PENDING; r.round = -1; r.model = -1; r.pad_ = 0; r.order = 0;   // that is only scored has no records)
+        sp_req_rec r; r.status = SP_PENDING; r.round = -1; r.model = -1; r.worker = 0; r.order = 0;   // that is only scored has no records)
         tb.recs[i] = r;
         tb.exact[i] = 0;
     }

@@ -2,7 +2,8 @@
 //   * k_exact_all      : fp64 scores (Section 4.1, Eq. 9, Eq. 12) and the data-aware label (Section 4.3) of every request,
 //                        one warp per request over the whole GPU;
 //   * k_sched_groups   : the greedy rounds of Algorithm 1 over data-aware sub-groups ("Enhancements for Grouped
-//                        Scheduling": requests of an application with the same predicted label form a group);
+//                        Scheduling": requests of an application with the same predicted label form a group), on one
+//                        worker or on several (Section 6: the worker that is free first takes the next batch);
 //   * k_exh_*          : the exhaustive branch of Algorithm 1 (number of groups at most the threshold): every order of
 //                        the groups times every model choice, one thread per solution;
 //   * k_baseline       : the request-level baselines of Section 5.1 (MaxAcc-EDF, LO-EDF, LO-Priority).
@@ -15,6 +16,7 @@
 
 namespace sp {
 
+constexpr int kMaxWorkers = 64;             // workers of the multi-worker rounds
 constexpr int kExhMaxGroups = 8;            // groups the exhaustive branch accepts (8! * M^8 solutions at most 2^31)
 
 // ------------------------------------------------------------------------------------------------ fp64 scores of all rows
@@ -49,6 +51,12 @@ struct GroupParams {
     int64_t cap;
     int32_t *n_done;
     int sort_cap, bmax, presorted;
+    // several workers (Section 6): W > 0 workers with their own latency profiles [W][sumM], clocks and resident models
+    // (single-instance contexts); W = 0: the one worker of the profiles
+    int W;
+    const int64_t *w_alpha, *w_beta, *w_swap;
+    int64_t *w_T;
+    int32_t *w_L;
 };
 
 __device__ __forceinline__ int group_of(const GroupParams &gp, int64_t id) {
@@ -140,11 +148,15 @@ __global__ void __launch_bounds__(1024, 1) k_sched_groups(GroupParams gp) {
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ InstState st;
     __shared__ int64_t s_emin[kMaxApps];
-    __shared__ int s_retired, s_live, s_best_g, s_best_ci;
+    __shared__ int s_retired, s_live, s_best_g, s_best_ci, s_wk;
     __shared__ double s_best_p, s_best_u;
+    __shared__ int64_t s_T[kMaxWorkers];
+    __shared__ int s_L[kMaxWorkers];
+    __shared__ unsigned char s_app_of[kMaxApps * kMaxModelsPerApp];
     const DevProfiles &P = gp.P;
     const DevTable &tb = gp.tb;
     const int inst = blockIdx.x;
+    const int W = gp.W;
     const int tid = threadIdx.x, NT = blockDim.x, lane = tid & 31, warp = tid >> 5, nwarps = NT >> 5;
     const int A = P.A, nB = P.nB, Mmax = P.Mmax, bmax = gp.bmax;
     const int GW = gp.labels ? P.C + 1 : 1;
@@ -162,12 +174,17 @@ __global__ void __launch_bounds__(1024, 1) k_sched_groups(GroupParams gp) {
     const int64_t r0 = tb.qstart[(int64_t)inst * A], r1 = tb.qstart[(int64_t)(inst + 1) * A];
     const int n_inst = (int)(r1 - r0);
     const int64_t gb = r0 + inst;
-    if (tid == 0) { st = gp.state[inst]; st.Tref = st.T; st.started = 1; }
+    if (tid == 0) { st = gp.state[inst]; st.Tref = st.T; st.started = 1; s_wk = 0; }
     for (int g = tid; g < P.sumM; g += NT) {
         al[g] = P.lat_alpha[(int64_t)inst * P.sumM + g];
         be[g] = P.lat_beta[(int64_t)inst * P.sumM + g];
         sw[g] = P.swap[(int64_t)inst * P.sumM + g];
+        int a2 = 0;
+        while (g >= P.mfirst[a2 + 1]) ++a2;
+        s_app_of[g] = (unsigned char)a2;
     }
+    __syncthreads();
+    for (int k = tid; k < W; k += NT) { s_T[k] = st.T; s_L[k] = st.L; }   // every worker starts at the instance's clock
     __syncthreads();
     const int G = build_group_queues(gp, inst, reinterpret_cast<SortKey *>(dyn + L.keys), st.Tref);
     const double tau = P.tau;
@@ -179,6 +196,19 @@ __global__ void __launch_bounds__(1024, 1) k_sched_groups(GroupParams gp) {
     bool finished = false;
     for (int64_t iter = 0; iter < max_iter; ++iter) {
         if (s_live == 0) { finished = true; break; }
+        if (W > 0) {                                     // the worker that is free first takes this round
+            if (tid == 0) {
+                int wk = 0;
+                for (int k = 1; k < W; ++k) if (s_T[k] < s_T[wk]) wk = k;
+                s_wk = wk; st.T = s_T[wk]; st.L = s_L[wk];
+            }
+            __syncthreads();
+            for (int g = tid; g < P.sumM; g += NT) {
+                al[g] = gp.w_alpha[(int64_t)s_wk * P.sumM + g]; be[g] = gp.w_beta[(int64_t)s_wk * P.sumM + g];
+                sw[g] = gp.w_swap[(int64_t)s_wk * P.sumM + g];
+            }
+            __syncthreads();
+        }
         if (st.T - st.Tref > reref_ns) {                 // keep exp((T - Tref)/tau) in range
             for (int p = tid; p < n_inst; p += NT)
                 gp.q_pw[r0 + p] = prio_weight(tb.v64[gp.q_id[r0 + p]], gp.q_dl[r0 + p], st.T, tau);
@@ -196,6 +226,14 @@ __global__ void __launch_bounds__(1024, 1) k_sched_groups(GroupParams gp) {
             s_emin[tid] = emin;
         }
         __syncthreads();
+        if (W > 1) {                                     // hopeless = no worker can complete the request in time
+            for (int kg = tid; kg < W * P.sumM; kg += NT) {
+                const int k = kg / P.sumM, g = kg - k * P.sumM;
+                const int64_t e = s_T[k] + (g != s_L[k] ? gp.w_swap[kg] : 0) + gp.w_alpha[kg] + gp.w_beta[kg] * (int64_t)P.batch[0];
+                atomicMin(reinterpret_cast<long long *>(&s_emin[s_app_of[g]]), (long long)e);
+            }
+            __syncthreads();
+        }
         for (int s = tid; s < G; s += NT) {
             const int head = gp.g_head[gb + s], tail = gp.g_start[gb + s + 1];
             if (head == tail) continue;
@@ -214,7 +252,7 @@ __global__ void __launch_bounds__(1024, 1) k_sched_groups(GroupParams gp) {
                 }
             }
             for (int p = head; p < nh; ++p) {
-                sp_req_rec r; r.status = SP_EXPIRED; r.round = st.round; r.model = -1; r.pad_ = 0; r.order = 0;
+                sp_req_rec r; r.status = SP_EXPIRED; r.round = st.round; r.model = -1; r.worker = 0; r.order = 0;
                 tb.recs[gp.q_id[r0 + p]] = r;
             }
             if (nh > head) { gp.g_head[gb + s] = nh; atomicAdd(&s_retired, nh - head); }
@@ -287,7 +325,7 @@ __global__ void __launch_bounds__(1024, 1) k_sched_groups(GroupParams gp) {
         const int ci = s_best_ci, bj = ci / nB, bbi = ci - bj * nB, g = m0 + bj, bp = cand_bp[ci];
         const int64_t e = cand_e[ci];
         for (int k = tid; k < bp; k += NT) {
-            sp_req_rec r; r.status = SP_SCHEDULED; r.round = st.round; r.model = g; r.pad_ = 0; r.order = st.next_order + k;
+            sp_req_rec r; r.status = SP_SCHEDULED; r.round = st.round; r.model = g; r.worker = s_wk; r.order = st.next_order + k;
             tb.recs[mem_id[k]] = r;
         }
         __syncthreads();
@@ -295,18 +333,24 @@ __global__ void __launch_bounds__(1024, 1) k_sched_groups(GroupParams gp) {
             if (gp.rounds_out && rounds_done < gp.cap) {
                 sp_round_rec rr;
                 rr.instance = inst; rr.round = st.round; rr.app = a; rr.model = g; rr.batch = P.batch[bbi];
-                rr.n_members = bp; rr.n_expired = st.exp_since; rr.exact = 3 | ((gp.labels ? gkey % GW : 0) << 8);
+                rr.n_members = bp; rr.n_expired = st.exp_since; rr.exact = 3 | (s_wk << 2) | ((gp.labels ? gkey % GW : 0) << 8);
                 rr.t_start_ns = st.T; rr.t_end_ns = e; rr.utility = s_best_u; rr.group_priority = s_best_p;
                 gp.rounds_out[(int64_t)inst * gp.cap + rounds_done] = rr;
             }
             gp.g_head[gb + s] = head + bp;
             st.T = e; st.L = g; st.round += 1; st.next_order += bp; st.exp_since = 0; s_live -= bp;
+            if (W > 0) { s_T[s_wk] = e; s_L[s_wk] = g; }
         }
         ++rounds_done;
         __syncthreads();
     }
     if (tid == 0) {
         if (!finished) dev_error(&gp.flags[0], kDevLimit);
+        if (W > 0) {                                     // per-worker clocks; the instance's clock is the last completion
+            int64_t tmax = s_T[0];
+            for (int k = 0; k < W; ++k) { gp.w_T[k] = s_T[k]; gp.w_L[k] = s_L[k]; tmax = s_T[k] > tmax ? s_T[k] : tmax; }
+            st.T = tmax; st.L = s_L[0];
+        }
         st.inserted = n_inst;
         for (int a2 = 0; a2 < kMaxApps; ++a2) { st.head[a2] = 0; st.tail[a2] = 0; st.cur[a2] = 0; }
         gp.state[inst] = st;
@@ -387,7 +431,7 @@ __device__ double exh_eval(const GroupParams &gp, const ExhInfo &info, const int
                 u = __dadd_rn(u, c);
                 total = __dadd_rn(total, c);
                 if (emit) {
-                    sp_req_rec r; r.status = SP_SCHEDULED; r.round = round; r.model = m; r.pad_ = 0; r.order = order++;
+                    sp_req_rec r; r.status = SP_SCHEDULED; r.round = round; r.model = m; r.worker = 0; r.order = order++;
                     tb.recs[id] = r;
                 }
             }
@@ -536,7 +580,7 @@ __global__ void __launch_bounds__(1024, 1) k_baseline(BaselineParams bp) {
         const int64_t e_best = __shfl_sync(0xffffffffu, (long long)e, bj);
         const double u_best = __shfl_sync(0xffffffffu, util, bj);
         if (lane == 0) {
-            sp_req_rec r; r.status = SP_SCHEDULED; r.round = pos; r.model = m0 + bj; r.pad_ = 0; r.order = pos + 1;
+            sp_req_rec r; r.status = SP_SCHEDULED; r.round = pos; r.model = m0 + bj; r.worker = 0; r.order = pos + 1;
             tb.recs[id] = r;
             if (gp.rounds_out && pos < gp.cap) {
                 sp_round_rec rr;

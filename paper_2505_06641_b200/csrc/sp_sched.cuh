@@ -582,7 +582,7 @@ __device__ void sched_instance(const SchedParams &sp, const int inst) {
             for (int a2 = 0; a2 < A; ++a2) {
                 const int64_t *qid = sp.q_id[st.cur[a2]] + s_base[a2];
                 for (int k = st.head[a2] + tid; k < s_lo[a2]; k += NT) {
-                    sp_req_rec r; r.status = SP_EXPIRED; r.round = st.round; r.model = -1; r.pad_ = 0; r.order = 0;
+                    sp_req_rec r; r.status = SP_EXPIRED; r.round = st.round; r.model = -1; r.worker = 0; r.order = 0;
                     tb.recs[qid[k]] = r;
                 }
             }
@@ -769,7 +769,7 @@ __device__ void sched_instance(const SchedParams &sp, const int inst) {
         const int bp = cand_bp[ci];
         const int64_t e = cand_e[ci];
         for (int k = tid; k < bp; k += NT) {
-            sp_req_rec r; r.status = SP_SCHEDULED; r.round = st.round; r.model = g; r.pad_ = 0;
+            sp_req_rec r; r.status = SP_SCHEDULED; r.round = st.round; r.model = g; r.worker = 0;
             r.order = st.next_order + k;
             tb.recs[mem_id[k]] = r;
         }

@@ -143,7 +143,7 @@ __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const 
             const int64_t em = shfl_i64(emin0, apv[u] & 31);
             const bool in = k < n_inst, keep = in && !(dlv[u] < em);
             if (in && !keep) {
-                sp_req_rec r; r.status = SP_EXPIRED; r.round = round; r.model = -1; r.pad_ = 0; r.order = 0;
+                sp_req_rec r; r.status = SP_EXPIRED; r.round = round; r.model = -1; r.worker = 0; r.order = 0;
                 tb.recs[r0 + k] = r;
             }
             const unsigned mask = __ballot_sync(0xffffffffu, keep);
@@ -215,7 +215,7 @@ __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const 
             for (int a = 0; a < A; ++a) {
                 const int h = __shfl_sync(0xffffffffu, head, a), h2 = __shfl_sync(0xffffffffu, nh, a);
                 for (int k = h + lane; k < h2; k += 32) {
-                    sp_req_rec r; r.status = SP_EXPIRED; r.round = round; r.model = -1; r.pad_ = 0; r.order = 0;
+                    sp_req_rec r; r.status = SP_EXPIRED; r.round = round; r.model = -1; r.worker = 0; r.order = 0;
                     tb.recs[r0 + (s_ida[k] & 0xFFFFFFu)] = r;
                 }
                 exp_since += h2 - h;
@@ -323,7 +323,7 @@ __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const 
         const int bp = bsz < na ? bsz : na;
         const int64_t e = shfl_i64(base_e, g & 31) + shfl_i64(my_be, g & 31) * (int64_t)bp;
         for (int k = lane; k < bp; k += 32) {
-            sp_req_rec r; r.status = SP_SCHEDULED; r.round = round; r.model = g; r.pad_ = 0; r.order = next_order + k;
+            sp_req_rec r; r.status = SP_SCHEDULED; r.round = round; r.model = g; r.worker = 0; r.order = next_order + k;
             tb.recs[r0 + (mida[k] & 0xFFFFFFu)] = r;
         }
         if (lane == 0 && sp.rounds_out && rounds_done < sp.cap) {
