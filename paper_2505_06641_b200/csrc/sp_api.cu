@@ -23,6 +23,8 @@ using namespace sp;
 namespace {
 
 constexpr double kDefaultGuardUtility = 2e-5, kDefaultGuardPriority = 2e-6;
+constexpr int64_t kDeferMinRows = 4096;   // single instances above this size get the grid-wide fp64 pass queued behind k_sched
+constexpr int kDeferExactRows = 512;      // rows a block re-scores by itself before it asks for that pass
 constexpr size_t kMaxSegments = 4096;   // sp_score calls that may build one request table
 
 struct Buf {                     // a device allocation that only grows
@@ -499,7 +501,8 @@ sp_status policy_prologue(sp_ctx *c, const char *who, GroupParams *gp, bool use_
         SP_CUDA(c, cudaFuncSetAttribute(k_exact_all, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         int64_t blocks = (n + warps - 1) / warps;
         if (blocks > (int64_t)c->n_sms * 8) blocks = (int64_t)c->n_sms * 8;
-        k_exact_all<<<(unsigned)blocks, warps * 32, smem, c->stream>>>(P, c->tb, (int32_t *)c->labels.p, (const int *)c->flags.p);
+        k_exact_all<<<(unsigned)blocks, warps * 32, smem, c->stream>>>(P, c->tb, (int32_t *)c->labels.p, (const int *)c->flags.p,
+                                                                       nullptr, nullptr);
         SP_TRY(launched(c, "k_exact_all"));
         c->have_exact_all = true;
     }
@@ -788,7 +791,7 @@ sp_status sp_reset(sp_ctx *c) {
     SP_CUDA(c, cudaSetDevice(c->device));
     k_state_reset<<<(c->P.I + 255) / 256, 256, 0, c->stream>>>((InstState *)c->state.p, c->P.I, 1);
     SP_TRY(launched(c, "k_state_reset"));
-    SP_CUDA(c, cudaMemsetAsync((int *)c->flags.p + 1, 0, sizeof(int), c->stream));
+    SP_CUDA(c, cudaMemsetAsync((int *)c->flags.p + 1, 0, 3 * sizeof(int), c->stream));
     SP_CUDA(c, cudaMemsetAsync(c->stats.p, 0, 4 * sizeof(unsigned long long), c->stream));
     drop_table(c);
     return SP_OK;
@@ -883,6 +886,7 @@ static sp_status score_impl(sp_ctx *c, int64_t n, const void *feats, const int32
 
     SP_CUDA(c, cudaMemsetAsync(tv.cnt, 0, nkeys * 4, c->stream));
     SP_CUDA(c, cudaMemsetAsync(tv.cursor, 0, nkeys * 4, c->stream));
+    SP_CUDA(c, cudaMemsetAsync((int *)c->flags.p + 2, 0, 2 * sizeof(int), c->stream));   // the new rows have no fp64 scores yet
     const unsigned gb = (unsigned)((n + 255) / 256);
     if (n > 0) {
         k_group_count<<<gb, 256, 0, c->stream>>>(P, tv, c->opt.trace_mode, (int *)c->flags.p,
@@ -1057,8 +1061,27 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
         sp.presorted = 1;
     }
     if (max_rounds > 0) c->sched_started = true;
+    // One large instance: a near-tie between group priorities may need the fp64 scores of every live request.  Beyond a
+    // few hundred rows the block stops before that round; the whole GPU then scores the rows that are not cached yet and
+    // a second launch resumes the instance (both return at once when the first launch did not ask for them).
+    const bool defer = P.I == 1 && c->tb.n > kDeferMinRows && max_rounds > 0;
+    sp.defer_exact_rows = defer ? kDeferExactRows : 0;
     sched_kernel<<<P.I, nt, L.end, c->stream>>>(sp);
     SP_TRY(launched(c, "k_sched"));
+    if (defer) {
+        int warps = 8;
+        while (warps > 1 && (size_t)warps * P.C * 8 > 200 * 1024) warps >>= 1;
+        const size_t smem = (size_t)warps * P.C * 8;
+        SP_CUDA(c, cudaFuncSetAttribute(k_exact_all, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        int64_t blocks = (c->tb.n + warps - 1) / warps;
+        if (blocks > (int64_t)c->n_sms * 8) blocks = (int64_t)c->n_sms * 8;
+        k_exact_all<<<(unsigned)blocks, warps * 32, smem, c->stream>>>(P, c->tb, nullptr, (const int *)c->flags.p,
+                                                                       (const int *)c->flags.p + 2, (unsigned long long *)c->stats.p);
+        SP_TRY(launched(c, "k_exact_all"));
+        sp.only_handed = 1; sp.presorted = 0;
+        sched_kernel<<<P.I, nt, L.end, c->stream>>>(sp);
+        SP_TRY(launched(c, "k_sched"));
+    }
     return mark(c, c->ev_sched);
 }
 

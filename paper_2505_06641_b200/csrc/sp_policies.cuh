@@ -21,15 +21,20 @@ constexpr int kExhMaxGroups = 8;            // groups the exhaustive branch acce
 
 // ------------------------------------------------------------------------------------------------ fp64 scores of all rows
 // One warp per request; zrow scratch in dynamic shared memory: [warps per block][C] doubles.
-__global__ void k_exact_all(DevProfiles P, DevTable tb, int32_t *labels, const int *flags) {
+// gate (optional): the pass runs only when *gate is set (a scheduler asked for it), and skips rows already cached.
+__global__ void k_exact_all(DevProfiles P, DevTable tb, int32_t *labels, const int *flags, const int *gate, unsigned long long *stats) {
     extern __shared__ __align__(16) unsigned char dyn[];
-    if (flags[1]) return;
+    if (flags[1] || (gate && !*gate)) return;
     const int warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     double *zrow = reinterpret_cast<double *>(dyn) + (size_t)warp * P.C;
+    unsigned long long done = 0;
     for (int64_t id = (int64_t)blockIdx.x * nwarps + warp; id < tb.n; id += (int64_t)gridDim.x * nwarps) {
+        if (gate && tb.exact[id]) continue;
         const int inst = tb.instance ? tb.instance[id] : 0;
         exact_row_core(P, tb, inst, id, zrow, labels ? labels + id : nullptr);
+        ++done;
     }
+    if (stats && done && (threadIdx.x & 31) == 0) atomicAdd(&stats[3], done);
 }
 
 // ------------------------------------------------------------------------------------------------ group queues

@@ -48,6 +48,12 @@ struct SchedParams {
     int bmax;                   // largest allowed batch size
     int zbuf_warps;             // zbuf rows per instance
     int presorted;              // 1: sort_scratch already holds the sorted keys of the whole (single) instance
+    // A near-tie between group priorities re-scores every live request of the contending groups in fp64.  One block
+    // does that for a few hundred rows; beyond defer_exact_rows (0 = never) it stops before the round instead, marks the
+    // instance (started = 2, handed = rounds done in this call) and raises flags[2]: the host has a grid-wide fp64 pass
+    // and a second launch with only_handed = 1 queued behind this kernel, which then finds every row cached.
+    int defer_exact_rows;
+    int only_handed;            // 1: continue instances that were handed over within this call, leave the others alone
 };
 
 __device__ __forceinline__ bool key_less(const SortKey &a, const SortKey &b) {
@@ -339,6 +345,10 @@ __device__ void sched_instance(const SchedParams &sp, const int inst) {
     if (tid == 0) st = sp.state[inst];
     if (tid <= A) s_base[tid] = tb.qstart[(int64_t)inst * A + tid];
     __syncthreads();
+    if (sp.only_handed) {
+        if (st.started != 2) return;            // this call's first launch finished the instance's work
+        if (tid == 0) { sp.flags[2] = 0; sp.flags[3] = 1; }   // the grid-wide pass has run: every row of the table is cached
+    }
 
     const double tau = P.tau;
     const int64_t reref_ns = tau > 1e8 ? INT64_MAX : (int64_t)(32.0 * tau * 1e9);   // exp((T - Tref)/tau) stays below e^32
@@ -650,6 +660,17 @@ __device__ void sched_instance(const SchedParams &sp, const int inst) {
         }
         __syncthreads();
         int round_exact = 0;
+        if (s_exactP && sp.defer_exact_rows > 0 && !sp.flags[3]) {
+            int64_t rows = 0;
+            for (int a = 0; a < A; ++a) rows += s_contend[a] ? st.tail[a] - st.head[a] : 0;
+            if (rows > sp.defer_exact_rows) {   // too many rows for one block: leave them to the whole GPU and resume
+                __syncthreads();
+                if (tid == 0) { st.started = 2; st.handed = rounds_done; sp.flags[2] = 1; }
+                __syncthreads();
+                finished = true;
+                break;
+            }
+        }
         if (s_exactP) {                        // near-tie between groups: decide on fp64 scores
             for (int a = 0; a < A; ++a) {
                 if (!s_contend[a]) continue;

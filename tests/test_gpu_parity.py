@@ -359,3 +359,16 @@ def test_zero_guards_select_the_defaults():
     ses.close()
     assert np.array_equal(ref.reqs, got.reqs)
     assert got.stats["exact_utility"] + got.stats["exact_priority"] == ref.stats["exact_utility"] + ref.stats["exact_priority"]
+
+
+@pytest.mark.parametrize("name,kw", [("C2", dict(n_requests=20000)), ("C5", dict(n_requests=20000)),
+                                     ("C3", dict(n_requests=6000, n_classes=200, feat_dim=256))])
+def test_near_ties_in_one_large_instance_are_rescored_by_the_whole_gpu(name, kw):
+    """Guards of 1.0 make every round a near-tie between groups, which needs the fp64 scores of every live request.  In a
+    large single instance that is thousands of rows: the block stops before the round, the whole GPU scores the rows,
+    and the rounds resume within the same call.  Same schedule as the oracle, and the rows are scored once."""
+    w = synth.make_workload(name, **kw)
+    s, od, res = _both(w, guards=(1.0, 1.0))
+    check_schedule(w, res, od)
+    assert res.stats["exact_priority"] > 0
+    assert 0 < res.stats["exact_rows"] <= w.n_requests
