@@ -12,7 +12,9 @@
 // contraction fused (running sum of 2^z * recall_j), flash-attention style; the two accumulators alternate so the
 // epilogue of a chunk overlaps the MMAs of the next one.
 //   * A operand: requests of a group are not contiguous, so 4 producer warps gather their rows with 16-byte
-//     cp.async copies into the swizzled slab (thread = row).
+//     cp.async copies into the swizzled slab.  Eight consecutive lanes copy the eight 16-byte pieces of one row's
+//     128 bytes, so every warp instruction asks for four whole 128-byte lines (one lane per row, eight instructions
+//     each touching 32 different lines, measured 1.8 x slower on the 2 GB trace workload and 1.3 x on C3).
 //   * B operand: the head is transposed once, when the profiles are loaded, into a K-major image
 //     Wt[(instance, application, label)][feature]; TMA tiles of NC labels x one slab of features stream from it
 //     (L2 resident).  The chunk's recall rows and bias arrive by TMA as well.
@@ -94,7 +96,7 @@ struct GCfg {
     static constexpr int bias = rtab + 2 * RBytes;                            // [2][NC] floats
     static constexpr int merge = bias + 2 * BiasSlot;                        // [EpiGroups - 1][128][kMergeFloats]
     static constexpr int bars = (merge + (EpiGroups - 1) * kGRows * kMergeFloats * 4 + 15) & ~15;
-    static constexpr int n_bars = 2 * kGMaxA + 2 * kGMaxB + 8 + 3;
+    static constexpr int n_bars = 3 * kGMaxA + 2 * kGMaxB + 8 + 3;
     static constexpr int misc = bars + n_bars * 8;
     static constexpr int end = misc + 16;
     static constexpr int bytes = end + 1024;
@@ -111,6 +113,8 @@ __device__ __forceinline__ constexpr int gbar_r_free(int b) { return kGBar2 + 6 
 constexpr int kGBarMergeReady = kGBar2 + 8;
 constexpr int kGBarMergeDone = kGBar2 + 9;
 constexpr int kGBarDrain = kGBar2 + 10;
+// fp32: every producer thread's copies of A stage s have landed (the threads then read rows other threads copied)
+__device__ __forceinline__ constexpr int gbar_landed(int s) { return kGBar2 + 11 + s; }
 
 struct GParams {
     DevProfiles P;
@@ -224,7 +228,9 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
     const int n_ch = (C + kNC - 1) / kNC;                  // label chunks
 
     if (tid == 0) {
-        for (int s = 0; s < kAStages; ++s) { mbar_init(bar(gbar_full_a(s)), kGAThreads); mbar_init(bar(gbar_free_a(s)), 1); }
+        for (int s = 0; s < kAStages; ++s) {
+            mbar_init(bar(gbar_full_a(s)), kGAThreads); mbar_init(bar(gbar_free_a(s)), 1); mbar_init(bar(gbar_landed(s)), kGAThreads);
+        }
         for (int s = 0; s < kBStages; ++s) { mbar_init(bar(gbar_full_b(s)), 1); mbar_init(bar(gbar_free_b(s)), 1); }
         for (int b = 0; b < 2; ++b) {
             mbar_init(bar(gbar_acc_full(b)), 1); mbar_init(bar(gbar_acc_empty(b)), kGEpiThreads);
@@ -330,14 +336,19 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
     } else if (warp < kGEpiWarp0) {
         // ================================================================ A producers: gather the rows of the tile
         const int aquad = warp & 3, row = aquad * 32 + lane;  // fp32: the thread's row is also its tensor-memory lane
+        const int pt = (warp - kGAWarp0) * 32 + lane;          // copies: piece pt & 7 of rows (pt >> 3) + 16 i, i = 0..7
+        const int pj = pt & 7, pr0 = pt >> 3;
         constexpr int kEsz = F32 ? 4 : 2, kPiece = 16 / kEsz; // bytes per feature, features per 16-byte piece
         uint32_t slab_seq = 0;
         bool ok = true;
         uint32_t issued = 0, signalled = 0;                    // slabs whose copies were issued / reported complete
-        // The copies of stage ps have landed: (fp32) store this row's x_lo into the stage's tensor-memory slot, then
-        // tell the MMA issuer that the A operand of the stage is complete.
-        auto signal = [&](int ps) {
+        // This thread's copies of stage ps have landed.  fp32: once every producer's have (the row a thread reads was
+        // copied by eight others), store the row's x_lo into the stage's tensor-memory slot.  Then tell the MMA issuer
+        // that the A operand of the stage is complete.
+        auto signal = [&](int ps, uint32_t use) -> bool {
             if (F32) {
+                mbar_arrive(bar(gbar_landed(ps)));
+                if (!warp_wait(bar(gbar_landed(ps)), use & 1, abort_flag)) return false;
                 const unsigned char *xrow = sm + GSmem::a_ring + ps * kASlabBytes + row * 128;
                 uint32_t v[32];
 #pragma unroll
@@ -357,38 +368,46 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
             }
             fence_proxy_async();
             mbar_arrive(bar(gbar_full_a(ps)));
+            return true;
         };
         for (int t = blockIdx.x; t < prm.n_tiles && ok; t += gridDim.x) {
             const int4 d = prm.tiles[t];
             if (d.x < 0) continue;
-            const int64_t req = tb.perm[d.y + (row < d.z ? row : 0)];
-            const unsigned char *src = (const unsigned char *)tb.feats + req * D * kEsz;
+            const unsigned char *srcs[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int r = pr0 + 16 * i;
+                srcs[i] = (const unsigned char *)tb.feats + tb.perm[d.y + (r < d.z ? r : 0)] * D * kEsz;
+            }
             for (int ch = 0; ch < n_ch && ok; ++ch) {
                 for (int ks = 0; ks < n_ks; ++ks, ++slab_seq) {
                     const int s = slab_seq % kAStages;
                     const uint32_t use = slab_seq / kAStages;
                     if (use > 0 && !warp_wait(bar(gbar_free_a(s)), (use - 1) & 1, abort_flag)) { ok = false; break; }
-                    const uint32_t dst = base + GSmem::a_ring + s * kASlabBytes + row * 128;
-                    const int k0 = ks * kKSlab;
+                    const int kk = ks * kKSlab + pj * kPiece;
+                    const int left = (D - kk) * kEsz;          // bytes of a row that exist from this piece on
+                    const uint32_t nbytes = left >= 16 ? 16u : left > 0 ? (uint32_t)left : 0u;
+                    const int koff = (kk < D ? kk : 0) * kEsz;
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const int kk = k0 + j * kPiece;
-                        const int left = (D - kk) * kEsz;      // bytes of the row that exist from this piece on
-                        cp_async16_zfill(dst + ((j ^ (row & 7)) << 4), src + (kk < D ? kk : 0) * kEsz,
-                                         left >= 16 ? 16u : left > 0 ? (uint32_t)left : 0u);
+                    for (int i = 0; i < 8; ++i) {
+                        const int r = pr0 + 16 * i;
+                        cp_async16_zfill(base + GSmem::a_ring + s * kASlabBytes + r * 128 + ((pj ^ (r & 7)) << 4), srcs[i] + koff, nbytes);
                     }
                     cp_async_commit();
                     ++issued;
                     if (issued - signalled > (uint32_t)G::ADepth) {    // keep ADepth slabs in flight: the oldest has landed
                         cp_async_wait<G::ADepth>();
-                        signal((int)(signalled % kAStages));
+                        if (!signal((int)(signalled % kAStages), signalled / kAStages)) { ok = false; break; }
                         ++signalled;
                     }
                 }
             }
         }
         cp_async_wait<0>();
-        while (ok && signalled < issued) { signal((int)(signalled % kAStages)); ++signalled; }
+        while (ok && signalled < issued) {
+            if (!signal((int)(signalled % kAStages), signalled / kAStages)) break;
+            ++signalled;
+        }
     } else {
         // ================================================================ epilogue warps (one row per thread, a quarter of the columns)
         const int eg = (warp - kGEpiWarp0) >> 2;               // column group of every chunk this warpgroup reads
