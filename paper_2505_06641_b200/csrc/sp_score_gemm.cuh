@@ -420,6 +420,7 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
         bool ok = true;
         constexpr int kGW = kNC / kGEpiGroups;                     // columns of a chunk per epilogue group
         constexpr int kBlk = kGEpiBlk;
+        constexpr float kMScale = F32 ? 1.f : kLog2e;                // units of the running maximum: base-2 (fp32) or natural (bf16) logits
         static_assert(kNC % (4 * kGEpiGroups) == 0, "a group's first column must keep 16-byte alignment in the tables");
         for (int t = blockIdx.x; t < prm.n_tiles && ok; t += gridDim.x) {
             const int4 d = prm.tiles[t];
@@ -452,26 +453,36 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
                                 z[c] = fmaf(bv.x, kLog2e, z[c]); z[c + 1] = fmaf(bv.y, kLog2e, z[c + 1]);
                                 z[c + 2] = fmaf(bv.z, kLog2e, z[c + 2]); z[c + 3] = fmaf(bv.w, kLog2e, z[c + 3]);
                             } else {
-                                z[c] = (z[c] + bv.x) * kLog2e; z[c + 1] = (z[c + 1] + bv.y) * kLog2e;
-                                z[c + 2] = (z[c + 2] + bv.z) * kLog2e; z[c + 3] = (z[c + 3] + bv.w) * kLog2e;
+                                z[c] += bv.x; z[c + 1] += bv.y; z[c + 2] += bv.z; z[c + 3] += bv.w;   // natural units; log2(e) goes into the exponent's FMA
                             }
                         }
                     }
+                    if (c_base + col0 + kBlk <= C && col0 + kBlk <= col_end) {   // whole block valid (uniform): no masking
 #pragma unroll
-                    for (int c = 0; c < kBlk; ++c) {
-                        if (c_base + col0 + c >= C || col0 + c >= col_end) z[c] = -INFINITY;
-                        bm = fmaxf(bm, z[c]);
+                        for (int c = 0; c < kBlk; ++c) bm = fmaxf(bm, z[c]);
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < kBlk; ++c) {
+                            if (c_base + col0 + c >= C || col0 + c >= col_end) z[c] = -INFINITY;
+                            bm = fmaxf(bm, z[c]);
+                        }
                     }
                     if (bm > run_m) {                                      // rescale what has been summed so far
-                        const float sc = exp2_unit(run_m - bm);            // 0 for the first block (run_m = -inf)
+                        const float sc = exp2_unit((run_m - bm) * kMScale); // 0 for the first block (run_m = -inf)
                         run_s *= sc;
 #pragma unroll
                         for (int j = 0; j < kMaxModelsPerApp; ++j) racc[j] *= sc;
                         run_m = bm;
                     }
                     float ps = 0.f;
+                    if (F32) {
 #pragma unroll
-                    for (int c = 0; c < kBlk; ++c) { z[c] = exp2_unit(z[c] - run_m); ps += z[c]; }
+                        for (int c = 0; c < kBlk; ++c) { z[c] = exp2_unit(z[c] - run_m); ps += z[c]; }
+                    } else {
+                        const float nm = -run_m * kLog2e;
+#pragma unroll
+                        for (int c = 0; c < kBlk; ++c) { z[c] = exp2_unit(fmaf(z[c], kLog2e, nm)); ps += z[c]; }
+                    }
                     run_s += ps;
                     // recall contraction with two-wide FMAs: label pairs (c, c + 1) of a model's row against the pair of
                     // numerators; the two halves of the accumulator are added once per block of labels
@@ -517,7 +528,7 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
                 float mm = run_m;
 #pragma unroll
                 for (int g = 0; g < kGEpiGroups - 1; ++g) mm = fmaxf(mm, merge_all[(g * kGRows + row) * kMergeFloats]);
-                const float s0 = run_m == -INFINITY ? 0.f : exp2_unit(run_m - mm);
+                const float s0 = run_m == -INFINITY ? 0.f : exp2_unit((run_m - mm) * kMScale);
                 float tot = run_s * s0;
 #pragma unroll
                 for (int j = 0; j < kMaxModelsPerApp; ++j) racc[j] *= s0;
@@ -525,7 +536,7 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
                 for (int g = 0; g < kGEpiGroups - 1; ++g) {
                     const float *mg = merge_all + (g * kGRows + row) * kMergeFloats;
                     const float om = mg[0];
-                    const float sg = om == -INFINITY ? 0.f : exp2_unit(om - mm);
+                    const float sg = om == -INFINITY ? 0.f : exp2_unit((om - mm) * kMScale);
                     tot = fmaf(mg[1], sg, tot);
 #pragma unroll
                     for (int j = 0; j < kMaxModelsPerApp; ++j) racc[j] = fmaf(mg[2 + j], sg, racc[j]);
