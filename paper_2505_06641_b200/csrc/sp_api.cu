@@ -63,7 +63,7 @@ struct sp_ctx {
     // profile buffers
     Buf W, bias, recall, prior, prior_dot, prior_sum, lat_alpha, lat_beta, swap;
     // per-instance state and scratch
-    Buf state, zbuf, flags, stats, cnt, gstart, cursor, small_start, tiled_start, small_tiles, scan_partial, wt_image, gemm_tiles, gemm_counter;
+    Buf state, zbuf, flags, stats, cnt, gstart, cursor, small_start, tiled_start, small_tiles, scan_partial, wt_image, gemm_tiles, gemm_counter, gemm_partial, gemm_count;
     // per-request buffers
     Buf acc32, v32, acc64, v64, exact, recs, perm, q_id0, q_id1, q_dl0, q_dl1, q_pw0, q_pw1, sort_scratch;
     // requests appended to a scored table: the context's own copies of application / arrival / deadline, the list of
@@ -345,8 +345,18 @@ sp_status score_rows(sp_ctx *c, const DevTable &tv, float *acc_out) {
             default: SP_TRY(launch_small<32>(c, tv, grid, acc_out)); break;
         }
     } else if (c->gemm_on) {
-        gemm::GParams gp{P, tv, (const int4 *)c->gemm_tiles.p, n_tiles, c->gemm_cp, P.I * P.A * c->gemm_cp, acc_out, (int *)c->flags.p};
-        const int ggrid = n_tiles < c->n_sms ? n_tiles : c->n_sms;
+        gemm::GParams gp{P, tv, (const int4 *)c->gemm_tiles.p, n_tiles, c->gemm_cp, P.I * P.A * c->gemm_cp, acc_out, (int *)c->flags.p,
+                         1, nullptr, nullptr};
+        // few tiles per block and at least two label chunks: halves of tiles as work items (see GParams::split)
+        const int nc = c->gemm_f32 ? gemm::GCfg<true>::NC : gemm::GCfg<false>::NC;
+        if ((P.C + nc - 1) / nc >= 2 && n_tiles < 8 * c->n_sms) {
+            SP_TRY(ensure(c, c->gemm_partial, (size_t)n_tiles * 2 * gemm::kMergeFloats * gemm::kGRows * 4));
+            SP_TRY(ensure(c, c->gemm_count, (size_t)n_tiles * gemm::kGRows * 4));
+            SP_CUDA(c, cudaMemsetAsync(c->gemm_count.p, 0, (size_t)n_tiles * gemm::kGRows * 4, c->stream));
+            gp.split = 2; gp.partial = (float *)c->gemm_partial.p; gp.part_count = (int *)c->gemm_count.p;
+        }
+        const int n_items = n_tiles * gp.split;
+        const int ggrid = n_items < c->n_sms ? n_items : c->n_sms;
         if (c->gemm_f32) {
             SP_CUDA(c, cudaFuncSetAttribute(gemm::k_score_gemm<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, gemm::GCfg<true>::bytes));
             gemm::k_score_gemm<true><<<ggrid, gemm::GCfg<true>::Threads, gemm::GCfg<true>::bytes, c->stream>>>(c->wt_map, c->r_map, c->b_map, gp);
@@ -560,7 +570,7 @@ void sp_destroy(sp_ctx *c) {
     drain_events(c->ev_sched, &dummy);
     Buf *all[] = {&c->W, &c->bias, &c->recall, &c->prior, &c->prior_dot, &c->prior_sum, &c->lat_alpha, &c->lat_beta,
                   &c->swap, &c->state, &c->zbuf, &c->flags, &c->stats, &c->cnt, &c->gstart, &c->cursor,
-                  &c->small_start, &c->tiled_start, &c->small_tiles, &c->scan_partial, &c->wt_image, &c->gemm_tiles, &c->gemm_counter, &c->acc32, &c->v32, &c->acc64, &c->v64, &c->exact, &c->recs,
+                  &c->small_start, &c->tiled_start, &c->small_tiles, &c->scan_partial, &c->wt_image, &c->gemm_tiles, &c->gemm_counter, &c->gemm_partial, &c->gemm_count, &c->acc32, &c->v32, &c->acc64, &c->v64, &c->exact, &c->recs,
                   &c->perm, &c->q_id0, &c->q_id1, &c->q_dl0, &c->q_dl1, &c->q_pw0, &c->q_pw1, &c->sort_scratch,
                   &c->h_feats, &c->h_app, &c->h_arrival, &c->h_deadline, &c->h_instance, &c->h_t0, &c->h_loaded,
                   &c->h_rounds, &c->h_ndone, &c->t_app, &c->t_arrival, &c->t_deadline, &c->a_cnt, &c->a_cursor,

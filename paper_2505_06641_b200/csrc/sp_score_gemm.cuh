@@ -125,6 +125,13 @@ struct GParams {
     int lo_row0;             // fp32: first row of the W_lo half of the image (= number of W_hi rows)
     float *acc_out;
     int *flags;
+    // Work items.  split = 1: an item is a tile.  split = 2: an item is half of a tile's label chunks, so that a launch
+    // of few tiles per block still spreads evenly (512 tiles on 148 blocks: 4 tiles on the busiest block, but 7 of 1,024
+    // halves); the two halves of a row meet in global memory: each writes its running (maximum, sum, sums per model) to
+    // `partial`, and the one that comes second (per-row counter `part_count`, zeroed before the launch) merges and stores.
+    int split;
+    float *partial;          // [n_tiles][2][kMergeFloats][128]
+    int *part_count;         // [n_tiles][128]
 };
 
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n.
@@ -226,6 +233,7 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
     const int A = P.A, C = P.C, D = P.D, Cp = prm.Cp;
     const int n_ks = (D + kKSlab - 1) / kKSlab;            // feature slabs
     const int n_ch = (C + kNC - 1) / kNC;                  // label chunks
+    const int S = prm.split, n_items = prm.n_tiles * S;    // work items: tiles, or halves of a tile's label chunks
 
     if (tid == 0) {
         for (int s = 0; s < kAStages; ++s) {
@@ -261,12 +269,13 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
         if (lane == 0) {
             uint32_t slab_seq = 0, chunk_seq = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < prm.n_tiles && ok; t += gridDim.x) {
+            for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+                const int t = it / S, hf = it - t * S;
                 const int4 d = prm.tiles[t];
                 if (d.x < 0) continue;
                 const int inst = d.x / A, a = d.x - inst * A;
                 const int wrow0 = d.x * Cp;                              // first row of this head in the image
-                for (int ch = 0; ch < n_ch && ok; ++ch, ++chunk_seq) {
+                for (int ch = hf * n_ch / S; ch < (hf + 1) * n_ch / S && ok; ++ch, ++chunk_seq) {
                     const int rb = chunk_seq & 1;
                     const uint32_t ruse = chunk_seq >> 1;
                     if (ruse > 0 && !mbar_wait(bar(gbar_r_free(rb)), (ruse - 1) & 1, abort_flag)) { ok = false; break; }
@@ -290,10 +299,11 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
         if (lane == 0) {
             uint32_t slab_seq = 0, chunk_seq = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < prm.n_tiles && ok; t += gridDim.x) {
+            for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+                const int t = it / S, hf = it - t * S;
                 const int4 d = prm.tiles[t];
                 if (d.x < 0) continue;
-                for (int ch = 0; ch < n_ch && ok; ++ch, ++chunk_seq) {
+                for (int ch = hf * n_ch / S; ch < (hf + 1) * n_ch / S && ok; ++ch, ++chunk_seq) {
                     const uint32_t b = chunk_seq & 1, acc_use = chunk_seq >> 1;
                     if (acc_use > 0 && !mbar_wait(bar(gbar_acc_empty(b)), (acc_use - 1) & 1, abort_flag)) { ok = false; break; }
                     tc_fence_after();
@@ -370,7 +380,8 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
             mbar_arrive(bar(gbar_full_a(ps)));
             return true;
         };
-        for (int t = blockIdx.x; t < prm.n_tiles && ok; t += gridDim.x) {
+        for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+            const int t = it / S, hf = it - t * S;
             const int4 d = prm.tiles[t];
             if (d.x < 0) continue;
             const unsigned char *srcs[8];
@@ -379,7 +390,7 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
                 const int r = pr0 + 16 * i;
                 srcs[i] = (const unsigned char *)tb.feats + tb.perm[d.y + (r < d.z ? r : 0)] * D * kEsz;
             }
-            for (int ch = 0; ch < n_ch && ok; ++ch) {
+            for (int ch = hf * n_ch / S; ch < (hf + 1) * n_ch / S && ok; ++ch) {
                 for (int ks = 0; ks < n_ks; ++ks, ++slab_seq) {
                     const int s = slab_seq % kAStages;
                     const uint32_t use = slab_seq / kAStages;
@@ -422,7 +433,8 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
         constexpr int kBlk = kGEpiBlk;
         constexpr float kMScale = F32 ? 1.f : kLog2e;                // units of the running maximum: base-2 (fp32) or natural (bf16) logits
         static_assert(kNC % (4 * kGEpiGroups) == 0, "a group's first column must keep 16-byte alignment in the tables");
-        for (int t = blockIdx.x; t < prm.n_tiles && ok; t += gridDim.x) {
+        for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+            const int t = it / S, hf = it - t * S;
             const int4 d = prm.tiles[t];
             if (d.x < 0) continue;
             const int inst = d.x / A, a = d.x - inst * A;
@@ -430,7 +442,7 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
             float run_m = -INFINITY, run_s = 0.f, racc[kMaxModelsPerApp];
 #pragma unroll
             for (int j = 0; j < kMaxModelsPerApp; ++j) racc[j] = 0.f;
-            for (int ch = 0; ch < n_ch && ok; ++ch, ++chunk_seq) {
+            for (int ch = hf * n_ch / S; ch < (hf + 1) * n_ch / S && ok; ++ch, ++chunk_seq) {
                 const uint32_t b = chunk_seq & 1, par = (chunk_seq >> 1) & 1;
                 if (!warp_wait(bar(gbar_r_full(b)), par, abort_flag)) { ok = false; break; }
                 if (!warp_wait(bar(gbar_acc_full(b)), par, abort_flag)) { ok = false; break; }
@@ -541,8 +553,30 @@ k_score_gemm(const __grid_constant__ CUtensorMap wt_map, const __grid_constant__
 #pragma unroll
                     for (int j = 0; j < kMaxModelsPerApp; ++j) racc[j] = fmaf(mg[2 + j], sg, racc[j]);
                 }
+                bool last = true;
+                if (S > 1) {
+                    // this half's state of the row goes to global memory; the half that arrives second finds the other
+                    // one's there (fence before the counter on both sides) and finishes the row
+                    float *mine = prm.partial + ((size_t)(t * 2 + hf) * kMergeFloats) * kGRows + row;
+                    mine[0] = mm; mine[kGRows] = tot;
+#pragma unroll
+                    for (int j = 0; j < kMaxModelsPerApp; ++j) mine[(2 + j) * kGRows] = racc[j];
+                    __threadfence();
+                    last = atomicAdd(prm.part_count + (size_t)t * kGRows + row, 1) == 1;
+                    if (last) {
+                        __threadfence();
+                        const float *other = prm.partial + ((size_t)(t * 2 + (1 - hf)) * kMergeFloats) * kGRows + row;
+                        const float om = __ldcg(other), os = __ldcg(other + kGRows);
+                        const float m2 = fmaxf(mm, om);
+                        const float sa = mm == -INFINITY ? 0.f : exp2_unit((mm - m2) * kMScale);
+                        const float sb = om == -INFINITY ? 0.f : exp2_unit((om - m2) * kMScale);
+                        tot = fmaf(os, sb, tot * sa);
+#pragma unroll
+                        for (int j = 0; j < kMaxModelsPerApp; ++j) racc[j] = fmaf(__ldcg(other + (2 + j) * kGRows), sb, racc[j] * sa);
+                    }
+                }
                 const float inv = 1.f / tot;
-                const bool valid = row < d.z;
+                const bool valid = last && row < d.z;
                 const int64_t req = tb.perm[d.y + (valid ? row : 0)];
                 float *dst = tb.acc32 + req * Mmax;
                 float *dst2 = prm.acc_out ? prm.acc_out + req * Mmax : nullptr;
