@@ -88,6 +88,7 @@ struct GCfg {
     static constexpr int BiasBytes = NC * 4;
     static constexpr int BiasSlot = (BiasBytes + 127) & ~127;     // TMA destinations are 128-byte aligned
     static_assert(RBytes % 128 == 0, "recall buffers must keep the 128-byte alignment of TMA destinations");
+    static_assert(AStages <= kGMaxA && BStages <= kGMaxB, "the barrier table holds kGMaxA / kGMaxB stages");
     static constexpr int TmemLo = 2 * NC;                      // fp32: x_lo slots (32 columns per stage) after the accumulators
     // byte offsets from the 1024-byte aligned base
     static constexpr int a_ring = 0;                                          // [AStages] slabs of 128 rows
