@@ -1041,23 +1041,23 @@ sp_status sp_schedule_round(sp_ctx *c, int32_t max_rounds, sp_round_rec *rounds_
     // Batched mode, first call on a fresh table: one warp per instance takes every instance that fits its slice of
     // shared memory and, block-wide, the few it has to hand over; no k_sched launch is needed then.
     // (A call for zero rounds changes nothing: it goes to k_sched, which returns before touching any queue.)
-    if (P.I > 1 && !c->opt.trace_mode && !c->sched_started && c->tb.n > 0 && !P.any_soft && max_rounds > 0) {
+    if (P.I > 1 && !c->opt.trace_mode && !c->sched_started && c->tb.n > 0 && max_rounds > 0) {
         int64_t wcap = 32;
         while (wcap < (c->tb.n + P.I - 1) / P.I) wcap <<= 1;
-        const WarpSchedSmem W((int)wcap, P.Mmax, sp.bmax);
+        const WarpSchedSmem W((int)wcap, P.Mmax, sp.bmax, P.any_soft != 0);
         if (wcap <= 2048 && P.sumM <= 32 && W.end * kWarpSchedWarps <= 200 * 1024 && c->sched_threads == kWarpSchedWarps * 32) {
             const int wgrid = (P.I + kWarpSchedWarps - 1) / kWarpSchedWarps;
             // the block-wide scheduler runs inside the same kernel for the instances a warp hands over: its shared
             // memory is laid over the warps' slices
             const size_t wsmem = W.end * kWarpSchedWarps > L.end ? W.end * kWarpSchedWarps : L.end;
-            if (P.Mmax <= 8 && P.Mmax * P.nB <= 64 && P.A <= 4) {   // short unrolled loops for small model, batch-size and application sets
-                SP_CUDA(c, cudaFuncSetAttribute(k_sched_warp<8, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)wsmem));
-                k_sched_warp<8, 2><<<wgrid, kWarpSchedWarps * 32, wsmem, c->stream>>>(sp, (int)wcap);
-            } else {
-                SP_CUDA(c, cudaFuncSetAttribute(k_sched_warp<kMaxModelsPerApp, kMaxModelsPerApp * kMaxBatchSizes / 32>,
-                                                cudaFuncAttributeMaxDynamicSharedMemorySize, (int)wsmem));
-                k_sched_warp<kMaxModelsPerApp, kMaxModelsPerApp * kMaxBatchSizes / 32><<<wgrid, kWarpSchedWarps * 32, wsmem, c->stream>>>(sp, (int)wcap);
-            }
+            constexpr int kBigCpl = kMaxModelsPerApp * kMaxBatchSizes / 32;
+            void (*wk)(SchedParams, int);
+            if (P.Mmax <= 8 && P.Mmax * P.nB <= 64 && P.A <= 4)   // short unrolled loops for small model, batch-size and application sets
+                wk = P.any_soft ? k_sched_warp<8, 2, true> : k_sched_warp<8, 2, false>;
+            else
+                wk = P.any_soft ? k_sched_warp<kMaxModelsPerApp, kBigCpl, true> : k_sched_warp<kMaxModelsPerApp, kBigCpl, false>;
+            SP_CUDA(c, cudaFuncSetAttribute(wk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)wsmem));
+            wk<<<wgrid, kWarpSchedWarps * 32, wsmem, c->stream>>>(sp, (int)wcap);
             SP_TRY(launched(c, "k_sched_warp"));
             c->sched_started = true;
             return mark(c, c->ev_sched);

@@ -8,6 +8,8 @@
 // latency and swap profiles in lane registers, one global round trip per round (the accuracy rows of the
 // candidate members).  Requests that are already hopeless at the starting clock are retired before the sort, so
 // only the survivors are sorted.
+// Applications with a linear or sigmoid penalty (SOFT instantiation) sum Eq. 2 member by member, and their hopeless
+// requests leave from the queue head only, as in k_sched.
 // A warp takes an instance that has not started, is not in trace mode and fits the per-warp capacity.  The warp
 // path does not contain the fp64 re-evaluation of near-ties (which keeps it small): when the two best group
 // priorities or candidate utilities of a round are closer than the guard band, the warp writes its queues and
@@ -24,12 +26,16 @@ constexpr int kWarpSchedWarps = 4;          // instances per block
 constexpr int kWarpLoadChunk = 8;           // requests per lane loaded together at the start
 
 struct WarpSchedSmem {                      // per-warp byte offsets (8-byte aligned pieces)
-    size_t dl, pw, ida, pref, end;
-    __host__ __device__ WarpSchedSmem(int cap, int Mmax, int bmax) {
+    size_t dl, pw, ida, pref, arr, end;
+    __host__ __device__ WarpSchedSmem(int cap, int Mmax, int bmax, bool soft) {
         size_t o = 0;
         dl = o;   o += (size_t)cap * sizeof(int64_t);
+        arr = o;  o += soft ? (size_t)cap * sizeof(int64_t) : 0;   // arrival times by request index (soft penalties)
         pw = o;   o += (size_t)cap * sizeof(double);
-        pref = o; o += (size_t)Mmax * (bmax + 1) * sizeof(double);
+        // prefix sums (step penalty), or the members' fp32 accuracy rows and relative deadlines (soft penalties)
+        const size_t pref_bytes = (size_t)Mmax * (bmax + 1) * sizeof(double);
+        const size_t soft_bytes = (((size_t)bmax * Mmax * sizeof(float) + 7) & ~(size_t)7) + (size_t)bmax * sizeof(int64_t);
+        pref = o; o += pref_bytes > soft_bytes ? pref_bytes : soft_bytes;
         ida = o;  o += (size_t)cap * sizeof(uint32_t);          // (application << 24) | request index in the instance
         end = (o + 15) & ~(size_t)15;
     }
@@ -47,6 +53,24 @@ __device__ __forceinline__ int warp_sum_i32(int v) {
 }
 __device__ __forceinline__ int64_t shfl_i64(int64_t v, int src) {
     return (int64_t)__shfl_sync(0xffffffffu, (long long)v, src);
+}
+
+// 1 - gamma of Eq. 2 in fp32 for the warp path's candidate sums.  Both x = (e - d) / delta and 1 - x come from integer
+// differences, so the result keeps fp32 relative accuracy also where gamma is close to 1 (no cancellation): far inside
+// the guard band under which a round goes to the block-wide scheduler and its fp64 penalty.
+__device__ __forceinline__ float penalty_keep_f32(int kind, int64_t d, int64_t delta, int64_t e) {
+    if (kind == SP_PEN_STEP || delta <= 0) return d < e ? 0.f : 1.f;
+    if (e <= d) return 1.f;
+    if (e - d >= delta) return 0.f;
+    const float fd = (float)delta;
+    const float xm = __fdividef((float)(delta - (e - d)), fd);       // 1 - x
+    if (kind == SP_PEN_LINEAR) return xm;
+    const float r = __fdividef(xm, __fdividef((float)(e - d), fd));  // (1 - x) / x
+    const float r3 = r * r * r;
+    // close to x = 1 the fp64 definition 1 - 1 / (1 + r^3) is itself rounded at 1e-16 absolute; there the value is taken
+    // from that definition (rare: the request is about to become hopeless), elsewhere r^3 / (1 + r^3) in fp32
+    if (r3 < 1e-3f) return (float)__dsub_rn(1.0, penalty_gamma(kind, d, delta, e));
+    return r3 < 1e30f ? __fdividef(r3, 1.f + r3) : 1.f;
 }
 
 // Ascending (application, deadline, index) order of the packed keys.
@@ -84,13 +108,14 @@ __device__ __forceinline__ void warp_sort(int64_t *dl, uint32_t *ida, int n) {
 // MM bounds the models per application and CPL the candidates per lane (models x batch sizes / 32): the loops over
 // them are unrolled, and the small instantiation (which also stands for at most 4 applications) keeps the code of a
 // round short.
-template <int MM, int CPL>
+template <int MM, int CPL, bool SOFT>
 __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const int inst, unsigned char *mine) {
     const DevProfiles &P = sp.P;
     const DevTable &tb = sp.tb;
     const int lane = threadIdx.x & 31;
     const int A = P.A, nB = P.nB, Mmax = P.Mmax, bmax = sp.bmax, sumM = P.sumM;
-    const WarpSchedSmem L(cap, Mmax, bmax);
+    const WarpSchedSmem L(cap, Mmax, bmax, SOFT);
+    int64_t *s_arr = reinterpret_cast<int64_t *>(mine + L.arr);
     int64_t *s_dl = reinterpret_cast<int64_t *>(mine + L.dl);
     double *s_pw = reinterpret_cast<double *>(mine + L.pw);
     uint32_t *s_ida = reinterpret_cast<uint32_t *>(mine + L.ida);
@@ -113,6 +138,7 @@ __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const 
     const int my_batch = lane < nB ? P.batch[lane] : 0;
     const int b_min = __shfl_sync(0xffffffffu, my_batch, 0);
     const int my_m0 = my_mfirst, my_M = __shfl_down_sync(0xffffffffu, my_mfirst, 1) - my_mfirst;   // lane a < A
+    const int my_pen = (SOFT && lane < A) ? P.pen[lane] : SP_PEN_STEP;                             // lane a < A
 
     // lane a < A: earliest completion any candidate of application a can reach from the current clock and model
     auto emin_lane = [&]() -> int64_t {
@@ -136,12 +162,14 @@ __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const 
             const int k = k0 + u * 32 + lane;
             dlv[u] = k < n_inst ? tb.deadline[r0 + k] : 0;
             apv[u] = k < n_inst ? tb.app[r0 + k] : 0;
+            if (SOFT && k < n_inst) s_arr[k] = tb.arrival[r0 + k];
         }
 #pragma unroll
         for (int u = 0; u < kWarpLoadChunk; ++u) {
             const int k = k0 + u * 32 + lane;
             const int64_t em = shfl_i64(emin0, apv[u] & 31);
-            const bool in = k < n_inst, keep = in && !(dlv[u] < em);
+            const bool step_app = !SOFT || __shfl_sync(0xffffffffu, my_pen, apv[u] & 31) == SP_PEN_STEP;
+            const bool in = k < n_inst, keep = in && !(step_app && dlv[u] < em);
             if (in && !keep) {
                 sp_req_rec r; r.status = SP_EXPIRED; r.round = round; r.model = -1; r.worker = 0; r.order = 0;
                 tb.recs[r0 + k] = r;
@@ -207,9 +235,17 @@ __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const 
         const int64_t emin = emin_lane();
         int nh = head;
         if (lane < A && tail > head) {
-            int lo = head, hi = tail;
-            while (lo < hi) { const int mid = (lo + hi) >> 1; if (s_dl[mid] < emin) lo = mid + 1; else hi = mid; }
-            nh = lo;
+            if (!SOFT || my_pen == SP_PEN_STEP) {
+                int lo = head, hi = tail;
+                while (lo < hi) { const int mid = (lo + hi) >> 1; if (s_dl[mid] < emin) lo = mid + 1; else hi = mid; }
+                nh = lo;
+            } else {                              // soft penalty: the head leaves while it is hopeless
+                while (nh < tail) {
+                    const int64_t dl = s_dl[nh];
+                    if (!penalty_hopeless(my_pen, dl, dl - s_arr[s_ida[nh] & 0xFFFFFFu], emin)) break;
+                    ++nh;
+                }
+            }
         }
         if (warp_sum_i32(lane < A ? nh - head : 0) > 0) {
             for (int a = 0; a < A; ++a) {
@@ -249,6 +285,17 @@ __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const 
         const int m0 = __shfl_sync(0xffffffffu, my_m0, a), M = __shfl_sync(0xffffffffu, my_M, a), ncand = M * nB;
         const int64_t *mdl = s_dl + qh;                       // deadlines of the members, ascending
         const uint32_t *mida = s_ida + qh;
+        const int pen = SOFT ? __shfl_sync(0xffffffffu, my_pen, a) : SP_PEN_STEP;
+        float *s_acc = reinterpret_cast<float *>(pref);                                  // soft: [nb][Mmax]
+        int64_t *s_delta = reinterpret_cast<int64_t *>(reinterpret_cast<unsigned char *>(pref) +
+                                                       (((size_t)bmax * Mmax * sizeof(float) + 7) & ~(size_t)7));
+        if (SOFT && pen != SP_PEN_STEP) {          // Eq. 2 member by member: stage the rows and relative deadlines
+            for (int k = lane; k < nb; k += 32) {
+                const int64_t id = r0 + (int64_t)(mida[k] & 0xFFFFFFu);
+                s_delta[k] = mdl[k] - s_arr[mida[k] & 0xFFFFFFu];
+                for (int j = 0; j < M; ++j) s_acc[k * Mmax + j] = tb.acc32[id * Mmax + j];
+            }
+        } else {
         for (int j = lane; j < M; j += 32) pref[(size_t)j * (bmax + 1)] = 0.0;
         {
             double carry[MM];
@@ -276,6 +323,7 @@ __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const 
                 }
             }
         }
+        }
         __syncwarp();
         // completion time base and slope of every model, for the candidates: lane g holds model g
         const int64_t base_e = T + (lane != Lm ? my_sw : 0) + my_al;
@@ -295,10 +343,19 @@ __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const 
                     const bool valid = cb == 0 || bprev < na;      // a larger size with the same members never wins
                     const int bp = b < na ? b : na;
                     const int64_t e = eb + es * (int64_t)bp;
-                    int lo = 0, hi = bp;                           // members with deadline < e are late
-                    while (lo < hi) { const int mid = (lo + hi) >> 1; if (mdl[mid] < e) lo = mid + 1; else hi = mid; }
-                    const double *pj = pref + (size_t)cj * (bmax + 1);
-                    const double u = valid ? pj[bp] - pj[lo] : -INFINITY;
+                    double u = -INFINITY;
+                    if (SOFT && pen != SP_PEN_STEP) {
+                        if (valid) {
+                            u = 0.0;
+                            for (int k = 0; k < bp; ++k)
+                                u += (double)(s_acc[k * Mmax + cj] * penalty_keep_f32(pen, mdl[k], s_delta[k], e));
+                        }
+                    } else {
+                        int lo = 0, hi = bp;                       // members with deadline < e are late
+                        while (lo < hi) { const int mid = (lo + hi) >> 1; if (mdl[mid] < e) lo = mid + 1; else hi = mid; }
+                        const double *pj = pref + (size_t)cj * (bmax + 1);
+                        if (valid) u = pj[bp] - pj[lo];
+                    }
                     cu[q] = u;
                     if (u > bu) { bu = u; bi_ = ci; }
                 }
@@ -368,7 +425,7 @@ __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const 
 
 // Four instances per block, one per warp; the instances a warp cannot finish are then run by the whole block with
 // the block-wide scheduler (the same code as k_sched), while the other blocks of the grid go on with theirs.
-template <int MM, int CPL>
+template <int MM, int CPL, bool SOFT>
 __global__ void __launch_bounds__(kWarpSchedWarps * 32)
 k_sched_warp(SchedParams sp, int cap) {
     extern __shared__ __align__(16) unsigned char dyn[];
@@ -380,15 +437,15 @@ k_sched_warp(SchedParams sp, int cap) {
         if (sp.flags[1]) {                   // request table failed validation: do nothing
             if (lane == 0 && sp.n_done) sp.n_done[inst] = 0;
         } else {
-            const WarpSchedSmem L(cap, sp.P.Mmax, sp.bmax);
-            if (sched_warp_instance<MM, CPL>(sp, cap, inst, dyn + (size_t)warp * L.end)) take = inst;
+            const WarpSchedSmem L(cap, sp.P.Mmax, sp.bmax, SOFT);
+            if (sched_warp_instance<MM, CPL, SOFT>(sp, cap, inst, dyn + (size_t)warp * L.end)) take = inst;
         }
     }
     if (lane == 0) s_takeover[warp] = take;
     __syncthreads();                         // queues and state of a handed-over instance are in global memory
     for (int w = 0; w < kWarpSchedWarps; ++w) {
         if (s_takeover[w] >= 0) {
-            sched_instance<false, (MM <= 8 ? 4 : kMaxApps), false>(sp, s_takeover[w]);   // the warp path runs for step penalties only
+            sched_instance<SOFT, (MM <= 8 ? 4 : kMaxApps), false>(sp, s_takeover[w]);
             __syncthreads();
         }
     }
