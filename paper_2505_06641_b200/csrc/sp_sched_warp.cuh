@@ -153,6 +153,32 @@ __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const 
 
     // ---- requests that are hopeless at the starting clock are retired at once; the others are compacted
     const int64_t emin0 = emin_lane();
+    // Soft penalties: hopeless requests leave from the head of the (deadline, index) order only.  The first key of an
+    // application that is NOT hopeless bounds that prefix, so one pass over the unsorted requests finds it, and the
+    // pass below retires every request ahead of it without sorting them first.
+    int64_t first_dl = INT64_MAX;                        // lane a < A: first non-hopeless key of application a
+    int first_k = 0x7fffffff;
+    if (SOFT) {
+        for (int a = 0; a < A; ++a) {
+            const int pen_a = __shfl_sync(0xffffffffu, my_pen, a);
+            if (pen_a == SP_PEN_STEP) continue;          // uniform
+            const int64_t em = shfl_i64(emin0, a);
+            int64_t bd = INT64_MAX;
+            int bk = 0x7fffffff;
+            for (int k = lane; k < n_inst; k += 32) {
+                if (tb.app[r0 + k] != a) continue;
+                const int64_t dl = tb.deadline[r0 + k];
+                if (!penalty_hopeless(pen_a, dl, dl - tb.arrival[r0 + k], em) && (dl < bd || (dl == bd && k < bk))) { bd = dl; bk = k; }
+            }
+#pragma unroll
+            for (int o = 16; o >= 1; o >>= 1) {
+                const int64_t od = shfl_i64(bd, lane ^ o);
+                const int ok = __shfl_xor_sync(0xffffffffu, bk, o);
+                if (od < bd || (od == bd && ok < bk)) { bd = od; bk = ok; }
+            }
+            if (lane == a) { first_dl = bd; first_k = bk; }
+        }
+    }
     int m = 0;                                           // survivors
     for (int k0 = 0; k0 < n_inst; k0 += 32 * kWarpLoadChunk) {
         int64_t dlv[kWarpLoadChunk];
@@ -169,7 +195,13 @@ __device__ bool sched_warp_instance(const SchedParams &sp, const int cap, const 
             const int k = k0 + u * 32 + lane;
             const int64_t em = shfl_i64(emin0, apv[u] & 31);
             const bool step_app = !SOFT || __shfl_sync(0xffffffffu, my_pen, apv[u] & 31) == SP_PEN_STEP;
-            const bool in = k < n_inst, keep = in && !(step_app && dlv[u] < em);
+            bool gone = step_app && dlv[u] < em;
+            if (SOFT) {                                  // ahead of the application's first request that is not hopeless
+                const int64_t fd = shfl_i64(first_dl, apv[u] & 31);
+                const int fk = __shfl_sync(0xffffffffu, first_k, apv[u] & 31);
+                gone = gone || (!step_app && (dlv[u] < fd || (dlv[u] == fd && k < fk)));
+            }
+            const bool in = k < n_inst, keep = in && !gone;
             if (in && !keep) {
                 sp_req_rec r; r.status = SP_EXPIRED; r.round = round; r.model = -1; r.worker = 0; r.order = 0;
                 tb.recs[r0 + k] = r;
